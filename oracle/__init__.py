@@ -1,0 +1,28 @@
+"""CPU oracle of the expanded W4A4 linear layer: test infrastructure, never the product path.
+
+Thin numpy binding over ``xq_oracle.c`` (plain C, fp64 / int64).  Only the tests, the smoke
+check and the CPU-baseline leg of the benchmark import this package; the CUDA library and its
+Python binding never do, and nothing here imports them.
+"""
+from .xq_oracle import (  # noqa: F401
+    Plan,
+    build,
+    plan,
+    hadamard_dense,
+    hadamard_entry,
+    bf16_to_f64,
+    f64_to_bf16,
+    rotate,
+    rotate_dense,
+    rotate_factored,
+    quantize,
+    pack_int4,
+    unpack_int4,
+    gemm_i64,
+    epilogue,
+    ref_product,
+    prepare_weights,
+    rotate_quant,
+    expanded_linear,
+    num_threads,
+)

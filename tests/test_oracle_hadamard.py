@@ -1,0 +1,172 @@
+"""Pins for the oracle's Hadamard construction and rotation (paper Sec. 3, Remarks 1-2).
+
+Each check is something the paper or the mathematics fixes, not a second copy of the oracle's
+formula: orthogonality with +-1 entries, a library Walsh-Hadamard matrix for the power-of-two
+case, a library Kronecker product for the index convention, the truncated-column norm, energy,
+rank and the rotation invariance of the linear layer.
+"""
+import numpy as np
+import pytest
+import scipy.linalg
+
+from paper_2503_17513_b200 import synth
+
+# (K, Kp): every order-p factor used by the workloads (68, 60, 36, 20, 1) on a small Sylvester
+# factor, plus further Paley orders (12, 28, 76, 140) from the paper's own Table 1 sizes.
+SMALL = [(100, 136), (60, 68), (200, 240), (130, 144), (70, 80), (64, 64), (40, 48), (20, 24),
+         (50, 56), (140, 152), (250, 280), (1, 2), (3, 4)]
+
+
+@pytest.mark.parametrize("K,Kp", SMALL)
+def test_entries_and_orthogonality(oracle, K, Kp):
+    pl = oracle.plan(K, Kp)
+    assert pl.p * (1 << pl.log2n) == Kp
+    H = oracle.hadamard_dense(pl).astype(np.int64)
+    assert set(np.unique(H)) <= {-1, 1}
+    assert np.array_equal(H @ H.T, Kp * np.eye(Kp, dtype=np.int64))  # Sec. 3: H_hat H_hat^T = I with gamma = 1/sqrt(M)
+    assert np.array_equal(H.T @ H, Kp * np.eye(Kp, dtype=np.int64))
+
+
+@pytest.mark.parametrize("K,Kp", [(2048, 2176), (4096, 4608)])
+def test_orthogonality_config_sizes(oracle, K, Kp):
+    pl = oracle.plan(K, Kp)
+    H = oracle.hadamard_dense(pl).astype(np.float64)  # +-1 sums below 2^53 are exact in fp64
+    G = H @ H.T
+    assert np.array_equal(G, Kp * np.eye(Kp))
+
+
+@pytest.mark.parametrize("n", [1, 2, 16, 64, 256])
+def test_power_of_two_is_the_library_walsh_hadamard(oracle, n):
+    pl = oracle.plan(n, n)
+    assert (pl.p, pl.paley_kind) == (1, 0)
+    assert np.array_equal(oracle.hadamard_dense(pl), scipy.linalg.hadamard(n).astype(np.int8))
+
+
+@pytest.mark.parametrize("K,Kp", [(100, 136), (200, 240), (130, 144), (70, 80), (40, 48)])
+def test_kronecker_convention_outer_factor_is_order_p(oracle, K, Kp):
+    """H = H_p (x) S_n with channel c = a * n + b.  H_p is read off H itself (rows/cols with
+    b = 0, where the Sylvester factor is +1) and the whole matrix must equal the library
+    Kronecker product of that block with the library Walsh-Hadamard matrix."""
+    pl = oracle.plan(K, Kp)
+    n = 1 << pl.log2n
+    H = oracle.hadamard_dense(pl).astype(np.int64)
+    Hp = H[::n, ::n]
+    assert Hp.shape == (pl.p, pl.p)
+    assert np.array_equal(Hp @ Hp.T, pl.p * np.eye(pl.p, dtype=np.int64))
+    assert np.array_equal(H, np.kron(Hp, scipy.linalg.hadamard(n)))
+
+
+def test_paley_structure(oracle):
+    """Paley-I (q = 3 mod 4): H - I is skew-symmetric with a +1 first row; Paley-II
+    (q = 1 mod 4): H is symmetric.  Both are textbook properties of the two constructions."""
+    for Kp, kind, q in [(68, 1, 67), (60, 1, 59), (20, 1, 19), (12, 1, 11), (36, 2, 17), (76, 2, 37)]:
+        pl = oracle.plan(Kp, Kp)
+        assert (pl.p, pl.paley_kind, pl.q, pl.log2n) == (Kp, kind, q, 0)
+        H = oracle.hadamard_dense(pl).astype(np.int64)
+        if kind == 1:
+            S = H - np.eye(Kp, dtype=np.int64)
+            assert np.array_equal(S, -S.T)
+            assert np.all(H[0] == 1)
+        else:
+            assert np.array_equal(H, H.T)
+
+
+def test_plan_factors_the_workload_and_paper_sizes(oracle):
+    # the workload sizes: K' = p * 2^k with the stated factors
+    for (K, Kp), want in {
+        (2048, 2176): (68, 5, 1, 67), (8192, 8704): (68, 7, 1, 67), (4096, 4352): (68, 6, 1, 67),
+        (14336, 15360): (60, 8, 1, 59), (4096, 4608): (36, 7, 2, 17), (4096, 5120): (20, 8, 1, 19),
+        (4096, 4096): (1, 12, 0, 0),
+    }.items():
+        pl = oracle.plan(K, Kp)
+        assert (pl.p, pl.log2n, pl.paley_kind, pl.q) == want
+    # Table 1's expanded down-projection sizes are all Hadamard orders that factor over a
+    # prime-field Paley matrix (22016 only through the large order 5504 = 5503 + 1).
+    for K, Kp in [(8192, 8960), (8192, 9728), (8192, 10240), (8192, 12288), (14336, 15360),
+                  (14336, 18432), (14336, 19968)]:
+        pl = oracle.plan(K, Kp)
+        assert pl.p * (1 << pl.log2n) == Kp and pl.paley_kind in (1, 2)
+    pl = oracle.plan(14336, 22016)
+    assert (pl.p, pl.log2n, pl.paley_kind, pl.q) == (5504, 2, 1, 5503)
+    g = np.random.default_rng(0)
+    rows = g.choice(22016, size=6, replace=False)
+    R = np.array([[oracle.hadamard_entry(pl, int(r), c) for c in range(22016)] for r in rows], dtype=np.int64)
+    assert np.array_equal(R @ R.T, 22016 * np.eye(6, dtype=np.int64))
+    with pytest.raises(ValueError):
+        oracle.plan(10, 8)
+    with pytest.raises(ValueError):
+        oracle.plan(4, 6)  # 6 = 3 * 2: no Hadamard matrix of order 6
+
+
+def test_table1_layer_sizes_are_down_proj_in_channels():
+    """Table 1: growing the 16 (1B) / 32 (8B) down projections from 8192 to 8960 (14336 to
+    15360) input channels accounts for the printed model-size increase, so 'layer size' is K'."""
+    assert abs((1.235e9 + 16 * 2048 * (8960 - 8192)) / 1e9 - 1.260) < 1e-3
+    assert abs((7.504e9 + 32 * 4096 * (15360 - 14336)) / 1e9 - 7.638) < 1e-3
+
+
+@pytest.mark.parametrize("K,Kp", [(100, 136), (200, 240), (130, 144), (64, 64), (2048, 2176)])
+def test_truncated_column_norm_energy(oracle, K, Kp):
+    pl = oracle.plan(K, Kp)
+    Hhat = oracle.hadamard_dense(pl, rows=K).astype(np.float64) / np.sqrt(Kp)
+    # Remark 2: every column of H_hat has norm sqrt(N / M)
+    assert np.allclose(np.linalg.norm(Hhat, axis=0), np.sqrt(K / Kp), rtol=1e-13)
+    # Sec. 3: H_hat H_hat^T = I_K
+    assert np.allclose(Hhat @ Hhat.T, np.eye(K), atol=1e-12)
+    x = synth.activations(5, K, seed=3)
+    y = oracle.rotate_dense(pl, x)
+    xf = oracle.bf16_to_f64(x)
+    # the rotation is x @ H_hat (library matmul) and preserves energy (Remark 2)
+    assert np.allclose(y, xf @ Hhat, rtol=0, atol=1e-12 * np.abs(xf).max() * np.sqrt(K))
+    assert np.allclose(np.linalg.norm(y, axis=1), np.linalg.norm(xf, axis=1), rtol=1e-13)
+
+
+def test_rank_preserved_nullity_grows(oracle):
+    """Remark 1: rank(X H_hat) = rank(X), so the nullity grows by M - N."""
+    K, Kp = 20, 24
+    pl = oracle.plan(K, Kp)
+    base = synth.bf16_bits_to_f32(synth.activations(3, K, seed=5))
+    X = np.vstack([base, base[0] + base[1], 2 * base[2], base[0] - base[2]])  # rank 3, 6 rows
+    xb = synth.f32_to_bf16_bits(X.astype(np.float32))
+    Xf = oracle.bf16_to_f64(xb)
+    r = np.linalg.matrix_rank(Xf)
+    y = oracle.rotate_dense(pl, xb)
+    assert np.linalg.matrix_rank(y) == r
+    assert (Kp - np.linalg.matrix_rank(y)) - (K - r) == Kp - K
+
+
+@pytest.mark.parametrize("K,Kp", [(100, 136), (200, 240), (130, 144), (70, 80), (64, 64), (2048, 2176)])
+def test_rotation_invariance(oracle, K, Kp):
+    """Sec. 3: X W = (X H_hat)(H_hat^T W); with out x in storage both operands get the same map."""
+    pl = oracle.plan(K, Kp)
+    x = synth.activations(4, K, seed=1)
+    w = synth.weights(6, K, seed=1)
+    ref = oracle.ref_product(x, w)
+    got = oracle.rotate_dense(pl, x) @ oracle.rotate_dense(pl, w).T
+    assert np.linalg.norm(got - ref) <= 1e-12 * np.linalg.norm(ref)
+
+
+@pytest.mark.parametrize("K,Kp", [(100, 136), (200, 240), (130, 144), (70, 80), (64, 64),
+                                  (2048, 2176), (4096, 4608), (4096, 5120)])
+def test_factored_matches_dense(oracle, K, Kp):
+    pl = oracle.plan(K, Kp)
+    x = synth.activations(3, K, seed=2, heavy_tail=True)
+    yd = oracle.rotate_dense(pl, x)
+    yf = oracle.rotate_factored(pl, x)
+    assert np.linalg.norm(yd - yf) <= 1e-12 * np.linalg.norm(yd)
+
+
+def test_factored_large_shape_energy_and_invariance(oracle):
+    """The largest workload order (15360 = 60 * 256) through the factored form only."""
+    K, Kp = 14336, 15360
+    pl = oracle.plan(K, Kp)
+    x = synth.activations(2, K, seed=4)
+    w = synth.weights(2, K, seed=4)
+    yx, yw = oracle.rotate_factored(pl, x), oracle.rotate_factored(pl, w)
+    xf = oracle.bf16_to_f64(x)
+    assert np.allclose(np.linalg.norm(yx, axis=1), np.linalg.norm(xf, axis=1), rtol=1e-12)
+    ref = oracle.ref_product(x, w)
+    assert np.linalg.norm(yx @ yw.T - ref) <= 1e-11 * np.linalg.norm(ref)
+    # one dense row of the definition as a spot check of the big index arithmetic
+    yd = oracle.rotate_dense(pl, x[:1])
+    assert np.linalg.norm(yd - yx[:1]) <= 1e-12 * np.linalg.norm(yd)
