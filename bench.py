@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the expanded W4A4 linear hot path (rotate+quantize, INT4 GEMM, bf16 epilogue).
+
+One step = one pass of every decoder-layer linear of the workload (all layers, distinct prepared
+weights per layer, so the weight stream is larger than L2) over one batch of M synthetic tokens,
+each linear running xq_rotate_quant then xq_w4a4_gemm through the C ABI.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload 1b-decode|1b-prefill|8b-decode|8b-prefill|sweep] [--tokens M]
+
+With --gpus N > 1 (under torchrun) every rank runs an independent replica (the path has no
+exchange step); the value is the sum over ranks divided by the slowest rank's time.
+--impl reference times the CPU oracle (tests' checker, as it stands) on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_17513_b200 import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (shape table, layers, default M, heavy-tailed activations)
+    "1b-decode": (synth.LLAMA_1B, 16, 32, False),
+    "1b-prefill": (synth.LLAMA_1B, 16, 2048, True),
+    "8b-decode": (synth.LLAMA_8B, 8, 16, False),
+    "8b-prefill": (synth.LLAMA_8B, 4, 4096, True),
+    "sweep": (synth.SWEEP_4096, 4, 8192, True),
+}
+METRIC = "expanded W4A4 linear tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops", 0.0)), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, 1590.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def host_inputs(table, layers, M, heavy):
+    """Seeded host tensors: one activation batch per linear, one weight matrix per (layer, linear).
+    Layers beyond the first reuse the first layer's draws rotated by whole rows (distinct memory, same
+    distribution) to keep host-side generation short."""
+    xs, ws = {}, {}
+    for name, (K, Kp, N) in table.items():
+        xs[name] = synth.activations(M, K, seed=0, tag=name, heavy_tail=heavy)
+        base = synth.weights(N, K, seed=0, tag=name)
+        ws[name] = [np.roll(base, 7 * layer, axis=0) if layer else base for layer in range(layers)]
+    return xs, ws
+
+
+def gemm_bytes(M, K, Kp, N):
+    """Algorithmic HBM bytes of one GEMM launch: packed weights + scales, packed activations + scales, bf16 out."""
+    return N * Kp // 2 + 4 * N + M * (Kp // 2 + 4) + 2 * M * N
+
+
+def rotate_bytes(M, K, Kp):
+    return M * (2 * K + Kp // 2 + 4)
+
+
+def run_reference(args, table, layers, M, heavy):
+    """CPU oracle on the host cores: each step = the online path of ONE layer's linears for min(M, 64) tokens
+    (weights prepared beforehand, as on the GPU); tokens/s scaled to the full layer count."""
+    import oracle
+
+    oracle.build()
+    Ms = min(M, 64)
+    prepared = {}
+    xs = {}
+    for name, (K, Kp, N) in table.items():
+        Ns = min(N, 1024)  # bounded sample of output channels, scaled below
+        pl = oracle.plan(K, Kp)
+        xs[name] = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
+        qw, sw = oracle.prepare_weights(pl, synth.weights(Ns, K, seed=0, tag=name))
+        prepared[name] = (pl, qw, sw, N / Ns)
+
+    def step():
+        t_scaled = 0.0
+        for name in table:
+            pl, qw, sw, scale = prepared[name]
+            t0 = time.perf_counter()
+            _, qx, sx = oracle.rotate_quant(pl, xs[name])
+            t1 = time.perf_counter()
+            acc = oracle.gemm_i64(qx, qw)
+            oracle.epilogue(acc, sx, sw)
+            t2 = time.perf_counter()
+            t_scaled += (t1 - t0) + (t2 - t1) * scale
+        return t_scaled
+
+    for _ in range(args.warmup):
+        step()
+    times = [step() for _ in range(args.steps)]
+    t_layer = sum(times) / len(times)
+    t_step = t_layer * layers * (M / Ms)
+    value = M / t_step
+    sample = (f"online path of one layer's linears for {Ms} tokens, {min(1024, min(v[2] for v in table.values()))}+ output "
+              f"channels per linear (GEMM time scaled to full N), scaled to {layers} layers and M={M}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64/int64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {','.join(table)} x {layers} layers, M={M}"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="1b-decode", choices=sorted(WORKLOADS))
+    ap.add_argument("--tokens", type=int, default=None)
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    table, layers, M, heavy = WORKLOADS[args.workload]
+    M = args.tokens or M
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, table, layers, M, heavy)
+        return
+
+    import torch
+
+    from paper_2503_17513_b200 import xq
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    xq.lib()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # ---- set-up (untimed): inputs, prepared weights, workspaces --------------------------------
+    xs_h, ws_h = host_inputs(table, layers, M, heavy)
+    names = list(table)
+    X = {n: torch.from_numpy(xs_h[n].view(np.int16)).cuda() for n in names}
+    Wt = {n: [xq.xq_prepare_weights(ws_h[n][l], table[n][1]) for l in range(layers)] for n in names}
+    out = {n: torch.empty((M, table[n][2]), dtype=torch.int16, device="cuda") for n in names}
+    wsp = {n: xq.new_workspace(M, Wt[n][0]) for n in names}
+    Xq = {n: torch.empty((M, table[n][1] // 2), dtype=torch.uint8, device="cuda") for n in names}
+    sx = {n: torch.empty((M,), dtype=torch.float32, device="cuda") for n in names}
+    weight_bytes = sum(layers * (table[n][2] * table[n][1] // 2) for n in names)
+    stream = torch.cuda.Stream()
+
+    def step_linear():
+        for l in range(layers):
+            for n in names:
+                xq.xq_expanded_linear(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
+
+    def step_rotate_only():
+        for l in range(layers):
+            for n in names:
+                xq.xq_rotate_quant(X[n], Wt[n][l].plan, Xq[n], sx[n], stream=stream)
+
+    def step_gemm_only():
+        for l in range(layers):
+            for n in names:
+                xq.xq_w4a4_gemm(Xq[n], sx[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
+
+    def make_runner(fn):
+        with torch.cuda.stream(stream):
+            fn()  # eager once (also sets function attributes outside capture)
+            stream.synchronize()
+            if args.no_graph:
+                return fn
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+            return g.replay
+
+    def timed(run, steps, warmup):
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                run()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            stream.synchronize()
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(steps):
+                run()
+            e1.record(stream)
+            stream.synchronize()
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+            return e0.elapsed_time(e1) * 1e-3
+
+    run_main = make_runner(step_linear)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    t_total = timed(run_main, args.steps, args.warmup)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        tt = torch.tensor([t_total], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_total = float(tt.item())
+    t_step = t_total / args.steps
+    value = world * M / t_step
+
+    # ---- per-kernel timing for the roofline (same launch configuration, same stream) ------------
+    n_sub = max(3, min(args.steps, 20))
+    t_rot = timed(make_runner(step_rotate_only), n_sub, 3) / n_sub
+    t_gemm = timed(make_runner(step_gemm_only), n_sub, 3) / n_sub
+    launches_per_step = 2 * layers * len(names)
+    hbm_peak, _, peak_kind = measured_peaks()
+    gbytes = sum(layers * gemm_bytes(M, *table[n]) for n in names)
+    rbytes = sum(layers * rotate_bytes(M, table[n][0], table[n][1]) for n in names)
+    ops = sum(layers * 2 * M * table[n][2] * table[n][1] for n in names)
+    if t_gemm >= t_rot:
+        dom, dbytes, dt = "xq_w4a4_gemm", gbytes, t_gemm
+    else:
+        dom, dbytes, dt = "xq_rotate_quant", rbytes, t_rot
+    achieved = dbytes / dt / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                "peak_source": peak_kind, "traffic": None,
+                "per_kernel": {"xq_w4a4_gemm": {"ms_per_step": t_gemm * 1e3, "GBps": gbytes / t_gemm / 1e9, "TOPS": ops / t_gemm / 1e12},
+                               "xq_rotate_quant": {"ms_per_step": t_rot * 1e3, "GBps": rbytes / t_rot / 1e9}}}
+
+    # ---- end to end through the host-buffer entry point -----------------------------------------
+    Xh = {n: torch.from_numpy(xs_h[n].view(np.int16)).pin_memory() for n in names}
+    Oh = {n: torch.empty((M, table[n][2]), dtype=torch.int16).pin_memory() for n in names}
+
+    def step_host():
+        for l in range(layers):
+            for n in names:
+                xq.xq_expanded_linear_host(Xh[n], Wt[n][l], Oh[n], wsp[n], stream=stream)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    t_e2e = timed(step_host, e2e_steps, 3) / e2e_steps
+    if dist is not None:
+        tt = torch.tensor([t_e2e], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_e2e = float(tt.item())
+    e2e = {"value": world * M / t_e2e, "unit": "tokens/s",
+           "h2d_bytes_per_step": sum(layers * M * table[n][0] * 2 for n in names),
+           "d2h_bytes_per_step": sum(layers * M * table[n][2] * 2 for n in names)}
+
+    for n in names:
+        assert xq.xq_poll_status(wsp[n]) == xq.OK
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline and world == 1:
+        cpu_baseline = cpu_baseline_leg(table, layers, M, heavy)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4xint4->int32",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {','.join(names)} x {layers} layers, M={M}", "tokens": M, "layers": layers,
+                   "weight_bytes": weight_bytes, "l2": "weights of one step exceed L2 (126 MB)" if weight_bytes > 126e6 else
+                   "weights fit in L2", "cuda_graph": not args.no_graph, "parallelism": "replicas" if world > 1 else "single"},
+        "TOPS": ops / t_step / 1e12, "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def cpu_baseline_leg(table, layers, M, heavy):
+    """The oracle, as it stands, on the host cores: online path of one layer's linears for a bounded
+    token and channel sample, scaled linearly (the path is independent per token and per channel)."""
+    import oracle
+
+    oracle.build()
+    Ms = min(M, 32)
+    t_layer = 0.0
+    for name, (K, Kp, N) in table.items():
+        Ns = min(N, 512)
+        pl = oracle.plan(K, Kp)
+        x = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
+        qw, sw = oracle.prepare_weights(pl, synth.weights(Ns, K, seed=0, tag=name))
+        t0 = time.perf_counter()
+        _, qx, sx = oracle.rotate_quant(pl, x)
+        t1 = time.perf_counter()
+        oracle.epilogue(oracle.gemm_i64(qx, qw), sx, sw)
+        t2 = time.perf_counter()
+        t_layer += (t1 - t0) + (t2 - t1) * (N / Ns)
+    t_step = t_layer * layers * (M / Ms)
+    return {"value": M / t_step, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"one layer, {Ms} tokens, up to 512 output channels per linear; scaled to {layers} layers, M={M}, full N"}
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,142 @@
+/*
+ * xq -- expanded W4A4 linear layer for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * The layer (paper Sec. 3, "Post-Training Model Expansion via Online Incoherence
+ * Processing"): an activation row x of K channels is zero-padded to K' channels and rotated by
+ * a Hadamard matrix of order K' scaled by 1/sqrt(K') -- equivalently multiplied by the first K
+ * rows of that matrix, the paper's truncated N x M matrix -- then quantized per token to 4 bits
+ * (Sec. 4, "Quantization Details") and multiplied with weights that were expanded, rotated and
+ * quantized per output channel offline; the product of the two quantized operands is what runs
+ * at inference ("online incoherence processing", Sec. 3).
+ *
+ * Letters: M tokens, K input channels, Kp = K' expanded channels, N output channels.  Weights
+ * are out x in: row n of W is output channel n, and the layer computes x W^T.
+ *
+ * Conventions for every call
+ *  - Returns an xq_status; nothing throws, aborts or traps.  All argument, shape and alignment
+ *    checks run on the host before anything is launched.
+ *  - "dev" pointers are CUDA device pointers of the current device, "host" pointers are host
+ *    memory.  The caller owns every buffer it passes (activations, outputs, workspace); the
+ *    library owns only xq_weights objects, released with xq_weights_free.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls taking a
+ *    stream only enqueue work; they do not synchronize unless stated.
+ *  - bf16 tensors are raw 16-bit patterns.  Device pointers must be 16-byte aligned.
+ *  - No global state: calls on distinct streams with distinct workspaces may run concurrently.
+ */
+#ifndef XQ_H_
+#define XQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  XQ_OK = 0,
+  XQ_ERR_INVALID_ARG = 1,       /* null pointer, non-positive size, misaligned pointer, bad ld */
+  XQ_ERR_UNSUPPORTED_ORDER = 2, /* K' has no Paley (prime field) x Sylvester factorisation the
+                                   kernels support */
+  XQ_ERR_WORKSPACE = 3,         /* workspace missing or smaller than xq_workspace_bytes */
+  XQ_ERR_ALLOC = 4,             /* device or host allocation failed */
+  XQ_ERR_CUDA = 5,              /* a CUDA runtime call or launch failed */
+  XQ_ERR_TIMEOUT = 6,           /* a bounded device-side wait ran out (sticky, see xq_poll_status) */
+  XQ_ERR_BOUNDS = 7             /* device-side self check failed (sticky) */
+} xq_status;
+
+/* Hadamard plan: Kp = p * 2^log2n and H = H_p (x) S_{2^log2n} (Kronecker product, the order-p
+ * factor outermost: channel c = a * 2^log2n + b).  S is the Sylvester matrix
+ * S[b][b'] = (-1)^popcount(b & b'); H_p is a Paley matrix over the prime field GF(q):
+ * paley_kind 1 (q = p - 1 = 3 mod 4) or 2 (q = p/2 - 1 = 1 mod 4); paley_kind 0 means p = 1.
+ * The paper asks only for "an expanded M x M Hadamard matrix" (Sec. 3); this family is the
+ * library's choice of one. */
+typedef struct {
+  int32_t K, Kp, p, log2n, paley_kind, q;
+} xq_hadamard_plan_t;
+
+/* Prepared (expanded, rotated, quantized, packed) weights of one linear layer.  Opaque; lives
+ * in device memory owned by the library. */
+typedef struct xq_weights xq_weights;
+
+/* Factor Kp.  Host only, pure.  p is the smallest odd(Kp) * 2^j (j >= 2) that is a Paley order.
+ * Errors: INVALID_ARG (out == NULL, K < 1, Kp < K, Kp odd and > 1), UNSUPPORTED_ORDER (no such
+ * factor, or p above the kernels' limit of 256). */
+xq_status xq_hadamard_plan(int32_t K, int32_t Kp, xq_hadamard_plan_t* out);
+
+/* Offline step (Sec. 3: expanded weights = truncated-Hadamard^T times W; Sec. 4: per-channel
+ * symmetric 4-bit).  Each of the N rows of W (bf16, HOST, row-major [N, K]) is zero-padded to
+ * Kp, multiplied by H / sqrt(Kp), scaled by absmax / 7, rounded to nearest even, clamped to
+ * [-8, 7] and packed into the device layout the GEMM kernels read.  Allocates device memory,
+ * runs on `stream` and synchronizes it before returning.  *out receives the new object.
+ * Kp must be a multiple of 8 (UNSUPPORTED_ORDER otherwise). */
+xq_status xq_prepare_weights(const void* W_bf16_host, int32_t N, int32_t K, int32_t Kp,
+                             void* stream, xq_weights** out);
+
+/* Build a weights object from already quantized values (HOST): codes int8 [N, Kp] row-major with
+ * values in -8..7 (INVALID_ARG otherwise), s_w float [N].  Synchronizes `stream`. */
+xq_status xq_weights_import(const int8_t* codes_host, const float* s_w_host, int32_t N, int32_t K,
+                            int32_t Kp, void* stream, xq_weights** out);
+
+/* Canonical form back to the HOST: codes int8 [N, Kp], s_w float [N].  Synchronizes. */
+xq_status xq_weights_export(const xq_weights* w, int8_t* codes_host, float* s_w_host);
+
+/* Sizes and plan of a weights object. */
+xq_status xq_weights_info(const xq_weights* w, int32_t* N, int32_t* K, int32_t* Kp,
+                          xq_hadamard_plan_t* plan);
+
+/* Releases the object and its device memory (NULL is allowed). */
+void xq_weights_free(xq_weights* w);
+
+/* Bytes of caller-provided device workspace that xq_w4a4_gemm / xq_expanded_linear(_host) need
+ * for up to M_max tokens against `w`.  0 on bad arguments. */
+size_t xq_workspace_bytes(int32_t M_max, const xq_weights* w);
+
+/* Must be called once on a fresh workspace (zeroes its status word and counters; enqueued on
+ * `stream`). */
+xq_status xq_workspace_init(void* ws_dev, size_t ws_bytes, void* stream);
+
+/* Online step (Sec. 3: expanded activations = X times the truncated Hadamard matrix; Sec. 4:
+ * per-token 4-bit, symmetric in this library).  For each of the M rows of X (bf16, dev,
+ * row-major, row pitch ldx elements, ldx >= K and a multiple of 8):
+ *   y = [x, 0] H / sqrt(Kp);  s_x = max|y| / 7 (1 if the row is zero);
+ *   code = clamp(round_half_even(y / s_x), -8, 7).
+ * Outputs: Xq dev [M, Kp/2] bytes, byte j of a row = code 2j in bits 0-3 and code 2j+1 in bits
+ * 4-7 (two's complement); s_x dev float [M]; if Y_f32_opt != NULL also the rotated values, dev
+ * float [M, Kp] (for stage-wise checking).  M = 0 is a no-op. */
+xq_status xq_rotate_quant(const void* X_bf16_dev, int32_t M, int64_t ldx,
+                          const xq_hadamard_plan_t* plan, uint8_t* Xq_dev, float* s_x_dev,
+                          float* Y_f32_opt_dev, void* stream);
+
+/* Quantized product with dequantizing epilogue (Sec. 3: Q(XR) Q(W~)):
+ *   acc[m][n] = sum_c qx[m][c] * qw[n][c]   (exact, int32)
+ *   out[m][n] = bf16( acc * s_x[m] * s_w[n] ).
+ * Xq, s_x in the xq_rotate_quant format (any nibble -8..7 is accepted).  out dev bf16 [M, N]
+ * row-major.  If acc_opt != NULL the int32 accumulators are also written, dev [M, N].
+ * ws: device workspace of at least xq_workspace_bytes(M, w), initialised once with
+ * xq_workspace_init; concurrent calls need distinct workspaces. */
+xq_status xq_w4a4_gemm(const uint8_t* Xq_dev, const float* s_x_dev, int32_t M, const xq_weights* w,
+                       void* out_bf16_dev, int32_t* acc_opt_dev, void* ws_dev, size_t ws_bytes,
+                       void* stream);
+
+/* The whole layer on device buffers: xq_rotate_quant then xq_w4a4_gemm on `stream`, the
+ * quantized activations staying in the workspace. */
+xq_status xq_expanded_linear(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w,
+                             void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
+/* The whole layer on HOST buffers: copies X (host, [M, K] contiguous; pinned memory makes the
+ * copies asynchronous) into the workspace, runs the layer, copies out (host, bf16 [M, N]) back
+ * and synchronizes `stream` before returning. */
+xq_status xq_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_weights* w,
+                                  void* out_bf16_host, void* ws_dev, size_t ws_bytes, void* stream);
+
+/* Synchronizes `stream` and returns the sticky device status stored in the workspace (XQ_OK,
+ * XQ_ERR_TIMEOUT or XQ_ERR_BOUNDS), or XQ_ERR_CUDA if the stream itself reports an error. */
+xq_status xq_poll_status(const void* ws_dev, void* stream);
+
+const char* xq_status_string(xq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XQ_H_ */

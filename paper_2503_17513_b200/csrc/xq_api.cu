@@ -1,0 +1,344 @@
+// C-ABI entry points of libxq: argument checks, the Hadamard plan, weight objects, workspace
+// bookkeeping.  Every step of the layer itself runs in the kernels of the other files.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "xq_internal.h"
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool prime(int v) {
+  if (v < 2) return false;
+  for (int d = 2; (long long)d * d <= v; ++d)
+    if (v % d == 0) return false;
+  return true;
+}
+
+struct DevBuf {  // scoped device allocation for the offline calls
+  void* p = nullptr;
+  cudaError_t alloc(size_t bytes) { return cudaMalloc(&p, bytes ? bytes : 1); }
+  ~DevBuf() {
+    if (p) cudaFree(p);
+  }
+};
+
+xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
+  xq_hadamard_plan_t pl;
+  xq_status st = xq_hadamard_plan(K, Kp, &pl);
+  if (st != XQ_OK) return st;
+  if (Kp % 8 != 0) return XQ_ERR_UNSUPPORTED_ORDER;  // the GEMM kernels read whole 8-code words
+  xq_weights* w = new (std::nothrow) xq_weights();
+  if (!w) return XQ_ERR_ALLOC;
+  w->N = N;
+  w->K = K;
+  w->Kp = Kp;
+  w->Np = (int32_t)align_up((size_t)N, XQ_ROW_PAD);
+  w->Kpp = (int32_t)align_up((size_t)Kp, XQ_K_BLOCK);
+  w->plan = pl;
+  w->packed = nullptr;
+  w->s_w = nullptr;
+  if (cudaGetDevice(&w->device) != cudaSuccess) {
+    delete w;
+    return XQ_ERR_CUDA;
+  }
+  const size_t bytes = (size_t)w->Np * w->Kpp / 2;
+  if (cudaMalloc((void**)&w->packed, bytes) != cudaSuccess ||
+      cudaMalloc((void**)&w->s_w, sizeof(float) * (size_t)w->Np) != cudaSuccess) {
+    cudaGetLastError();
+    xq_weights_free(w);
+    return XQ_ERR_ALLOC;
+  }
+  *out = w;
+  return XQ_OK;
+}
+
+}  // namespace
+
+xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w) {
+  xq_ws_layout L;
+  size_t off = 0;
+  L.header = off;
+  off += 256;
+  L.xq = off;
+  off += align_up((size_t)M_max * (size_t)(w->Kpp / 2), 256);
+  L.sx = off;
+  off += align_up(sizeof(float) * (size_t)M_max, 256);
+  L.xstage = off;
+  off += align_up((size_t)M_max * (size_t)w->K * 2, 256);
+  L.ostage = off;
+  off += align_up((size_t)M_max * (size_t)w->N * 2, 256);
+  L.partial = off;
+  L.counters = off;
+  L.total = off;
+  return L;
+}
+
+extern "C" {
+
+const char* xq_status_string(xq_status s) {
+  switch (s) {
+    case XQ_OK: return "ok";
+    case XQ_ERR_INVALID_ARG: return "invalid argument";
+    case XQ_ERR_UNSUPPORTED_ORDER: return "unsupported Hadamard order";
+    case XQ_ERR_WORKSPACE: return "workspace missing or too small";
+    case XQ_ERR_ALLOC: return "allocation failed";
+    case XQ_ERR_CUDA: return "CUDA error";
+    case XQ_ERR_TIMEOUT: return "device-side wait timed out";
+    case XQ_ERR_BOUNDS: return "device-side bounds check failed";
+  }
+  return "unknown status";
+}
+
+xq_status xq_hadamard_plan(int32_t K, int32_t Kp, xq_hadamard_plan_t* out) {
+  if (!out || K < 1 || Kp < K) return XQ_ERR_INVALID_ARG;
+  if (Kp > 1 && (Kp & 1)) return XQ_ERR_INVALID_ARG;
+  int odd = Kp, twos = 0;
+  while (!(odd & 1)) {
+    odd >>= 1;
+    ++twos;
+  }
+  xq_hadamard_plan_t pl = {K, Kp, 1, twos, 0, 0};
+  if (odd > 1) {
+    bool found = false;
+    for (int j = 2; j <= twos && !found; ++j) {
+      const long long p = (long long)odd << j;
+      if (p > XQ_MAX_P) break;
+      const int q1 = (int)p - 1, q2 = (int)p / 2 - 1;
+      if (prime(q1) && q1 % 4 == 3) {
+        pl.p = (int)p; pl.log2n = twos - j; pl.paley_kind = 1; pl.q = q1;
+        found = true;
+      } else if (prime(q2) && q2 % 4 == 1) {
+        pl.p = (int)p; pl.log2n = twos - j; pl.paley_kind = 2; pl.q = q2;
+        found = true;
+      }
+    }
+    if (!found) return XQ_ERR_UNSUPPORTED_ORDER;
+  }
+  *out = pl;
+  return XQ_OK;
+}
+
+void xq_weights_free(xq_weights* w) {
+  if (!w) return;
+  if (w->packed) cudaFree(w->packed);
+  if (w->s_w) cudaFree(w->s_w);
+  delete w;
+}
+
+xq_status xq_weights_info(const xq_weights* w, int32_t* N, int32_t* K, int32_t* Kp, xq_hadamard_plan_t* plan) {
+  if (!w) return XQ_ERR_INVALID_ARG;
+  if (N) *N = w->N;
+  if (K) *K = w->K;
+  if (Kp) *Kp = w->Kp;
+  if (plan) *plan = w->plan;
+  return XQ_OK;
+}
+
+xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t Kp, void* stream,
+                             xq_weights** out) {
+  if (!W_host || !out || N < 1 || K < 1 || Kp < K) return XQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  xq_weights* w = nullptr;
+  xq_status s = make_weights(N, K, Kp, &w);
+  if (s != XQ_OK) return s;
+  // Rows of W go through the same pad + rotate + quantize kernel as activation rows (both
+  // operands receive the map v -> [v, 0] H / sqrt(K')), then into the block layout.
+  const int64_t ldw = (int64_t)align_up((size_t)K, 8);
+  DevBuf dW, dCanon;
+  if (dW.alloc((size_t)N * ldw * 2) != cudaSuccess || dCanon.alloc((size_t)N * (Kp / 2)) != cudaSuccess) {
+    cudaGetLastError();
+    xq_weights_free(w);
+    return XQ_ERR_ALLOC;
+  }
+  cudaError_t e = cudaMemcpy2DAsync(dW.p, (size_t)ldw * 2, W_host, (size_t)K * 2, (size_t)K * 2, (size_t)N,
+                                    cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(w->s_w, 0, sizeof(float) * (size_t)w->Np, st);
+  if (e == cudaSuccess)
+    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, st);
+  if (e == cudaSuccess)
+    e = xq_launch_relayout_to_blocks((const uint8_t*)dCanon.p, N, Kp, w->packed, w->Np, w->Kpp, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    xq_weights_free(w);
+    return XQ_ERR_CUDA;
+  }
+  *out = w;
+  return XQ_OK;
+}
+
+xq_status xq_weights_import(const int8_t* codes, const float* s_w, int32_t N, int32_t K, int32_t Kp,
+                            void* stream, xq_weights** out) {
+  if (!codes || !s_w || !out || N < 1 || K < 1 || Kp < K) return XQ_ERR_INVALID_ARG;
+  const size_t count = (size_t)N * Kp;
+  for (size_t i = 0; i < count; ++i)
+    if (codes[i] < -8 || codes[i] > 7) return XQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  xq_weights* w = nullptr;
+  xq_status s = make_weights(N, K, Kp, &w);
+  if (s != XQ_OK) return s;
+  DevBuf dCodes, dCanon;
+  if (dCodes.alloc(count) != cudaSuccess || dCanon.alloc(count / 2) != cudaSuccess) {
+    cudaGetLastError();
+    xq_weights_free(w);
+    return XQ_ERR_ALLOC;
+  }
+  cudaError_t e = cudaMemcpyAsync(dCodes.p, codes, count, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(w->s_w, 0, sizeof(float) * (size_t)w->Np, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(w->s_w, s_w, sizeof(float) * (size_t)N, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = xq_launch_pack_codes((const int8_t*)dCodes.p, (int64_t)(count / 2), (uint8_t*)dCanon.p, st);
+  if (e == cudaSuccess)
+    e = xq_launch_relayout_to_blocks((const uint8_t*)dCanon.p, N, Kp, w->packed, w->Np, w->Kpp, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    xq_weights_free(w);
+    return XQ_ERR_CUDA;
+  }
+  *out = w;
+  return XQ_OK;
+}
+
+xq_status xq_weights_export(const xq_weights* w, int8_t* codes, float* s_w) {
+  if (!w || !codes || !s_w) return XQ_ERR_INVALID_ARG;
+  const size_t count = (size_t)w->N * w->Kp;
+  DevBuf dCodes, dCanon;
+  if (dCodes.alloc(count) != cudaSuccess || dCanon.alloc(count / 2) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_ALLOC;
+  }
+  cudaStream_t st = nullptr;
+  cudaError_t e = xq_launch_relayout_from_blocks(w->packed, w->Np, w->Kpp, (uint8_t*)dCanon.p, w->N, w->Kp, st);
+  if (e == cudaSuccess) e = xq_launch_unpack_codes((const uint8_t*)dCanon.p, (int64_t)(count / 2), (int8_t*)dCodes.p, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(codes, dCodes.p, count, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(s_w, w->s_w, sizeof(float) * (size_t)w->N, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+size_t xq_workspace_bytes(int32_t M_max, const xq_weights* w) {
+  if (!w || M_max < 1) return 0;
+  return xq_ws_compute(M_max, w).total;
+}
+
+xq_status xq_workspace_init(void* ws, size_t ws_bytes, void* stream) {
+  if (!ws || ws_bytes < 256 || !aligned16(ws)) return XQ_ERR_WORKSPACE;
+  if (cudaMemsetAsync(ws, 0, 256, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq,
+                          float* s_x, float* Yopt, void* stream) {
+  if (!plan || M < 0) return XQ_ERR_INVALID_ARG;
+  if (M == 0) return XQ_OK;
+  if (!X || !Xq || !s_x) return XQ_ERR_INVALID_ARG;
+  // the plan must be one xq_hadamard_plan would return
+  xq_hadamard_plan_t chk;
+  xq_status s = xq_hadamard_plan(plan->K, plan->Kp, &chk);
+  if (s != XQ_OK) return s;
+  if (memcmp(&chk, plan, sizeof(chk)) != 0) return XQ_ERR_INVALID_ARG;
+  if (ldx < plan->K || (ldx % 8) != 0) return XQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Xq) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
+      (Yopt && !aligned16(Yopt)))
+    return XQ_ERR_INVALID_ARG;
+  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+xq_status xq_w4a4_gemm(const uint8_t* Xq, const float* s_x, int32_t M, const xq_weights* w, void* out,
+                       int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
+  if (!w || M < 0) return XQ_ERR_INVALID_ARG;
+  if (M == 0) return XQ_OK;
+  if (!Xq || !s_x || !out) return XQ_ERR_INVALID_ARG;
+  if (!aligned16(Xq) || !aligned16(out) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
+      (acc_opt && !aligned16(acc_opt)))
+    return XQ_ERR_INVALID_ARG;
+  const xq_ws_layout L = xq_ws_compute(M, w);
+  if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
+  if (xq_launch_gemm(Xq, s_x, M, w, out, acc_opt, ws, L, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out, void* ws,
+                             size_t ws_bytes, void* stream) {
+  if (!w || M < 0) return XQ_ERR_INVALID_ARG;
+  if (M == 0) return XQ_OK;
+  if (!X || !out) return XQ_ERR_INVALID_ARG;
+  if (ldx < w->K || (ldx % 8) != 0 || !aligned16(X) || !aligned16(out)) return XQ_ERR_INVALID_ARG;
+  const xq_ws_layout L = xq_ws_compute(M, w);
+  if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
+  uint8_t* base = (uint8_t*)ws;
+  uint8_t* Xq = base + L.xq;
+  float* sx = (float*)(base + L.sx);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, st) != cudaSuccess ||
+      xq_launch_gemm(Xq, sx, M, w, out, nullptr, ws, L, st) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+xq_status xq_expanded_linear_host(const void* X_host, int32_t M, const xq_weights* w, void* out_host, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  if (!w || M < 0) return XQ_ERR_INVALID_ARG;
+  if (M == 0) return XQ_OK;
+  if (!X_host || !out_host) return XQ_ERR_INVALID_ARG;
+  const xq_ws_layout L = xq_ws_compute(M, w);
+  if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
+  uint8_t* base = (uint8_t*)ws;
+  cudaStream_t st = (cudaStream_t)stream;
+  // staged rows must stay 16-byte aligned at pitch K
+  if (w->K % 8 != 0) return XQ_ERR_INVALID_ARG;
+  const int64_t ldx = w->K;
+  cudaError_t e = cudaMemcpyAsync(base + L.xstage, X_host, (size_t)M * w->K * 2, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  xq_status s = xq_expanded_linear(base + L.xstage, M, ldx, w, base + L.ostage, ws, ws_bytes, stream);
+  if (s != XQ_OK) return s;
+  e = cudaMemcpyAsync(out_host, base + L.ostage, (size_t)M * w->N * 2, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+xq_status xq_poll_status(const void* ws, void* stream) {
+  if (!ws) return XQ_ERR_WORKSPACE;
+  int32_t word = 0;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  if (word == XQ_ERR_TIMEOUT) return XQ_ERR_TIMEOUT;
+  if (word != 0) return XQ_ERR_BOUNDS;
+  return XQ_OK;
+}
+
+}  // extern "C"

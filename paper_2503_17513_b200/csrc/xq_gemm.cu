@@ -1,0 +1,53 @@
+// Quantized product of the expanded layer (paper Sec. 3: Q(XR) Q(W~), computed at inference)
+// with the dequantizing epilogue: acc = sum_c qx qw (int32, exact), out = bf16(acc s_x s_w).
+#include <cuda_bf16.h>
+
+#include "xq_internal.h"
+
+namespace {
+
+// Nibble split: a word of 8 two's-complement nibbles becomes two words of 4 int8 lanes, each
+// lane 16 x the code (the nibble moved to the top of its byte).  Products of two such lanes
+// are 256 x the code product, removed exactly by an arithmetic shift of the int32 sum.
+__device__ __forceinline__ void split16(uint32_t w, uint32_t& even, uint32_t& odd) {
+  even = (w << 4) & 0xF0F0F0F0u;
+  odd = w & 0xF0F0F0F0u;
+}
+
+// General kernel: one thread per output, any M, N, K' (K' a multiple of 8).  Shape-agnostic
+// path for sizes the tiled kernels do not take.
+__global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __restrict__ Xq, const float* __restrict__ sx, int M,
+                                                           const uint8_t* __restrict__ Wb, const float* __restrict__ sw, int N,
+                                                           int Kp, int k_blocks, __nv_bfloat16* __restrict__ out,
+                                                           int32_t* __restrict__ acc_opt) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int m = blockIdx.y;
+  if (n >= N || m >= M) return;
+  const int words = Kp / 8;
+  const uint32_t* xrow = Xq + (long long)m * words;
+  int acc = 0;
+  for (int kg = 0; kg < words; ++kg) {
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(Wb + xq_weight_word_offset(n, kg, k_blocks));
+    uint32_t we, wo, xe, xo;
+    split16(w, we, wo);
+    split16(xrow[kg], xe, xo);
+    acc = __dp4a((int)we, (int)xe, acc);
+    acc = __dp4a((int)wo, (int)xo, acc);
+  }
+  acc >>= 8;
+  if (acc_opt) acc_opt[(long long)m * N + n] = acc;
+  out[(long long)m * N + n] = __float2bfloat16_rn((float)acc * sx[m] * sw[n]);
+}
+
+}  // namespace
+
+cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+                           int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st) {
+  (void)ws;
+  (void)L;
+  if (w->Kp % 8 != 0) return cudaErrorInvalidValue;
+  dim3 grid((w->N + 127) / 128, M);
+  gemm_general_kernel<<<grid, 128, 0, st>>>((const uint32_t*)Xq, sx, M, w->packed, w->s_w, w->N, w->Kp,
+                                            w->Kpp / XQ_K_BLOCK, (__nv_bfloat16*)out, acc_opt);
+  return cudaGetLastError();
+}

@@ -1,0 +1,72 @@
+// Internal declarations shared by the translation units of libxq (never installed, never
+// included by the oracle).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "xq.h"
+
+// ---------------------------------------------------------------------------------------------
+// Prepared-weights device layout.
+//
+// Codes are grouped in 32-bit words of 8 nibbles; word kg of row n holds codes 8kg..8kg+7 with
+// code 8kg+j in bits 4j..4j+3 (the same nibble order as the activation format).  Words are
+// stored in blocks of 16 rows x 128 codes (1 KiB).  A block is two 512-byte halves of 64 codes;
+// inside a half the 16-byte piece of lane l = 4g + t (g = row mod 8, t = word mod 4) holds the
+// words {(row g, word t), (row g+8, word t), (row g, word t+4), (row g+8, word t+4)}: after the
+// nibble split this is exactly the A-fragment pair of two m16n8k32 integer MMAs, so the decode
+// kernel feeds tensor cores from one 128-bit load per lane, and the prefill kernel expands the
+// same pieces into the shared-memory operand tiles of tcgen05.mma.  Blocks are ordered
+// [row block][k block], k fastest, so all codes of 16 output channels are contiguous.
+// Rows are padded to a multiple of 128 and K' to a multiple of 128 with zero codes.
+// ---------------------------------------------------------------------------------------------
+constexpr int XQ_ROW_BLOCK = 16;
+constexpr int XQ_K_BLOCK = 128;
+constexpr int XQ_BLOCK_BYTES = XQ_ROW_BLOCK * XQ_K_BLOCK / 2;  // 1024
+constexpr int XQ_ROW_PAD = 128;
+
+struct xq_weights {
+  int32_t N, K, Kp;    // logical sizes
+  int32_t Np, Kpp;     // padded sizes (multiples of 128)
+  xq_hadamard_plan_t plan;
+  uint8_t* packed;     // device, Np * Kpp / 2 bytes, block layout above
+  float* s_w;          // device, Np floats (padding rows hold 0)
+  int device;
+};
+
+// Byte offset of the 32-bit word holding codes 8*kg .. 8*kg+7 of row n.
+__host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_blocks) {
+  const int rb = n >> 4, r = n & 15, g = r & 7, hi_row = r >> 3;
+  const int kb = kg >> 4, kin = kg & 15, half = kin >> 3, ks = kin & 7, t = ks & 3, hi_k = ks >> 2;
+  return ((size_t)rb * k_blocks + kb) * XQ_BLOCK_BYTES + (size_t)half * 512 + (size_t)(4 * g + t) * 16 +
+         (size_t)(hi_row + 2 * hi_k) * 4;
+}
+
+// Workspace layout (all offsets multiples of 256 bytes).
+struct xq_ws_layout {
+  size_t header;   // 256 bytes: word 0 = sticky status
+  size_t xq;       // M_max * Kp/2 bytes of packed activations
+  size_t sx;       // M_max floats
+  size_t xstage;   // M_max * K bf16 (host entry point)
+  size_t ostage;   // M_max * N bf16 (host entry point)
+  size_t partial;  // split-K partial accumulators
+  size_t counters; // split-K arrival counters
+  size_t total;
+};
+xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
+
+constexpr int XQ_MAX_P = 256;
+constexpr int XQ_DECODE_MAX_M = 32;
+
+// Launchers (each returns the CUDA error of its launch).
+cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl,
+                                   uint8_t* Xq, float* sx, float* Yopt, cudaStream_t st);
+cudaError_t xq_launch_relayout_to_blocks(const uint8_t* canon, int32_t N, int32_t Kp, uint8_t* blocks,
+                                         int32_t Np, int32_t Kpp, cudaStream_t st);
+cudaError_t xq_launch_relayout_from_blocks(const uint8_t* blocks, int32_t Np, int32_t Kpp, uint8_t* canon,
+                                           int32_t N, int32_t Kp, cudaStream_t st);
+cudaError_t xq_launch_pack_codes(const int8_t* codes, int64_t count_pairs, uint8_t* packed, cudaStream_t st);
+cudaError_t xq_launch_unpack_codes(const uint8_t* packed, int64_t count_pairs, int8_t* codes, cudaStream_t st);
+cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+                           int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st);

@@ -1,0 +1,200 @@
+"""Thin binding over the C-ABI library ``libxq.so``: argument marshalling only.
+
+Function names match ``include/xq.h``.  Tensors are torch CUDA tensors used purely as device
+memory (their ``data_ptr()`` is what crosses the boundary); bf16 data may be passed either as
+``torch.bfloat16`` or as 16-bit integer bit patterns.  There is no fallback: a missing library
+raises at first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libxq.so")
+_lib = None
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_ORDER, ERR_WORKSPACE, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = range(8)
+
+
+class XqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (xq_status {status})")
+
+
+class HadamardPlan(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("K", "Kp", "p", "log2n", "paley_kind", "q")]
+
+    def astuple(self):
+        return (self.K, self.Kp, self.p, self.log2n, self.paley_kind, self.q)
+
+
+EXPORTS = [
+    "xq_status_string", "xq_hadamard_plan", "xq_prepare_weights", "xq_weights_import", "xq_weights_export",
+    "xq_weights_info", "xq_weights_free", "xq_workspace_bytes", "xq_workspace_init", "xq_rotate_quant",
+    "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status",
+]
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2503_17513_b200.build` "
+                "(there is no non-CUDA fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        L.xq_status_string.restype = ctypes.c_char_p
+        L.xq_status_string.argtypes = [ctypes.c_int]
+        L.xq_hadamard_plan.argtypes = [i32, i32, ctypes.POINTER(HadamardPlan)]
+        L.xq_prepare_weights.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.xq_weights_import.argtypes = [vp, vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.xq_weights_export.argtypes = [vp, vp, vp]
+        L.xq_weights_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                      ctypes.POINTER(HadamardPlan)]
+        L.xq_weights_free.argtypes = [vp]
+        L.xq_weights_free.restype = None
+        L.xq_workspace_bytes.argtypes = [i32, vp]
+        L.xq_workspace_bytes.restype = sz
+        L.xq_workspace_init.argtypes = [vp, sz, vp]
+        L.xq_rotate_quant.argtypes = [vp, i32, i64, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp]
+        L.xq_w4a4_gemm.argtypes = [vp, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.xq_expanded_linear.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
+        L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
+        L.xq_poll_status.argtypes = [vp, vp]
+        for name in EXPORTS:
+            if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().xq_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise XqError(status, where)
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dp(t) -> ctypes.c_void_p:
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous()
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _hp(a: np.ndarray) -> ctypes.c_void_p:
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def xq_hadamard_plan(K: int, Kp: int) -> HadamardPlan:
+    pl = HadamardPlan()
+    _check(lib().xq_hadamard_plan(K, Kp, ctypes.byref(pl)), "xq_hadamard_plan")
+    return pl
+
+
+class Weights:
+    """Owner of one ``xq_weights*`` (freed with the object)."""
+
+    def __init__(self, handle: int):
+        self.handle = ctypes.c_void_p(handle)
+        n, k, kp, pl = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32(), HadamardPlan()
+        _check(lib().xq_weights_info(self.handle, ctypes.byref(n), ctypes.byref(k), ctypes.byref(kp), ctypes.byref(pl)),
+               "xq_weights_info")
+        self.N, self.K, self.Kp, self.plan = n.value, k.value, kp.value, pl
+
+    def free(self):
+        if self.handle:
+            lib().xq_weights_free(self.handle)
+            self.handle = ctypes.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def xq_prepare_weights(W_bf16_host: np.ndarray, Kp: int, stream=None) -> Weights:
+    """W: host uint16 bf16 bit patterns [N, K] (out x in)."""
+    W = np.ascontiguousarray(W_bf16_host, dtype=np.uint16)
+    N, K = W.shape
+    h = ctypes.c_void_p()
+    _check(lib().xq_prepare_weights(_hp(W), N, K, Kp, _stream(stream), ctypes.byref(h)), "xq_prepare_weights")
+    return Weights(h.value)
+
+
+def xq_weights_import(codes_host: np.ndarray, s_w_host: np.ndarray, K: int, stream=None) -> Weights:
+    codes = np.ascontiguousarray(codes_host, dtype=np.int8)
+    s_w = np.ascontiguousarray(s_w_host, dtype=np.float32)
+    N, Kp = codes.shape
+    assert s_w.shape == (N,)
+    h = ctypes.c_void_p()
+    _check(lib().xq_weights_import(_hp(codes), _hp(s_w), N, K, Kp, _stream(stream), ctypes.byref(h)), "xq_weights_import")
+    return Weights(h.value)
+
+
+def xq_weights_export(w: Weights):
+    codes = np.empty((w.N, w.Kp), dtype=np.int8)
+    s_w = np.empty((w.N,), dtype=np.float32)
+    _check(lib().xq_weights_export(w.handle, _hp(codes), _hp(s_w)), "xq_weights_export")
+    return codes, s_w
+
+
+def xq_workspace_bytes(M_max: int, w: Weights) -> int:
+    return int(lib().xq_workspace_bytes(M_max, w.handle))
+
+
+def xq_workspace_init(ws: torch.Tensor, stream=None) -> None:
+    _check(lib().xq_workspace_init(_dp(ws), ws.numel() * ws.element_size(), _stream(stream)), "xq_workspace_init")
+
+
+def new_workspace(M_max: int, w: Weights, device="cuda") -> torch.Tensor:
+    """Allocate (with torch) and initialise a workspace for up to M_max tokens."""
+    ws = torch.empty(max(xq_workspace_bytes(M_max, w), 256), dtype=torch.uint8, device=device)
+    xq_workspace_init(ws)
+    return ws
+
+
+def xq_rotate_quant(X, plan: HadamardPlan, Xq, s_x, Y_f32=None, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_rotate_quant(ctypes.c_void_p(X.data_ptr()), M, ldx, ctypes.byref(plan), _dp(Xq), _dp(s_x), _dp(Y_f32),
+                                 _stream(stream)), "xq_rotate_quant")
+
+
+def xq_w4a4_gemm(Xq, s_x, M: int, w: Weights, out, ws, acc=None, stream=None) -> None:
+    _check(lib().xq_w4a4_gemm(_dp(Xq), _dp(s_x), M, w.handle, _dp(out), _dp(acc), _dp(ws), ws.numel() * ws.element_size(),
+                              _stream(stream)), "xq_w4a4_gemm")
+
+
+def xq_expanded_linear(X, w: Weights, out, ws, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_expanded_linear(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _dp(ws),
+                                    ws.numel() * ws.element_size(), _stream(stream)), "xq_expanded_linear")
+
+
+def xq_expanded_linear_host(X_host, w: Weights, out_host, ws, M=None, stream=None) -> None:
+    """X_host / out_host: CPU tensors (pinned for asynchronous copies) of 16-bit elements."""
+    M = X_host.shape[0] if M is None else M
+    _check(lib().xq_expanded_linear_host(ctypes.c_void_p(X_host.data_ptr()), M, w.handle,
+                                         ctypes.c_void_p(out_host.data_ptr()), _dp(ws), ws.numel() * ws.element_size(),
+                                         _stream(stream)), "xq_expanded_linear_host")
+
+
+def xq_poll_status(ws, stream=None) -> int:
+    return int(lib().xq_poll_status(_dp(ws), _stream(stream)))
