@@ -48,6 +48,8 @@ def rel_l2(a, b):
 def run_rotate_quant(xq, x_bits, K, Kp, want_y=True, ldx=None):
     M = x_bits.shape[0]
     pl = xq.xq_hadamard_plan(K, Kp)
+    if ldx is None and K % 8:
+        ldx = (K + 7) // 8 * 8  # row pitch must be a multiple of 8 elements
     if ldx is None:
         X = dev(x_bits)
     else:
@@ -190,7 +192,10 @@ def test_expanded_linear_end_to_end(xq, oracle, M, N, K, Kp, heavy):
     w = xq.xq_prepare_weights(wb, Kp)
     ws = xq.new_workspace(M, w)
     out = torch.empty((M, N), dtype=torch.int16, device="cuda")
-    xq.xq_expanded_linear(dev(x), w, out, ws)
+    ldx = (K + 7) // 8 * 8
+    X = torch.zeros((M, ldx), dtype=torch.int16, device="cuda")
+    X[:, :K] = dev(x)
+    xq.xq_expanded_linear(X, w, out, ws, M=M, ldx=ldx)
     assert xq.xq_poll_status(ws) == xq.OK
     out_ref, _ = oracle.expanded_linear(oracle.plan(K, Kp), x, wb)
     got = synth.bf16_bits_to_f32(host_u16(out))
