@@ -43,7 +43,8 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
   w->plan = pl;
   w->packed = nullptr;
   w->s_w = nullptr;
-  if (cudaGetDevice(&w->device) != cudaSuccess) {
+  if (cudaGetDevice(&w->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&w->sms, cudaDevAttrMultiProcessorCount, w->device) != cudaSuccess) {
     delete w;
     return XQ_ERR_CUDA;
   }
@@ -64,7 +65,7 @@ xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w) {
   xq_ws_layout L;
   size_t off = 0;
   L.header = off;
-  off += 256;
+  off += XQ_WS_HEADER_BYTES;
   L.xq = off;
   off += align_up((size_t)M_max * (size_t)(w->Kpp / 2), 256);
   L.sx = off;
@@ -74,7 +75,7 @@ xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w) {
   L.ostage = off;
   off += align_up((size_t)M_max * (size_t)w->N * 2, 256);
   L.partial = off;
-  L.counters = off;
+  off += align_up(xq_decode_ws_bytes(w, w->sms), 256);
   L.total = off;
   return L;
 }
@@ -160,7 +161,7 @@ xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t K
                                     cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(w->s_w, 0, sizeof(float) * (size_t)w->Np, st);
   if (e == cudaSuccess)
-    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, st);
+    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, nullptr, w->sms, st);
   if (e == cudaSuccess)
     e = xq_launch_relayout_to_blocks((const uint8_t*)dCanon.p, N, Kp, w->packed, w->Np, w->Kpp, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -232,8 +233,8 @@ size_t xq_workspace_bytes(int32_t M_max, const xq_weights* w) {
 }
 
 xq_status xq_workspace_init(void* ws, size_t ws_bytes, void* stream) {
-  if (!ws || ws_bytes < 256 || !aligned16(ws)) return XQ_ERR_WORKSPACE;
-  if (cudaMemsetAsync(ws, 0, 256, (cudaStream_t)stream) != cudaSuccess) {
+  if (!ws || ws_bytes < XQ_WS_HEADER_BYTES || !aligned16(ws)) return XQ_ERR_WORKSPACE;
+  if (cudaMemsetAsync(ws, 0, XQ_WS_HEADER_BYTES, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
@@ -254,7 +255,12 @@ xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadama
   if (!aligned16(X) || !aligned16(Xq) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
       (Yopt && !aligned16(Yopt)))
     return XQ_ERR_INVALID_ARG;
-  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, (cudaStream_t)stream) != cudaSuccess) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, nullptr, sms, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
@@ -290,7 +296,7 @@ xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_wei
   uint8_t* Xq = base + L.xq;
   float* sx = (float*)(base + L.sx);
   cudaStream_t st = (cudaStream_t)stream;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, st) != cudaSuccess ||
+  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, nullptr, w->sms, st) != cudaSuccess ||
       xq_launch_gemm(Xq, sx, M, w, out, nullptr, ws, L, st) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;

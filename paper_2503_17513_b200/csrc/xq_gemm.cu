@@ -43,9 +43,11 @@ __global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __res
 
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st) {
-  (void)ws;
-  (void)L;
   if (w->Kp % 8 != 0) return cudaErrorInvalidValue;
+  int32_t* header = (int32_t*)ws;
+  if (xq_decode_supported(M, w) && w->Np / 16 <= XQ_WS_MAX_ROW_BLOCKS)
+    return xq_launch_gemm_decode(Xq, sx, M, w, out, acc_opt, (int32_t*)((uint8_t*)ws + L.partial),
+                                 header + XQ_WS_COUNTER_OFFSET_WORDS, header, w->sms, st);
   dim3 grid((w->N + 127) / 128, M);
   gemm_general_kernel<<<grid, 128, 0, st>>>((const uint32_t*)Xq, sx, M, w->packed, w->s_w, w->N, w->Kp,
                                             w->Kpp / XQ_K_BLOCK, (__nv_bfloat16*)out, acc_opt);

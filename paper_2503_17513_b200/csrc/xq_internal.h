@@ -33,6 +33,7 @@ struct xq_weights {
   uint8_t* packed;     // device, Np * Kpp / 2 bytes, block layout above
   float* s_w;          // device, Np floats (padding rows hold 0)
   int device;
+  int sms;             // multiprocessors of that device
 };
 
 // Byte offset of the 32-bit word holding codes 8*kg .. 8*kg+7 of row n.
@@ -43,15 +44,19 @@ __host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_blo
          (size_t)(hi_row + 2 * hi_k) * 4;
 }
 
-// Workspace layout (all offsets multiples of 256 bytes).
+// Workspace layout (all offsets multiples of 256 bytes).  The header is what xq_workspace_init
+// clears: word 0 is the sticky status, words 64.. are the split-K arrival counters (one per
+// 16-channel row block; kernels leave them at zero).
+constexpr size_t XQ_WS_HEADER_BYTES = 64 * 1024;
+constexpr int XQ_WS_COUNTER_OFFSET_WORDS = 64;
+constexpr int XQ_WS_MAX_ROW_BLOCKS = (int)(XQ_WS_HEADER_BYTES / 4) - XQ_WS_COUNTER_OFFSET_WORDS;
 struct xq_ws_layout {
-  size_t header;   // 256 bytes: word 0 = sticky status
+  size_t header;   // XQ_WS_HEADER_BYTES
   size_t xq;       // M_max * Kp/2 bytes of packed activations
   size_t sx;       // M_max floats
   size_t xstage;   // M_max * K bf16 (host entry point)
   size_t ostage;   // M_max * N bf16 (host entry point)
   size_t partial;  // split-K partial accumulators
-  size_t counters; // split-K arrival counters
   size_t total;
 };
 xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
@@ -60,13 +65,19 @@ constexpr int XQ_MAX_P = 256;
 constexpr int XQ_DECODE_MAX_M = 32;
 
 // Launchers (each returns the CUDA error of its launch).
+// A8opt (optional): byte-per-code copy of the codes in the operand format of the tcgen05 GEMM, [M, Kp].
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl,
-                                   uint8_t* Xq, float* sx, float* Yopt, cudaStream_t st);
+                                   uint8_t* Xq, float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st);
 cudaError_t xq_launch_relayout_to_blocks(const uint8_t* canon, int32_t N, int32_t Kp, uint8_t* blocks,
                                          int32_t Np, int32_t Kpp, cudaStream_t st);
 cudaError_t xq_launch_relayout_from_blocks(const uint8_t* blocks, int32_t Np, int32_t Kpp, uint8_t* canon,
                                            int32_t N, int32_t Kp, cudaStream_t st);
 cudaError_t xq_launch_pack_codes(const int8_t* codes, int64_t count_pairs, uint8_t* packed, cudaStream_t st);
 cudaError_t xq_launch_unpack_codes(const uint8_t* packed, int64_t count_pairs, int8_t* codes, cudaStream_t st);
+bool xq_decode_supported(int32_t M, const xq_weights* w);
+size_t xq_decode_ws_bytes(const xq_weights* w, int sms);
+cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+                                  int32_t* acc_opt, int32_t* partial, int32_t* counters, int32_t* status, int sms,
+                                  cudaStream_t st);
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st);

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 
 #include "xq_internal.h"
+#include "xq_ptx.cuh"
 
 namespace {
 
@@ -65,7 +66,7 @@ __device__ __forceinline__ int quant_code(float y, float s) {
 __global__ void __launch_bounds__(256) rotate_quant_general_kernel(const __nv_bfloat16* __restrict__ X, int M,
                                                                    long long ldx, xq_hadamard_plan_t pl, float gamma,
                                                                    uint8_t* __restrict__ Xq, float* __restrict__ sx,
-                                                                   float* __restrict__ Yopt) {
+                                                                   float* __restrict__ Yopt, uint8_t* __restrict__ A8opt) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int K = pl.K, Kp = pl.Kp, p = pl.p, n = 1 << pl.log2n, q = pl.q;
   float* bufA = reinterpret_cast<float*>(smem_raw);
@@ -120,10 +121,252 @@ __global__ void __launch_bounds__(256) rotate_quant_general_kernel(const __nv_bf
     for (int j = threadIdx.x; j < Kp / 2; j += blockDim.x) {
       const int lo = quant_code(y[2 * j], s), hi = quant_code(y[2 * j + 1], s);
       out[j] = (uint8_t)((lo & 0xF) | ((hi & 0xF) << 4));
+      if (A8opt) {
+        // operand format of the tcgen05 GEMM: word kg of 8 codes -> 4 bytes of even codes x16, 4 of odd
+        uint8_t* a8 = A8opt + (long long)row * Kp + (j >> 2) * 8 + (j & 3);
+        a8[0] = (uint8_t)(lo << 4);
+        a8[4] = (uint8_t)(hi << 4);
+      }
     }
     if (Yopt)
       for (int c = threadIdx.x; c < Kp; c += blockDim.x) Yopt[(long long)row * Kp + c] = y[c];
     __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tensor-core kernel for p > 1, 32 <= n <= 256, ceil(K / n) <= 64.
+//
+// With the row viewed as V[a][b] (a < p, b < n) the layer needs Y = H_p^T V S_n.  The outer
+// factor goes first, on the raw bf16 inputs: +-1 times bf16 is exact and the sums accumulate in
+// fp32, so H_p^T V runs as m16n8k16 bf16 MMAs (A = H_p^T built from the character table, B = V
+// read from shared memory with a transposing ldmatrix).  Warp (mt, bc) owns 16 rows a' and a
+// chunk of NB = min(n, 128) columns b, so the Sylvester butterflies along b stay inside the
+// warp: bit 0 inside a thread, bits 1-2 across the four lanes of a quad, higher bits across
+// accumulator registers.  For n = 256 the last butterfly crosses the two column chunks through
+// shared memory.  absmax, scale, rounding and nibble packing follow in registers; the packed row
+// leaves through shared memory as 128-bit stores (and, on request, as the byte-per-code operand
+// format of the tcgen05 GEMM).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_ptr) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+
+__device__ __forceinline__ uint32_t sign_bf16(int s) { return s > 0 ? 0x3F80u : (s < 0 ? 0xBF80u : 0u); }
+
+template <int LOG2NB, int KS>
+__global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx,
+                                                              xq_hadamard_plan_t pl, float gamma, uint8_t* __restrict__ Xq,
+                                                              float* __restrict__ sx, float* __restrict__ Yopt,
+                                                              uint8_t* __restrict__ A8opt) {
+  constexpr int NB = 1 << LOG2NB;  // columns per warp
+  constexpr int NT8 = NB / 8;      // n-tiles per warp
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int K = pl.K, Kp = pl.Kp, p = pl.p, n = 1 << pl.log2n, q = pl.q;
+  const int NC = n / NB;            // column chunks (1 or 2)
+  const int pitch = n + 8;          // bf16 elements per staged row (conflict-free ldmatrix)
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int mt = warp / NC, bc = warp - mt * NC;
+  const int nthreads = blockDim.x;
+
+  __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
+  uint32_t* outp = reinterpret_cast<uint32_t*>(Xs + KS * 16 * pitch);  // Kp / 8 words
+  float* red = reinterpret_cast<float*>(outp + Kp / 8);               // 32 floats
+  int8_t* chi2 = reinterpret_cast<int8_t*>(red + 32);
+  int8_t* sq = chi2 + 2 * q + 1;
+  float* exch = reinterpret_cast<float*>(smem_raw + (((size_t)(sq + q - reinterpret_cast<int8_t*>(smem_raw)) + 15) & ~(size_t)15));
+
+  build_chi(q, chi2, sq);
+  xqptx::pdl_launch_dependents();
+  // A = H_p^T, rows a' = 16 mt + {g, g+8}, k = a = 16 ks + {2t, 2t+1, 2t+8, 2t+9}
+  uint32_t afrag[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int a2 = 16 * mt + g + (r & 1) * 8;
+      const int a = 16 * ks + 2 * t + (r >> 1) * 8;
+      uint32_t lo = 0, hi = 0;
+      if (a2 < p) {
+        if (a < p) lo = sign_bf16(paley_sign(pl.paley_kind, q, chi2, a, a2));
+        if (a + 1 < p) hi = sign_bf16(paley_sign(pl.paley_kind, q, chi2, a + 1, a2));
+      }
+      afrag[ks][r] = lo | (hi << 16);
+    }
+  }
+  // zero the staged rows once: rows past the data and the tail of a partial last row stay zero
+  for (int i = tid; i < KS * 16 * pitch / 8; i += nthreads) reinterpret_cast<uint4*>(Xs)[i] = make_uint4(0, 0, 0, 0);
+  xqptx::pdl_wait();
+  __syncthreads();
+
+  const int chunks = K / 8;  // 16-byte pieces of a row
+  for (int row = blockIdx.x; row < M; row += gridDim.x) {
+    const __nv_bfloat16* x = X + (long long)row * ldx;
+    for (int i = tid; i < chunks; i += nthreads) {
+      const int c = 8 * i, a = c >> pl.log2n, b = c & (n - 1);
+      xqptx::cp_async16(Xs + a * pitch + b, x + c);
+    }
+    xqptx::cp_async_wait_all();
+    __syncthreads();
+
+    float acc[NT8][4];
+#pragma unroll
+    for (int j = 0; j < NT8; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const __nv_bfloat16* base = Xs + (16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8) * pitch + bc * NB + ((lane >> 4) & 1) * 8;
+#pragma unroll
+      for (int jp = 0; jp < NT8 / 2; ++jp) {
+        uint32_t bfr[4];
+        ldmatrix_x4_trans(bfr, base + 16 * jp);
+        xqptx::mma_bf16_16x8x16(acc[2 * jp], afrag[ks], bfr[0], bfr[1]);
+        xqptx::mma_bf16_16x8x16(acc[2 * jp + 1], afrag[ks], bfr[2], bfr[3]);
+      }
+    }
+    // Sylvester butterflies along b = 8 j + 2 t + e
+#pragma unroll
+    for (int j = 0; j < NT8; ++j) {
+      const float u0 = acc[j][0], u1 = acc[j][1], u2 = acc[j][2], u3 = acc[j][3];
+      acc[j][0] = u0 + u1; acc[j][1] = u0 - u1; acc[j][2] = u2 + u3; acc[j][3] = u2 - u3;
+    }
+#pragma unroll
+    for (int bit = 1; bit <= 2; ++bit) {
+      const float sgn = (t & bit) ? -1.f : 1.f;
+#pragma unroll
+      for (int j = 0; j < NT8; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float o = __shfl_xor_sync(0xffffffffu, acc[j][e], bit);
+          acc[j][e] = fmaf(sgn, acc[j][e], o);
+        }
+    }
+#pragma unroll
+    for (int s = 1; s < NT8; s <<= 1)
+#pragma unroll
+      for (int j = 0; j < NT8; ++j)
+        if (!(j & s)) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float u = acc[j][e], w = acc[j | s][e];
+            acc[j][e] = u + w;
+            acc[j | s][e] = u - w;
+          }
+        }
+    if (NC == 2) {
+      // last butterfly (bit log2(NB) of b) between the two column chunks
+      float* mine = exch + ((size_t)(16 * mt + g) * n + bc * NB + 2 * t);
+#pragma unroll
+      for (int j = 0; j < NT8; ++j) {
+        *reinterpret_cast<float2*>(mine + 8 * j) = make_float2(acc[j][0], acc[j][1]);
+        *reinterpret_cast<float2*>(mine + 8 * n + 8 * j) = make_float2(acc[j][2], acc[j][3]);
+      }
+      __syncthreads();
+      const float* other = exch + ((size_t)(16 * mt + g) * n + (bc ^ 1) * NB + 2 * t);
+      const float sgn = bc ? -1.f : 1.f;
+#pragma unroll
+      for (int j = 0; j < NT8; ++j) {
+        const float2 o0 = *reinterpret_cast<const float2*>(other + 8 * j);
+        const float2 o1 = *reinterpret_cast<const float2*>(other + 8 * n + 8 * j);
+        acc[j][0] = fmaf(sgn, acc[j][0], o0.x);
+        acc[j][1] = fmaf(sgn, acc[j][1], o0.y);
+        acc[j][2] = fmaf(sgn, acc[j][2], o1.x);
+        acc[j][3] = fmaf(sgn, acc[j][3], o1.y);
+      }
+    }
+    // scale by 1/sqrt(K'), per-token absmax
+    float amax = 0.f;
+#pragma unroll
+    for (int j = 0; j < NT8; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        acc[j][e] *= gamma;
+        amax = fmaxf(amax, fabsf(acc[j][e]));
+      }
+    amax = block_max(amax, red);
+    float s = amax > 0.f ? __fdiv_rn(amax, 7.f) : 1.f;
+    if (!(s > 0.f)) s = 1.f;
+    const float inv = __frcp_rn(s);
+    // quantize, pack: the quad's four bytes of one (row, j) form one word of 8 codes
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int a2 = 16 * mt + g + 8 * r;
+#pragma unroll
+      for (int j = 0; j < NT8; ++j) {
+        const int lo = max(-8, min(7, __float2int_rn(acc[j][2 * r] * inv)));
+        const int hi = max(-8, min(7, __float2int_rn(acc[j][2 * r + 1] * inv)));
+        uint32_t w = (uint32_t)((lo & 0xF) | ((hi & 0xF) << 4)) << (8 * t);
+        w |= __shfl_xor_sync(0xffffffffu, w, 1);
+        w |= __shfl_xor_sync(0xffffffffu, w, 2);
+        if (t == 0 && a2 < p) outp[(a2 * n + bc * NB) / 8 + j] = w;
+      }
+    }
+    if (Yopt) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int a2 = 16 * mt + g + 8 * r;
+        if (a2 < p) {
+          float* yrow = Yopt + (long long)row * Kp + a2 * n + bc * NB + 2 * t;
+#pragma unroll
+          for (int j = 0; j < NT8; ++j) *reinterpret_cast<float2*>(yrow + 8 * j) = make_float2(acc[j][2 * r], acc[j][2 * r + 1]);
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == 0) sx[row] = s;
+    uint4* dst = reinterpret_cast<uint4*>(Xq + (long long)row * (Kp / 2));
+    for (int i = tid; i < Kp / 32; i += nthreads) {
+      const uint4 v = reinterpret_cast<const uint4*>(outp)[i];
+      dst[i] = v;
+      if (A8opt) {
+        uint4 e0, e1;
+        xqptx::split16(v.x, e0.x, e0.y);
+        xqptx::split16(v.y, e0.z, e0.w);
+        xqptx::split16(v.z, e1.x, e1.y);
+        xqptx::split16(v.w, e1.z, e1.w);
+        uint4* d8 = reinterpret_cast<uint4*>(A8opt + (long long)row * Kp);
+        d8[2 * i] = e0;
+        d8[2 * i + 1] = e1;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+template <int LOG2NB, int KS>
+cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
+                      float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+  const int n = 1 << pl.log2n, NB = 1 << LOG2NB, NC = n / NB, MT = (pl.p + 15) / 16;
+  size_t smem = (size_t)KS * 16 * (n + 8) * 2 + (size_t)pl.Kp / 2 + 128 + (size_t)(3 * pl.q + 1) + 32;
+  if (NC == 2) smem += (size_t)MT * 16 * n * 4;
+  auto kern = rotate_quant_tc_kernel<LOG2NB, KS>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const int per_sm = smem > 100 * 1024 ? 1 : (smem > 48 * 1024 ? 2 : 4);
+  const int grid = M < sms * per_sm ? M : sms * per_sm;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(32 * MT * NC);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt);
+}
+
+template <int LOG2NB>
+cudaError_t launch_tc_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
+                         float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+  switch (ks) {
+    case 1: return launch_tc<LOG2NB, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 2: return launch_tc<LOG2NB, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 3: return launch_tc<LOG2NB, 3>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    default: return launch_tc<LOG2NB, 4>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
   }
 }
 
@@ -182,13 +425,26 @@ inline int grid_for(long long work, int threads) {
 }  // namespace
 
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq,
-                                   float* sx, float* Yopt, cudaStream_t st) {
+                                   float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
+  const int n = 1 << pl.log2n;
+  const int rows_a = (pl.K + n - 1) / n;
+  const int MT = (pl.p + 15) / 16;
+  const bool tc = pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 8 && pl.K % 8 == 0 && rows_a <= 64 &&
+                  MT * (n > 128 ? 2 : 1) <= 16;
+  if (tc) {
+    const int ks = (rows_a + 15) / 16;
+    switch (pl.log2n) {
+      case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+      case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+      default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    }
+  }
   const size_t smem = sizeof(float) * (2 * (size_t)pl.Kp + 32) + (size_t)(3 * pl.q + 1) + 16;
   cudaError_t e = cudaFuncSetAttribute(rotate_quant_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int grid = M < 148 * 8 ? M : 148 * 8;
-  rotate_quant_general_kernel<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, M, (long long)ldx, pl, gamma, Xq, sx, Yopt);
+  const int grid = M < sms * 8 ? M : sms * 8;
+  rotate_quant_general_kernel<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt);
   return cudaGetLastError();
 }
 

@@ -164,7 +164,7 @@ def xq_workspace_init(ws: torch.Tensor, stream=None) -> None:
 
 def new_workspace(M_max: int, w: Weights, device="cuda") -> torch.Tensor:
     """Allocate (with torch) and initialise a workspace for up to M_max tokens."""
-    ws = torch.empty(max(xq_workspace_bytes(M_max, w), 256), dtype=torch.uint8, device=device)
+    ws = torch.empty(xq_workspace_bytes(M_max, w), dtype=torch.uint8, device=device)
     xq_workspace_init(ws)
     return ws
 
