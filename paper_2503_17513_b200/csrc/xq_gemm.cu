@@ -3,16 +3,11 @@
 #include <cuda_bf16.h>
 
 #include "xq_internal.h"
+#include "xq_ptx.cuh"
+
+using xqptx::split16;
 
 namespace {
-
-// Nibble split: a word of 8 two's-complement nibbles becomes two words of 4 int8 lanes, each
-// lane 16 x the code (the nibble moved to the top of its byte).  Products of two such lanes
-// are 256 x the code product, removed exactly by an arithmetic shift of the int32 sum.
-__device__ __forceinline__ void split16(uint32_t w, uint32_t& even, uint32_t& odd) {
-  even = (w << 4) & 0xF0F0F0F0u;
-  odd = w & 0xF0F0F0F0u;
-}
 
 // General kernel: one thread per output, any M, N, K' (K' a multiple of 8).  Shape-agnostic
 // path for sizes the tiled kernels do not take.
@@ -48,6 +43,7 @@ cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const 
   if (xq_decode_supported(M, w) && w->Np / 16 <= XQ_WS_MAX_ROW_BLOCKS)
     return xq_launch_gemm_decode(Xq, sx, M, w, out, acc_opt, (int32_t*)((uint8_t*)ws + L.partial),
                                  header + XQ_WS_COUNTER_OFFSET_WORDS, header, w->sms, st);
+  if (xq_prefill_supported(M, w)) return xq_launch_gemm_prefill(Xq, sx, M, w, out, acc_opt, header, w->sms, st);
   dim3 grid((w->N + 127) / 128, M);
   gemm_general_kernel<<<grid, 128, 0, st>>>((const uint32_t*)Xq, sx, M, w->packed, w->s_w, w->N, w->Kp,
                                             w->Kpp / XQ_K_BLOCK, (__nv_bfloat16*)out, acc_opt);

@@ -3,13 +3,17 @@
 // inference; here the case where the weight stream, not the arithmetic, sets the time).
 //
 // Work is cut into 1 KiB units (16 output channels x 128 codes, contiguous in the weight layout,
-// k fastest).  Each of the <= #SM persistent CTAs takes one contiguous range of units -- so the
-// HBM stream of a CTA is one linear run, fetched by a producer warp with bulk copies into a
-// shared-memory ring -- and eight consumer warps turn 512-byte half units into two
-// m16n8k32 integer MMAs per 8 tokens (weights as the 16-row operand, tokens as the 8 columns).
-// A range that ends inside a 16-channel row block leaves a partial sum; the CTAs sharing a row
-// block meet through per-CTA partial slots and an arrival counter, the last one to arrive adds
-// the others' slots and runs the epilogue.  No CTA ever waits for another.
+// k fastest).  Each persistent CTA takes one contiguous range of units -- so its HBM stream is one
+// linear run, fetched by a producer warp with bulk copies into a shared-memory ring of 8 KiB
+// chunks, the first ring-full requested before the kernel waits for its predecessor in the
+// stream.  Eight consumer warps take one unit of every chunk each: two 128-bit loads give a lane
+// the codes of rows g and g+8, the nibble split turns them into the A fragments of four
+// m16n8k32 integer MMAs (weights as the 16-row operand, 8 tokens as the columns).  The token
+// operand is expanded once per CTA into shared memory in fragment order when it fits, else kept
+// packed and split on the fly.  A warp adds its fragment into the CTA's per-row-block tile with
+// shared-memory reductions whenever its unit crosses into another row block.  A row block that
+// spans several CTAs is finished by the last CTA to arrive: contributors publish partial tiles in
+// per-CTA slots and bump an arrival counter; nobody ever waits for another CTA.
 #include <cuda_bf16.h>
 
 #include "xq_internal.h"
@@ -19,10 +23,13 @@ using namespace xqptx;
 
 namespace {
 
-constexpr int kConsumerWarps = 16;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kChunkBytes = 8192;       // 8 units per ring stage
-constexpr int kSubPerChunk = kChunkBytes / 512;
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;
+constexpr int kChunkUnits = kConsumerWarps;                 // one unit per consumer warp
+constexpr int kChunkBytes = kChunkUnits * XQ_BLOCK_BYTES;   // 8 KiB
+constexpr int kMaxStages = 16;
+constexpr int kSlotInts = 16 * 32;
 
 struct DecodeParams {
   const uint8_t* W;
@@ -36,68 +43,31 @@ struct DecodeParams {
   int32_t* status;
   int U;              // units in total (fits 31 bits: checked on the host)
   int M, N, Kp, KB;   // KB = Kp / 128
-  int stages, pitch_words;
-  int split_units;    // 1: ranges cut at any unit (balanced bytes, partial row blocks meet through the slots);
-                      // 0: ranges cut at row blocks only (no partials)
+  int stages;         // ring stages
+  int act_pitch;      // bytes between token rows of the shared-memory token operand
+  int max_tiles;      // row blocks a CTA's range can touch
 };
 
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Wait on an mbarrier phase for at most about one second; on expiry record the time-out in the
-// status word and in the CTA-wide flag so that every later wait returns at once.
-__device__ __forceinline__ void wait_or_flag(uint64_t* bar, uint32_t parity, volatile int* failed, int32_t* status) {
-  if (*failed) return;
-  uint64_t t0 = 0;
-  for (uint32_t i = 0;; ++i) {
-    if (mbar_try_wait(bar, parity)) return;
-    if ((i & 255u) == 255u) {
-      const uint64_t now = globaltimer_ns();
-      if (t0 == 0) t0 = now;
-      if (now - t0 > 1000000000ull || *failed) break;
-    }
-  }
-  *failed = 1;
-  atomicExch(status, (int)XQ_ERR_TIMEOUT);
-}
-
-#ifdef XQ_DECODE_TIMING
-#define TSTAMP(i) do { if (blockIdx.x == XQ_DECODE_TIMING && (threadIdx.x == 0)) ((long long*)(p.status + 16))[i] = clock64(); } while (0)
-#else
-#define TSTAMP(i) do { } while (0)
-#endif
-
-template <int NT>  // token tiles of 8: M <= 8 * NT
+template <int NT, bool PRESPLIT>  // token tiles of 8: M <= 8 * NT
 __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
-  constexpr int MT = 8 * NT;        // padded token count
-  constexpr int RP = MT + 2;        // pitch of the reduction scratch (ints)
+  constexpr int MT = 8 * NT;   // padded token count
+  constexpr int TP = MT + 8;   // pitch of a tile row (ints)
 
   unsigned char* ring = smem;
-  uint32_t* act = reinterpret_cast<uint32_t*>(ring + (size_t)p.stages * kChunkBytes);
-  int* red = reinterpret_cast<int*>(act + (size_t)MT * p.pitch_words);
-  uint64_t* full = reinterpret_cast<uint64_t*>(red + kConsumerWarps * 16 * RP);
+  unsigned char* act = ring + (size_t)p.stages * kChunkBytes;
+  int* tiles = reinterpret_cast<int*>(act + (size_t)MT * p.act_pitch);
+  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)p.max_tiles * 16 * TP);
   uint64_t* empty = full + p.stages;
   uint64_t* actbar = empty + p.stages;
   volatile int* flags = reinterpret_cast<volatile int*>(actbar + 1);  // [0] failed, [1] is_last
 
-  int u0, u1;
-  if (p.split_units) {
-    u0 = (int)((long long)cta * p.U / G);
-    u1 = (int)((long long)(cta + 1) * p.U / G);
-  } else {
-    const int RB = p.U / p.KB;
-    u0 = (int)((long long)cta * RB / G) * p.KB;
-    u1 = (int)((long long)(cta + 1) * RB / G) * p.KB;
-  }
-  const int sb0 = 2 * u0, sb1 = 2 * u1;  // half units (512 B) of this CTA
+  const int u0 = (int)((long long)cta * p.U / G), u1 = (int)((long long)(cta + 1) * p.U / G);
+  const int n_units = u1 - u0;
+  const int rbA = u0 / p.KB;
 
-  TSTAMP(0);
   if (tid < p.stages) {
     mbar_init(&full[tid], 1);
     mbar_init(&empty[tid], kConsumerWarps);
@@ -109,152 +79,200 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   }
   mbar_fence_init();
   __syncthreads();
-  TSTAMP(1);
   pdl_launch_dependents();
 
   if (warp == kConsumerWarps) {
     // ---------------- producer ------------------------------------------------------------------
     // The weights are constants: their first ring-full is requested at once.  The activations
     // may come from the kernel before this one, so they wait for the grid dependency.
-    const long long bytes = (long long)(u1 - u0) * XQ_BLOCK_BYTES;
+    const long long bytes = (long long)n_units * XQ_BLOCK_BYTES;
     const unsigned char* src = p.W + (size_t)u0 * XQ_BLOCK_BYTES;
-    const int chunks = (int)((bytes + kChunkBytes - 1) / kChunkBytes);
-    auto issue = [&](int ci) {
-      const int s = ci % p.stages;
-      if (ci >= p.stages) wait_or_flag(&empty[s], ((ci / p.stages) - 1) & 1, flags, p.status);
+    const int chunks = (n_units + kChunkUnits - 1) / kChunkUnits;
+    int s = 0;
+    uint32_t wrap = 0;  // times the ring index wrapped
+    auto issue = [&](int ci) -> bool {
+      if (ci >= p.stages && !mbar_wait_bounded(&empty[s], (wrap - 1) & 1, flags, p.status, (int)XQ_ERR_TIMEOUT)) return false;
       const long long off = (long long)ci * kChunkBytes;
       const uint32_t n = (uint32_t)min((long long)kChunkBytes, bytes - off);
       mbar_expect_tx(&full[s], n);
       bulk_g2s(ring + (size_t)s * kChunkBytes, src + off, n, &full[s]);
+      if (++s == p.stages) {
+        s = 0;
+        ++wrap;
+      }
+      return true;
     };
     const int first = min(chunks, p.stages);
     if (lane == 0)
       for (int ci = 0; ci < first; ++ci) issue(ci);
     pdl_wait();
-    const uint32_t row_bytes = (uint32_t)(p.Kp / 2);
-    if (lane == 0) mbar_expect_tx(actbar, row_bytes * (uint32_t)p.M);
-    __syncwarp();
-    if (lane < p.M) bulk_g2s(act + (size_t)lane * p.pitch_words, p.Xq + (size_t)lane * row_bytes, row_bytes, actbar);
+    if (!PRESPLIT) {
+      const uint32_t row_bytes = (uint32_t)(p.Kp / 2);
+      if (lane == 0) mbar_expect_tx(actbar, row_bytes * (uint32_t)p.M);
+      __syncwarp();
+      if (lane < p.M) bulk_g2s(act + (size_t)lane * p.act_pitch, p.Xq + (size_t)lane * row_bytes, row_bytes, actbar);
+    }
     if (lane == 0)
-      for (int ci = first; ci < chunks; ++ci) issue(ci);
+      for (int ci = first; ci < chunks; ++ci)
+        if (!issue(ci)) break;
     return;
   }
 
   // ---------------- consumers ------------------------------------------------------------------
-  pdl_wait();  // the workspace (partial slots, counters) may still be in use by the kernel before
-  for (int i = tid; i < (MT - p.M) * p.pitch_words; i += kConsumerWarps * 32)
-    act[(size_t)p.M * p.pitch_words + i] = 0u;  // token rows beyond M
-  TSTAMP(2);
-  wait_or_flag(actbar, 0, flags, p.status);
-  TSTAMP(3);
-  bar_sync(1, kConsumerWarps * 32);
-  TSTAMP(4);
+  for (int i = tid; i < p.max_tiles * 16 * TP; i += kConsumerThreads) tiles[i] = 0;
+  if (PRESPLIT) {
+    // token rows beyond M are zero
+    for (int i = tid; i < (MT - p.M) * (p.act_pitch / 16); i += kConsumerThreads)
+      reinterpret_cast<uint4*>(act + (size_t)p.M * p.act_pitch)[i] = make_uint4(0, 0, 0, 0);
+    pdl_wait();
+    // expand the packed tokens once: a 16-byte piece (words w0..w3) becomes 32 bytes
+    // {even(w0), odd(w0), even(w1), odd(w1) | even(w2), odd(w2), even(w3), odd(w3)}
+    const int pieces = p.Kp / 32;
+    for (int m = warp; m < p.M; m += kConsumerWarps) {
+      const uint4* srow = reinterpret_cast<const uint4*>(p.Xq + (size_t)m * (p.Kp / 2));
+      uint4* drow = reinterpret_cast<uint4*>(act + (size_t)m * p.act_pitch);
+      for (int c = lane; c < pieces; c += 32) {
+        const uint4 v = __ldg(srow + c);
+        uint4 lo, hi;
+        split16(v.x, lo.x, lo.y);
+        split16(v.y, lo.z, lo.w);
+        split16(v.z, hi.x, hi.y);
+        split16(v.w, hi.z, hi.w);
+        drow[2 * c] = lo;
+        drow[2 * c + 1] = hi;
+      }
+    }
+  } else {
+    pdl_wait();  // the workspace (partial slots, counters) may still be in use by the kernel before
+    for (int i = tid; i < (MT - p.M) * (p.act_pitch / 16); i += kConsumerThreads)
+      reinterpret_cast<uint4*>(act + (size_t)p.M * p.act_pitch)[i] = make_uint4(0, 0, 0, 0);
+    mbar_wait_bounded(actbar, 0, flags, p.status, (int)XQ_ERR_TIMEOUT);
+  }
+  bar_sync(1, kConsumerThreads);
 
   const int g = lane >> 2, t = lane & 3;
-  int cur_chunk = -1;
-  const int sbs_per_rb = 2 * p.KB;
-
-  int seg_lo = sb0;
-  while (seg_lo < sb1) {
-    const int rb = seg_lo / sbs_per_rb;
-    const int seg_hi = min(sb1, (rb + 1) * sbs_per_rb);
-    int acc[NT][4], acc2[NT][4];  // two chains per token tile: the MMA latency is long
+  {
+    int acc[NT][2][4];
 #pragma unroll
-    for (int j = 0; j < NT; ++j) {
-      acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0;
-      acc2[j][0] = acc2[j][1] = acc2[j][2] = acc2[j][3] = 0;
-    }
-
-    // this warp's half units: global index congruent to the warp number modulo the warp count
-    int sb = seg_lo + ((warp - (seg_lo & (kConsumerWarps - 1))) & (kConsumerWarps - 1));
-    for (; sb < seg_hi; sb += kConsumerWarps) {
-      const int ci = (sb - sb0) / kSubPerChunk;
-      if (ci != cur_chunk) {
-        if (cur_chunk >= 0) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&empty[cur_chunk % p.stages]);
-        }
-        wait_or_flag(&full[ci % p.stages], (ci / p.stages) & 1, flags, p.status);
-        cur_chunk = ci;
-      }
-#ifdef XQ_DECODE_TIMING
-      const int it_ = (sb - sb0) / kConsumerWarps;
-      if (it_ < 6) TSTAMP(9 + 2 * it_);
-#endif
-      const unsigned char* src = ring + (size_t)(ci % p.stages) * kChunkBytes + (size_t)((sb - sb0) % kSubPerChunk) * 512;
-      const uint4 wv = *reinterpret_cast<const uint4*>(src + lane * 16);
-      uint32_t a0[4], a1[4];
-      split16(wv.x, a0[0], a0[2]);  // (row g   , word t)
-      split16(wv.y, a0[1], a0[3]);  // (row g+8 , word t)
-      split16(wv.z, a1[0], a1[2]);  // (row g   , word t+4)
-      split16(wv.w, a1[1], a1[3]);  // (row g+8 , word t+4)
-      const int kg0 = (sb - rb * sbs_per_rb) * 8;  // first 8-code word of this half unit
+    for (int j = 0; j < NT; ++j)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) acc[j][c][0] = acc[j][c][1] = acc[j][c][2] = acc[j][c][3] = 0;
+    auto flush = [&](int tile_index) {
+      int* tl = tiles + (size_t)tile_index * 16 * TP;
 #pragma unroll
       for (int j = 0; j < NT; ++j) {
-        const uint32_t* xr = act + (size_t)(8 * j + g) * p.pitch_words + kg0 + t;
-        uint32_t b0, b1, b2, b3;
-        split16(xr[0], b0, b1);
-        split16(xr[4], b2, b3);
-        mma_s8_16x8x32(acc[j], a0, b0, b1);
-        mma_s8_16x8x32(acc2[j], a1, b2, b3);
+        atomicAdd(&tl[g * TP + 8 * j + 2 * t], acc[j][0][0] + acc[j][1][0]);
+        atomicAdd(&tl[g * TP + 8 * j + 2 * t + 1], acc[j][0][1] + acc[j][1][1]);
+        atomicAdd(&tl[(g + 8) * TP + 8 * j + 2 * t], acc[j][0][2] + acc[j][1][2]);
+        atomicAdd(&tl[(g + 8) * TP + 8 * j + 2 * t + 1], acc[j][0][3] + acc[j][1][3]);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) acc[j][c][0] = acc[j][c][1] = acc[j][c][2] = acc[j][c][3] = 0;
       }
-#ifdef XQ_DECODE_TIMING
-      if (it_ < 6) { if (acc[0][0] == 0x7fffffff) flags[1] = 5; TSTAMP(10 + 2 * it_); }
-#endif
-    }
+    };
 
-    TSTAMP(5);
-    // ---- fold the eight warps' fragments, then finish or hand over the row block ---------------
-    int* my = red + warp * 16 * RP;
-#pragma unroll
-    for (int j = 0; j < NT; ++j) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[j][e] += acc2[j][e];
-      *reinterpret_cast<int2*>(&my[g * RP + 8 * j + 2 * t]) = make_int2(acc[j][0], acc[j][1]);
-      *reinterpret_cast<int2*>(&my[(g + 8) * RP + 8 * j + 2 * t]) = make_int2(acc[j][2], acc[j][3]);
+    // this warp's units: local index warp, warp + 8, ...; (rb, kb) follow incrementally
+    int kb = (u0 - rbA * p.KB) + warp, rb = rbA;
+    while (kb >= p.KB) {
+      kb -= p.KB;
+      ++rb;
     }
-    bar_sync(1, kConsumerWarps * 32);
-    const bool active = tid < MT * 8;
-    const int m = tid >> 3, np = tid & 7;  // token, pair of output channels
+    int cur_rb = rb, s = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int ul = warp; ul < n_units; ul += kChunkUnits) {
+      if (rb != cur_rb) {
+        flush(cur_rb - rbA);
+        cur_rb = rb;
+      }
+      ok = mbar_wait_bounded(&full[s], phase, flags, p.status, (int)XQ_ERR_TIMEOUT);
+      if (!ok) break;
+      const unsigned char* unit = ring + (size_t)s * kChunkBytes + warp * XQ_BLOCK_BYTES;
+      const uint4 w0 = *reinterpret_cast<const uint4*>(unit + g * 64 + t * 16);        // row g, codes 32t..32t+31
+      const uint4 w1 = *reinterpret_cast<const uint4*>(unit + (g + 8) * 64 + t * 16);  // row g+8
+      uint32_t a[4][4];
+      split16(w0.x, a[0][0], a[0][2]);
+      split16(w1.x, a[0][1], a[0][3]);
+      split16(w0.y, a[1][0], a[1][2]);
+      split16(w1.y, a[1][1], a[1][3]);
+      split16(w0.z, a[2][0], a[2][2]);
+      split16(w1.z, a[2][1], a[2][3]);
+      split16(w0.w, a[3][0], a[3][2]);
+      split16(w1.w, a[3][1], a[3][3]);
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        uint32_t b[4][2];
+        if (PRESPLIT) {
+          const uint4* xr = reinterpret_cast<const uint4*>(act + (size_t)(8 * j + g) * p.act_pitch + kb * 128 + t * 32);
+          const uint4 x0 = xr[0], x1 = xr[1];
+          b[0][0] = x0.x; b[0][1] = x0.y; b[1][0] = x0.z; b[1][1] = x0.w;
+          b[2][0] = x1.x; b[2][1] = x1.y; b[3][0] = x1.z; b[3][1] = x1.w;
+        } else {
+          const uint4 x = *reinterpret_cast<const uint4*>(act + (size_t)(8 * j + g) * p.act_pitch + kb * 64 + t * 16);
+          split16(x.x, b[0][0], b[0][1]);
+          split16(x.y, b[1][0], b[1][1]);
+          split16(x.z, b[2][0], b[2][1]);
+          split16(x.w, b[3][0], b[3][1]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) mma_s8_16x8x32(acc[j][i & 1], a[i], b[i][0], b[i][1]);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);
+      if (++s == p.stages) {
+        s = 0;
+        phase ^= 1u;
+      }
+      kb += kChunkUnits;
+      while (kb >= p.KB) {
+        kb -= p.KB;
+        ++rb;
+      }
+    }
+    if (n_units > warp) flush(cur_rb - rbA);
+  }
+  bar_sync(1, kConsumerThreads);
+
+  // ---------------- finish or hand over every row block of the range -----------------------------
+  const int rbB = (u1 - 1) / p.KB;
+  const bool active = tid < MT * 8;
+  const int m = tid >> 3, np = tid & 7;  // token, pair of output channels
+  for (int rb = rbA; rb <= rbB && n_units > 0; ++rb) {
+    const int* tl = tiles + (size_t)(rb - rbA) * 16 * TP;
     int v0 = 0, v1 = 0;
     if (active) {
-#pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) {
-        v0 += red[w * 16 * RP + (2 * np) * RP + m];
-        v1 += red[w * 16 * RP + (2 * np + 1) * RP + m];
-      }
+      v0 = tl[(2 * np) * TP + m];
+      v1 = tl[(2 * np + 1) * TP + m];
     }
-    TSTAMP(6);
-    const bool whole = (seg_lo == rb * sbs_per_rb) && (seg_hi == (rb + 1) * sbs_per_rb);
+    const bool whole = (long long)rb * p.KB >= u0 && (long long)(rb + 1) * p.KB <= u1;
     bool finish = whole;
     if (!whole) {
       // contributors of this row block: CTAs c_first..c_last (c(u) = largest c with u0(c) <= u)
       const long long ua = (long long)rb * p.KB, ub = (long long)(rb + 1) * p.KB - 1;
       const int c_first = (int)(((ua + 1) * G - 1) / p.U), c_last = (int)(((ub + 1) * G - 1) / p.U);
-      int32_t* slot = p.partial + ((size_t)rb + cta) * (16 * 32);
+      int32_t* slot = p.partial + ((size_t)rb + cta) * kSlotInts;
       if (active) *reinterpret_cast<int2*>(&slot[2 * tid]) = make_int2(v0, v1);
-      bar_sync(1, kConsumerWarps * 32);
+      bar_sync(1, kConsumerThreads);
       if (tid == 0) {
         __threadfence();  // cumulative: publishes the whole CTA's slot (ordered by the barrier)
         const int old = atomicAdd(&p.counters[rb], 1);
         __threadfence();
         flags[1] = (old == c_last - c_first) ? 1 : 0;
       }
-      bar_sync(1, kConsumerWarps * 32);
+      bar_sync(1, kConsumerThreads);
       finish = flags[1] != 0;
       if (finish) {
         if (active) {
           for (int c = c_first; c <= c_last; ++c) {
             if (c == cta) continue;
-            const int2 o = __ldcg(reinterpret_cast<const int2*>(p.partial + ((size_t)rb + c) * (16 * 32) + 2 * tid));
+            const int2 o = __ldcg(reinterpret_cast<const int2*>(p.partial + ((size_t)rb + c) * kSlotInts + 2 * tid));
             v0 += o.x;
             v1 += o.y;
           }
         }
         if (tid == 0) p.counters[rb] = 0;  // ready for the next launch
       }
+      bar_sync(1, kConsumerThreads);  // flags[1] is reused by the next partial row block
     }
-    TSTAMP(7);
     if (finish && active && m < p.M) {
       v0 >>= 8;  // every product carries 16 x 16
       v1 >>= 8;
@@ -278,15 +296,47 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         }
       }
     }
-    bar_sync(1, kConsumerWarps * 32);  // scratch and flags are reused by the next segment
-    TSTAMP(8);
-    seg_lo = seg_hi;
   }
 }
 
-template <int NT>
+struct DecodePlan {
+  int nt, stages, act_pitch, max_tiles, grid;
+  bool presplit;
+  size_t smem;
+};
+
+// Shared-memory plan for M tokens on `sms` multiprocessors; stages == 0 means it does not fit.
+DecodePlan decode_plan(int M, const xq_weights* w, int sms) {
+  DecodePlan d = {};
+  d.nt = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
+  const int MT = 8 * d.nt, KB = w->Kp / 128;
+  const long long U = (long long)(w->Np / 16) * KB;
+  d.grid = (int)(U < sms ? U : sms);
+  const long long per_cta = (U + d.grid - 1) / d.grid;
+  d.max_tiles = (int)(per_cta / KB) + 2;
+  const size_t tiles = (size_t)d.max_tiles * 16 * (MT + 8) * 4;
+  const size_t misc = (2 * kMaxStages + 1) * 8 + 64 + 128;
+  const size_t cap = 227 * 1024;
+  const int want = (int)((per_cta + kChunkUnits - 1) / kChunkUnits);  // chunks of the longest range
+  // row pitches that keep the 128-bit fragment reads of eight token rows on distinct banks
+  const int pitch_split = w->Kp + 16, pitch_packed = w->Kp / 2 + ((w->Kp / 2) % 128 == 0 ? 64 : 0);
+  const size_t act_split = (size_t)MT * pitch_split, act_packed = (size_t)MT * pitch_packed;
+  const size_t min_ring = 4 * (size_t)kChunkBytes;
+  d.presplit = act_split + tiles + misc + min_ring <= cap;
+  const size_t actb = d.presplit ? act_split : act_packed;
+  d.act_pitch = d.presplit ? pitch_split : pitch_packed;
+  if (actb + tiles + misc + 2 * (size_t)kChunkBytes > cap) return d;  // stages == 0
+  int s = (int)((cap - actb - tiles - misc) / kChunkBytes);
+  if (s > kMaxStages) s = kMaxStages;
+  if (s > want) s = want < 2 ? 2 : want;
+  d.stages = s;
+  d.smem = actb + tiles + misc + (size_t)s * kChunkBytes;
+  return d;
+}
+
+template <int NT, bool PRESPLIT>
 cudaError_t launch_nt(const DecodeParams& p, int grid, size_t smem, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<NT, PRESPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
@@ -298,46 +348,26 @@ cudaError_t launch_nt(const DecodeParams& p, int grid, size_t smem, cudaStream_t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<NT>, p);
+  return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<NT, PRESPLIT>, p);
 }
 
 }  // namespace
 
-// Shared-memory plan of the decode kernel for M tokens; stages == 0 means it does not fit.
-static void decode_smem_plan(int M, int Kp, int* stages, int* pitch_words, size_t* bytes) {
-  const int MT = M <= 8 ? 8 : (M <= 16 ? 16 : 32);
-  int pitch = Kp / 8;
-  pitch += ((4 - pitch) % 32 + 32) % 32;  // pitch = 4 (mod 32): conflict-free fragment reads
-  const size_t act = (size_t)MT * pitch * 4;
-  const size_t red = (size_t)kConsumerWarps * 16 * (MT + 2) * 4;
-  const size_t fixed = act + red + 8 /*act barrier*/ + 64 /*flags*/ + 128 /*alignment slack*/;
-  const size_t cap = 227 * 1024;
-  int s = 0;
-  if (fixed + 2 * (kChunkBytes + 16) <= cap) {
-    s = (int)((cap - fixed) / (kChunkBytes + 16));
-    if (s > 24) s = 24;
-  }
-  *stages = s;
-  *pitch_words = pitch;
-  *bytes = fixed + (size_t)s * (kChunkBytes + 16);
-}
-
 bool xq_decode_supported(int32_t M, const xq_weights* w) {
   if (M < 1 || M > XQ_DECODE_MAX_M || w->Kp % 128 != 0) return false;
-  int s, pw;
-  size_t b;
-  decode_smem_plan(M, w->Kp, &s, &pw, &b);
-  return s >= 2;
+  if ((long long)(w->Np / 16) * (w->Kp / 128) > 0x7fffffffLL) return false;
+  return decode_plan(M, w, w->sms).stages >= 2;
 }
 
 size_t xq_decode_ws_bytes(const xq_weights* w, int sms) {
   const size_t rbs = (size_t)w->Np / 16;
-  return (rbs + sms) * 16 * 32 * sizeof(int32_t);
+  return (rbs + sms) * kSlotInts * sizeof(int32_t);
 }
 
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                                   int32_t* acc_opt, int32_t* partial, int32_t* counters, int32_t* status, int sms,
                                   cudaStream_t st) {
+  const DecodePlan d = decode_plan(M, w, sms);
   DecodeParams p;
   p.W = w->packed;
   p.sw = w->s_w;
@@ -350,15 +380,18 @@ cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M,
   p.status = status;
   p.KB = w->Kp / 128;
   p.U = (w->Np / 16) * p.KB;
-  p.split_units = 0;
   p.M = M;
   p.N = w->N;
   p.Kp = w->Kp;
-  size_t smem;
-  decode_smem_plan(M, w->Kp, &p.stages, &p.pitch_words, &smem);
-  const int RB = w->Np / 16;
-  const int grid = RB < sms ? RB : sms;
-  if (M <= 8) return launch_nt<1>(p, grid, smem, st);
-  if (M <= 16) return launch_nt<2>(p, grid, smem, st);
-  return launch_nt<4>(p, grid, smem, st);
+  p.stages = d.stages;
+  p.act_pitch = d.act_pitch;
+  p.max_tiles = d.max_tiles;
+  if (d.presplit) {
+    if (d.nt == 1) return launch_nt<1, true>(p, d.grid, d.smem, st);
+    if (d.nt == 2) return launch_nt<2, true>(p, d.grid, d.smem, st);
+    return launch_nt<4, true>(p, d.grid, d.smem, st);
+  }
+  if (d.nt == 1) return launch_nt<1, false>(p, d.grid, d.smem, st);
+  if (d.nt == 2) return launch_nt<2, false>(p, d.grid, d.smem, st);
+  return launch_nt<4, false>(p, d.grid, d.smem, st);
 }

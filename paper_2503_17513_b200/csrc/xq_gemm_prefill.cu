@@ -1,0 +1,337 @@
+// Prefill-shape W4A4 GEMM (many tokens): the quantized product Q(XR) Q(W~) of the paper's Sec. 3
+// as a dense integer contraction on the fifth-generation tensor cores.
+//
+// Tile: 128 tokens x 256 output channels, K in blocks of 128 codes.  A persistent CTA per SM
+// walks its tiles with four kinds of warps:
+//   producer (1 warp)   TMA: the packed activation tile (tensor map over the [M, K'/2] byte
+//                       matrix, out-of-range rows and columns read as zero) and sixteen 1 KiB
+//                       bulk copies of packed weights per K block, into a ring of packed stages;
+//   unpack   (8 warps)  expand packed nibbles to signed bytes (16 x the code: the nibble moved
+//                       to the top of its byte) and write them into the 128-byte-swizzled
+//                       K-major operand stages that tcgen05.mma reads;
+//   mma      (1 warp)   one thread issues tcgen05.mma kind::i8, 128 x 256 x 32 per instruction,
+//                       int32 accumulators in tensor memory (two buffers of 256 columns);
+//   epilogue (4 warps)  tcgen05.ld the finished accumulator, remove the factor 256 exactly,
+//                       multiply by the per-token and per-channel scales, write bf16.
+// Inside a word of eight codes the even positions come first after expansion (0,2,4,6,1,3,5,7);
+// activations and weights are expanded by the same rule, so the sum over K is unchanged.
+// All barrier waits are time-bounded: on expiry the CTA records XQ_ERR_TIMEOUT in the workspace
+// status word, every role leaves its loop, and tensor memory is released before exit.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "xq_internal.h"
+#include "xq_ptx.cuh"
+
+using namespace xqptx;
+
+namespace {
+
+constexpr int BM = 128, BN = 256;
+constexpr int kPkStages = 4, kI8Stages = 2;
+constexpr int kPkABytes = BM * 64, kPkBBytes = BN * 64;     // packed: 8 KiB + 16 KiB
+constexpr int kI8ABytes = BM * 128, kI8BBytes = BN * 128;   // expanded: 16 KiB + 32 KiB
+constexpr int kPkStageBytes = kPkABytes + kPkBBytes;
+constexpr int kI8StageBytes = kI8ABytes + kI8BBytes;
+constexpr int kUnpackWarps = 8, kEpiWarps = 4;
+constexpr int kFirstEpiWarp = 2, kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
+constexpr int kThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;  // 448
+constexpr int kTmemCols = 512;
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kI8Stages * kI8StageBytes + (size_t)kPkStages * kPkStageBytes +
+                              kEpiWarps * BN * sizeof(float) + 256 /*barriers, flags*/;
+
+struct PrefillParams {
+  const uint8_t* W;    // block layout
+  const float* sw;
+  const float* sx;
+  __nv_bfloat16* out;
+  int32_t* acc_opt;
+  int32_t* status;
+  int M, N, KB;        // KB = K'' / 128 (k blocks of the padded weights)
+  int tiles_m, tiles_n;
+};
+
+// Expand one 16-byte piece (32 codes of one row) and store it as two 16-byte pieces of the
+// swizzled 128-byte row `r` (pieces 2j and 2j+1 before the XOR with r mod 8).
+__device__ __forceinline__ void expand_store(const uint4 v, unsigned char* tile, int r, int j) {
+  uint4 lo, hi;
+  split16(v.x, lo.x, lo.y);
+  split16(v.y, lo.z, lo.w);
+  split16(v.z, hi.x, hi.y);
+  split16(v.w, hi.z, hi.w);
+  unsigned char* row = tile + r * 128;
+  const int x = r & 7;
+  *reinterpret_cast<uint4*>(row + (((2 * j) ^ x) << 4)) = lo;
+  *reinterpret_cast<uint4*>(row + (((2 * j + 1) ^ x) << 4)) = hi;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap mapA, const PrefillParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  unsigned char* base = smem_raw + (((raw + 1023u) & ~1023u) - raw);
+  unsigned char* i8 = base;                                         // kI8Stages x [A 16 KiB | B 32 KiB], 1024-aligned
+  unsigned char* pk = i8 + (size_t)kI8Stages * kI8StageBytes;       // kPkStages x [A 8 KiB | B 16 KiB]
+  float* sw_tile = reinterpret_cast<float*>(pk + (size_t)kPkStages * kPkStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sw_tile + kEpiWarps * BN);
+  uint64_t* pk_full = bars;
+  uint64_t* pk_empty = pk_full + kPkStages;
+  uint64_t* i8_full = pk_empty + kPkStages;
+  uint64_t* i8_empty = i8_full + kI8Stages;
+  uint64_t* acc_full = i8_empty + kI8Stages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint64_t* drain = acc_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tiles = p.tiles_m * p.tiles_n;
+
+  if (tid == 0) {
+    for (int s = 0; s < kPkStages; ++s) {
+      mbar_init(&pk_full[s], 1);
+      mbar_init(&pk_empty[s], kUnpackWarps);
+    }
+    for (int s = 0; s < kI8Stages; ++s) {
+      mbar_init(&i8_full[s], kUnpackWarps);
+      mbar_init(&i8_empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], kEpiWarps);
+    }
+    mbar_init(drain, 1);
+    *failed = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&mapA);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();
+  pdl_wait();  // activations and their scales may come from the kernel before this one
+
+  if (warp == 0) {
+    // ---------------- producer ------------------------------------------------------------------
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+      const unsigned char* wsrc = p.W + ((size_t)(tn * (BN / 16) + (lane & 15)) * p.KB) * XQ_BLOCK_BYTES;
+      for (int kb = 0; kb < p.KB; ++kb, ++it) {
+        const int s = it % kPkStages;
+        if (it >= (uint32_t)kPkStages) {
+          ok = mbar_wait_bounded(&pk_empty[s], ((it / kPkStages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+          if (!ok) break;
+        }
+        unsigned char* stage = pk + (size_t)s * kPkStageBytes;
+        if (lane == 0) {
+          mbar_expect_tx(&pk_full[s], kPkStageBytes);
+          tma_load_2d(stage, &mapA, kb * 64, tm * BM, &pk_full[s]);
+        }
+        __syncwarp();
+        if (lane < 16) bulk_g2s(stage + kPkABytes + lane * XQ_BLOCK_BYTES, wsrc + (size_t)kb * XQ_BLOCK_BYTES, XQ_BLOCK_BYTES, &pk_full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issue -----------------------------------------------------------------
+    constexpr uint32_t idesc = umma_idesc_s8(BM, BN);
+    uint32_t it = 0, tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
+      const uint32_t buf = tcount & 1u;
+      if (tcount >= 2u) {
+        ok = mbar_wait_bounded(&acc_empty[buf], ((tcount >> 1) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+        if (!ok) break;
+      }
+      tc_fence_after_sync();
+      const uint32_t d_tmem = tmem_base + buf * BN;
+      for (int kb = 0; kb < p.KB; ++kb, ++it) {
+        const int u = it % kI8Stages;
+        ok = mbar_wait_bounded(&i8_full[u], (it / kI8Stages) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+        if (!ok) break;
+        tc_fence_after_sync();
+        if (lane == 0) {
+          const uint32_t a_addr = smem_u32(i8 + (size_t)u * kI8StageBytes);
+          const uint64_t adesc = umma_desc_k128(a_addr), bdesc = umma_desc_k128(a_addr + kI8ABytes);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) umma_i8_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit(&i8_empty[u]);
+        }
+        __syncwarp();
+      }
+      if (ok && lane == 0) umma_commit(&acc_full[buf]);
+      __syncwarp();
+    }
+    // every MMA issued by this warp has completed before tensor memory is released
+    if (lane == 0) umma_commit(drain);
+    __syncwarp();
+    mbar_wait_bounded(drain, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);
+  } else if (warp < kFirstUnpackWarp) {
+    // ---------------- epilogue ------------------------------------------------------------------
+    const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    float* sw_mine = sw_tile + (warp - kFirstEpiWarp) * BN;  // a private copy per warp: no cross-warp barrier
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
+      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+      const uint32_t buf = tcount & 1u;
+      const int n0 = tn * BN;
+      __syncwarp();
+      for (int i = lane; i < BN; i += 32) sw_mine[i] = (n0 + i < p.N) ? p.sw[n0 + i] : 0.f;
+      __syncwarp();
+      const int m = tm * BM + q * 32 + lane;
+      const float sxm = m < p.M ? p.sx[m] : 0.f;
+      ok = mbar_wait_bounded(&acc_full[buf], (tcount >> 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(taddr + c * 32, v);
+        tmem_ld_wait();
+        const int nc = n0 + c * 32;
+        if (m < p.M && nc < p.N) {
+          const size_t o = (size_t)m * p.N + nc;
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            if (nc + 8 * g8 < p.N) {  // N is a multiple of 8 on this path
+              int a[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) a[e] = (int)v[8 * g8 + e] >> 8;  // every product carries 16 x 16
+              if (p.acc_opt) {
+                *reinterpret_cast<int4*>(p.acc_opt + o + 8 * g8) = make_int4(a[0], a[1], a[2], a[3]);
+                *reinterpret_cast<int4*>(p.acc_opt + o + 8 * g8 + 4) = make_int4(a[4], a[5], a[6], a[7]);
+              }
+              uint32_t h[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float f0 = (float)a[2 * e] * sxm * sw_mine[c * 32 + 8 * g8 + 2 * e];
+                const float f1 = (float)a[2 * e + 1] * sxm * sw_mine[c * 32 + 8 * g8 + 2 * e + 1];
+                const __nv_bfloat162 b2 = __halves2bfloat162(__float2bfloat16_rn(f0), __float2bfloat16_rn(f1));
+                h[e] = *reinterpret_cast<const uint32_t*>(&b2);
+              }
+              *reinterpret_cast<uint4*>(p.out + o + 8 * g8) = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
+    }
+  } else {
+    // ---------------- unpack --------------------------------------------------------------------
+    const int ut = tid - kFirstUnpackWarp * 32;  // 0..255
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+      for (int kb = 0; kb < p.KB; ++kb, ++it) {
+        const int s = it % kPkStages, u = it % kI8Stages;
+        ok = mbar_wait_bounded(&pk_full[s], (it / kPkStages) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+        if (!ok) break;
+        if (it >= (uint32_t)kI8Stages) {
+          ok = mbar_wait_bounded(&i8_empty[u], ((it / kI8Stages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+          if (!ok) break;
+        }
+        const unsigned char* src = pk + (size_t)s * kPkStageBytes;   // [A rows | B rows], 64 bytes per row
+        unsigned char* dstA = i8 + (size_t)u * kI8StageBytes;
+        unsigned char* dstB = dstA + kI8ABytes;
+        constexpr int kPieces = (BM + BN) * 4 / (kUnpackWarps * 32);  // 16-byte pieces per thread: 6
+        uint4 v[kPieces];
+#pragma unroll
+        for (int i = 0; i < kPieces; ++i) v[i] = *reinterpret_cast<const uint4*>(src + (size_t)(ut + i * kUnpackWarps * 32) * 16);
+#pragma unroll
+        for (int i = 0; i < kPieces; ++i) {
+          const int piece = ut + i * kUnpackWarps * 32, r = piece >> 2, j = piece & 3;
+          if (r < BM) expand_store(v[i], dstA, r, j);
+          else expand_store(v[i], dstB, r - BM, j);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&i8_full[u]);
+          mbar_arrive(&pk_empty[s]);
+        }
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0 && *failed) {
+    // bounded drain of copies that may still be landing in this CTA's shared memory
+    for (int s = 0; s < kPkStages; ++s) mbar_wait(&pk_full[s], 0, 1u << 16), mbar_wait(&pk_full[s], 1, 1u << 16);
+  }
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return (EncodeTiledFn)f;
+  }();
+  return fn;
+}
+
+}  // namespace
+
+bool xq_prefill_supported(int32_t M, const xq_weights* w) {
+  return M >= 1 && w->Kp % 32 == 0 && w->N % 8 == 0 && w->Np % BN == 0;
+}
+
+cudaError_t xq_launch_gemm_prefill(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+                                   int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return cudaErrorNotSupported;
+  CUtensorMap mapA;
+  const cuuint64_t dims[2] = {(cuuint64_t)(w->Kp / 2), (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)(w->Kp / 2)};
+  const cuuint32_t box[2] = {64, (cuuint32_t)BM};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)Xq, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  PrefillParams p;
+  p.W = w->packed;
+  p.sw = w->s_w;
+  p.sx = sx;
+  p.out = (__nv_bfloat16*)out;
+  p.acc_opt = acc_opt;
+  p.status = status;
+  p.M = M;
+  p.N = w->N;
+  p.KB = w->Kpp / XQ_K_BLOCK;
+  p.tiles_m = (M + BM - 1) / BM;
+  p.tiles_n = (w->N + BN - 1) / BN;
+  cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (e != cudaSuccess) return e;
+  const int tiles = p.tiles_m * p.tiles_n;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles < sms ? tiles : sms);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_prefill_kernel, mapA, p);
+}

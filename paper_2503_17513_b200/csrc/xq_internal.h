@@ -10,25 +10,23 @@
 // ---------------------------------------------------------------------------------------------
 // Prepared-weights device layout.
 //
-// Codes are grouped in 32-bit words of 8 nibbles; word kg of row n holds codes 8kg..8kg+7 with
-// code 8kg+j in bits 4j..4j+3 (the same nibble order as the activation format).  Words are
-// stored in blocks of 16 rows x 128 codes (1 KiB).  A block is two 512-byte halves of 64 codes;
-// inside a half the 16-byte piece of lane l = 4g + t (g = row mod 8, t = word mod 4) holds the
-// words {(row g, word t), (row g+8, word t), (row g, word t+4), (row g+8, word t+4)}: after the
-// nibble split this is exactly the A-fragment pair of two m16n8k32 integer MMAs, so the decode
-// kernel feeds tensor cores from one 128-bit load per lane, and the prefill kernel expands the
-// same pieces into the shared-memory operand tiles of tcgen05.mma.  Blocks are ordered
-// [row block][k block], k fastest, so all codes of 16 output channels are contiguous.
-// Rows are padded to a multiple of 128 and K' to a multiple of 128 with zero codes.
+// Codes are packed two per byte exactly like the activation format (byte j of a row = code 2j in
+// bits 0-3, code 2j+1 in bits 4-7, two's complement).  Bytes are stored in units of 16 output
+// channels x 128 codes (1 KiB): inside a unit the 16 rows follow one another, 64 bytes each.
+// Units are ordered [row block][k block], k fastest, so all codes of 16 output channels are
+// contiguous (the decode kernel streams them linearly) and 16 consecutive row blocks at one k
+// block, fetched as 16 bulk copies, land in shared memory as a plain 256-row x 64-byte tile (the
+// prefill kernel expands that tile into the operand layout of tcgen05.mma).
+// Rows are padded to a multiple of 256 and K' to a multiple of 128 with zero codes.
 // ---------------------------------------------------------------------------------------------
 constexpr int XQ_ROW_BLOCK = 16;
 constexpr int XQ_K_BLOCK = 128;
 constexpr int XQ_BLOCK_BYTES = XQ_ROW_BLOCK * XQ_K_BLOCK / 2;  // 1024
-constexpr int XQ_ROW_PAD = 128;
+constexpr int XQ_ROW_PAD = 256;
 
 struct xq_weights {
   int32_t N, K, Kp;    // logical sizes
-  int32_t Np, Kpp;     // padded sizes (multiples of 128)
+  int32_t Np, Kpp;     // padded sizes (multiples of 256 and 128)
   xq_hadamard_plan_t plan;
   uint8_t* packed;     // device, Np * Kpp / 2 bytes, block layout above
   float* s_w;          // device, Np floats (padding rows hold 0)
@@ -38,10 +36,8 @@ struct xq_weights {
 
 // Byte offset of the 32-bit word holding codes 8*kg .. 8*kg+7 of row n.
 __host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_blocks) {
-  const int rb = n >> 4, r = n & 15, g = r & 7, hi_row = r >> 3;
-  const int kb = kg >> 4, kin = kg & 15, half = kin >> 3, ks = kin & 7, t = ks & 3, hi_k = ks >> 2;
-  return ((size_t)rb * k_blocks + kb) * XQ_BLOCK_BYTES + (size_t)half * 512 + (size_t)(4 * g + t) * 16 +
-         (size_t)(hi_row + 2 * hi_k) * 4;
+  const int rb = n >> 4, r = n & 15, kb = kg >> 4, kin = kg & 15;
+  return ((size_t)rb * k_blocks + kb) * XQ_BLOCK_BYTES + (size_t)r * 64 + (size_t)kin * 4;
 }
 
 // Workspace layout (all offsets multiples of 256 bytes).  The header is what xq_workspace_init
@@ -79,5 +75,8 @@ size_t xq_decode_ws_bytes(const xq_weights* w, int sms);
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                                   int32_t* acc_opt, int32_t* partial, int32_t* counters, int32_t* status, int sms,
                                   cudaStream_t st);
+bool xq_prefill_supported(int32_t M, const xq_weights* w);
+cudaError_t xq_launch_gemm_prefill(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+                                   int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st);
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st);

@@ -114,6 +114,8 @@ GEMM_CASES = [
     (1, 16, 100, 136), (3, 100, 200, 240), (8, 37, 130, 144), (5, 130, 70, 80), (33, 257, 64, 64),
     (1, 2048, 2048, 2176), (16, 2048, 2048, 2176), (8, 3072, 2048, 2176), (32, 2048, 8192, 8704),
     (17, 384, 4096, 4352), (160, 256, 2048, 2176), (300, 200, 4096, 4608),
+    # tensor-core tiles: ragged token and channel tails, several tiles per CTA, a K tail inside a block
+    (130, 264, 2048, 2176), (64, 2048, 8192, 8704), (1100, 4608, 250, 256), (129, 512, 90, 96), (2048, 2048, 2048, 2176),
 ]
 
 
