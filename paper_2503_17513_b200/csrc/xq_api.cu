@@ -74,8 +74,6 @@ xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w) {
   off += align_up((size_t)M_max * (size_t)w->K * 2, 256);
   L.ostage = off;
   off += align_up((size_t)M_max * (size_t)w->N * 2, 256);
-  L.partial = off;
-  off += align_up(xq_decode_ws_bytes(w, w->sms), 256);
   L.total = off;
   return L;
 }

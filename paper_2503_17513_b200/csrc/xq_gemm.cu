@@ -13,7 +13,7 @@ namespace {
 // path for sizes the tiled kernels do not take.
 __global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __restrict__ Xq, const float* __restrict__ sx, int M,
                                                            const uint8_t* __restrict__ Wb, const float* __restrict__ sw, int N,
-                                                           int Kp, int k_blocks, __nv_bfloat16* __restrict__ out,
+                                                           int Kp, int k_groups, __nv_bfloat16* __restrict__ out,
                                                            int32_t* __restrict__ acc_opt) {
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   const int m = blockIdx.y;
@@ -22,7 +22,7 @@ __global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __res
   const uint32_t* xrow = Xq + (long long)m * words;
   int acc = 0;
   for (int kg = 0; kg < words; ++kg) {
-    const uint32_t w = *reinterpret_cast<const uint32_t*>(Wb + xq_weight_word_offset(n, kg, k_blocks));
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(Wb + xq_weight_word_offset(n, kg, k_groups));
     uint32_t we, wo, xe, xo;
     split16(w, we, wo);
     split16(xrow[kg], xe, xo);
@@ -40,12 +40,13 @@ cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const 
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st) {
   if (w->Kp % 8 != 0) return cudaErrorInvalidValue;
   int32_t* header = (int32_t*)ws;
-  if (xq_decode_supported(M, w) && w->Np / 16 <= XQ_WS_MAX_ROW_BLOCKS)
-    return xq_launch_gemm_decode(Xq, sx, M, w, out, acc_opt, (int32_t*)((uint8_t*)ws + L.partial),
-                                 header + XQ_WS_COUNTER_OFFSET_WORDS, header, w->sms, st);
+  if (M <= XQ_DECODE_MAX_M) {
+    const cudaError_t e = xq_launch_gemm_decode(Xq, sx, M, w, out, acc_opt, header, st);
+    if (e != cudaErrorNotSupported) return e;
+  }
   if (xq_prefill_supported(M, w)) return xq_launch_gemm_prefill(Xq, sx, M, w, out, acc_opt, header, w->sms, st);
   dim3 grid((w->N + 127) / 128, M);
   gemm_general_kernel<<<grid, 128, 0, st>>>((const uint32_t*)Xq, sx, M, w->packed, w->s_w, w->N, w->Kp,
-                                            w->Kpp / XQ_K_BLOCK, (__nv_bfloat16*)out, acc_opt);
+                                            w->Kpp / XQ_K_GROUP, (__nv_bfloat16*)out, acc_opt);
   return cudaGetLastError();
 }

@@ -2,19 +2,24 @@
 // packed INT4 weights once from HBM (paper Sec. 3: the quantized product Q(XR) Q(W~) computed at
 // inference; here the case where the weight stream, not the arithmetic, sets the time).
 //
-// Work is cut into 1 KiB units (16 output channels x 128 codes, contiguous in the weight layout,
-// k fastest).  Each persistent CTA takes one contiguous range of units -- so its HBM stream is one
-// linear run, fetched by a producer warp with bulk copies into a shared-memory ring of 8 KiB
-// chunks, the first ring-full requested before the kernel waits for its predecessor in the
-// stream.  Eight consumer warps take one unit of every chunk each: two 128-bit loads give a lane
-// the codes of rows g and g+8, the nibble split turns them into the A fragments of four
-// m16n8k32 integer MMAs (weights as the 16-row operand, 8 tokens as the columns).  The token
-// operand is expanded once per CTA into shared memory in fragment order when it fits, else kept
-// packed and split on the fly.  A warp adds its fragment into the CTA's per-row-block tile with
-// shared-memory reductions whenever its unit crosses into another row block.  A row block that
-// spans several CTAs is finished by the last CTA to arrive: contributors publish partial tiles in
-// per-CTA slots and bump an arrival counter; nobody ever waits for another CTA.
+// Decomposition.  Output channels are handled in blocks of 8; a thread-block cluster of C CTAs
+// owns a contiguous range of blocks and cuts K between its CTAs in multiples of 32 codes, so a
+// CTA needs only its K slice of the quantized tokens.  In the weight layout the K slice of one
+// block is one contiguous run of bytes; a producer warp fetches runs with bulk copies (pieces of
+// at most 4 KiB) into a shared-memory ring, the first ring-full before the kernel waits for its
+// predecessor in the stream.  Each of the eight consumer warps owns whole blocks (block j of
+// the range goes to warp j mod 8), so a block's partial sums stay in one warp's registers:
+// MMA i of a chunk of four 32-code groups takes group i; lane (channel g, word t) loads its word
+// of eight codes with one conflict-free 32-bit load, the nibble split turns it into the B
+// fragment of an m16n8k32 integer MMA (even codes in K slots 4t.., odd codes in 16+4t..), and the
+// A fragments (16 tokens) come from the token slice that the CTA expanded once into shared
+// memory in exactly that fragment order.  The C partial tiles of a
+// block meet through distributed shared memory: after one cluster barrier CTA s sums and
+// finishes the blocks j with j mod C == s (scales, bf16, 16-byte stores).  No global scratch,
+// no atomics, no CTA waits on another outside the two cluster barriers.
 #include <cuda_bf16.h>
+
+#include <mutex>
 
 #include "xq_internal.h"
 #include "xq_ptx.cuh"
@@ -26,10 +31,9 @@ namespace {
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;
-constexpr int kChunkUnits = kConsumerWarps;                 // one unit per consumer warp
-constexpr int kChunkBytes = kChunkUnits * XQ_BLOCK_BYTES;   // 8 KiB
-constexpr int kMaxStages = 16;
-constexpr int kSlotInts = 16 * 32;
+constexpr int kPieceGroups = 32;                               // 32-code groups per ring stage
+constexpr int kStageBytes = kPieceGroups * XQ_GROUP_BYTES;     // 4 KiB
+constexpr int kMaxStages = 32;
 
 struct DecodeParams {
   const uint8_t* W;
@@ -38,336 +42,349 @@ struct DecodeParams {
   const float* sx;
   __nv_bfloat16* out;
   int32_t* acc_opt;
-  int32_t* partial;   // [(row blocks + grid)] slots of 16 x 32 int32
-  int32_t* counters;  // [row blocks], zero between launches
   int32_t* status;
-  int U;              // units in total (fits 31 bits: checked on the host)
-  int M, N, Kp, KB;   // KB = Kp / 128
-  int stages;         // ring stages
-  int act_pitch;      // bytes between token rows of the shared-memory token operand
-  int max_tiles;      // row blocks a CTA's range can touch
+  int M, N, Kp;
+  int k_groups;     // groups of 32 codes per channel block in the weight layout (K'' / 32)
+  int n_blocks;     // channel blocks holding real channels: ceil(N / 8)
+  int stages;       // ring stages, a multiple of 8
+  int act_pitch;    // bytes between token rows of the expanded token slice
+  int max_blocks;   // blocks in the longest cluster range
 };
 
-template <int NT, bool PRESPLIT>  // token tiles of 8: M <= 8 * NT
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// 16 bytes from the shared memory of CTA `rank` of the cluster, at the address that `local_ptr`
+// has in this CTA.
+__device__ __forceinline__ int4 ld_cluster_v4(const void* local_ptr, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(rank));
+  int4 v;
+  asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(remote) : "memory");
+  return v;
+}
+
+template <int NT, int C>  // NT token tiles of 16 (M <= 16 NT), clusters of C CTAs
 __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int G = gridDim.x, cta = blockIdx.x;
-  constexpr int MT = 8 * NT;   // padded token count
-  constexpr int TP = MT + 8;   // pitch of a tile row (ints)
+  constexpr int MT = 16 * NT;  // padded token count
+  const int rank = C == 1 ? 0 : (int)cluster_ctarank();
+  const int cid = blockIdx.x / C, n_clusters = gridDim.x / C;
 
   unsigned char* ring = smem;
-  unsigned char* act = ring + (size_t)p.stages * kChunkBytes;
-  int* tiles = reinterpret_cast<int*>(act + (size_t)MT * p.act_pitch);
-  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)p.max_tiles * 16 * TP);
+  unsigned char* act = ring + (size_t)p.stages * kStageBytes;
+  int* tiles = reinterpret_cast<int*>(act + (size_t)MT * p.act_pitch);   // [block][token][8 channels]
+  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)p.max_blocks * MT * 8);
   uint64_t* empty = full + p.stages;
-  uint64_t* actbar = empty + p.stages;
-  volatile int* flags = reinterpret_cast<volatile int*>(actbar + 1);  // [0] failed, [1] is_last
+  volatile int* failed = reinterpret_cast<volatile int*>(empty + p.stages);
 
-  const int u0 = (int)((long long)cta * p.U / G), u1 = (int)((long long)(cta + 1) * p.U / G);
-  const int n_units = u1 - u0;
-  const int rbA = u0 / p.KB;
+  // this cluster's channel blocks and this CTA's K slice (in groups of 32 codes)
+  const int b0 = (int)((long long)cid * p.n_blocks / n_clusters), b1 = (int)((long long)(cid + 1) * p.n_blocks / n_clusters);
+  const int n_blk = b1 - b0;
+  const int groups = p.Kp / XQ_K_GROUP;
+  const int g0 = rank * groups / C, g1 = (rank + 1) * groups / C;
+  const int L = g1 - g0;                                  // groups in the slice
+  const int parts = (L + kPieceGroups - 1) / kPieceGroups;  // ring pieces per block
+  const int rounds = (n_blk + kConsumerWarps - 1) / kConsumerWarps;
 
   if (tid < p.stages) {
     mbar_init(&full[tid], 1);
-    mbar_init(&empty[tid], kConsumerWarps);
+    mbar_init(&empty[tid], 1);
   }
-  if (tid == 32) {
-    mbar_init(actbar, 1);
-    flags[0] = 0;
-    flags[1] = 0;
-  }
+  if (tid == 32) *failed = 0;
   mbar_fence_init();
   __syncthreads();
   pdl_launch_dependents();
 
   if (warp == kConsumerWarps) {
     // ---------------- producer ------------------------------------------------------------------
-    // The weights are constants: their first ring-full is requested at once.  The activations
-    // may come from the kernel before this one, so they wait for the grid dependency.
-    const long long bytes = (long long)n_units * XQ_BLOCK_BYTES;
-    const unsigned char* src = p.W + (size_t)u0 * XQ_BLOCK_BYTES;
-    const int chunks = (n_units + kChunkUnits - 1) / kChunkUnits;
-    int s = 0;
-    uint32_t wrap = 0;  // times the ring index wrapped
-    auto issue = [&](int ci) -> bool {
-      if (ci >= p.stages && !mbar_wait_bounded(&empty[s], (wrap - 1) & 1, flags, p.status, (int)XQ_ERR_TIMEOUT)) return false;
-      const long long off = (long long)ci * kChunkBytes;
-      const uint32_t n = (uint32_t)min((long long)kChunkBytes, bytes - off);
-      mbar_expect_tx(&full[s], n);
-      bulk_g2s(ring + (size_t)s * kChunkBytes, src + off, n, &full[s]);
-      if (++s == p.stages) {
-        s = 0;
-        ++wrap;
+    // Piece i = (round r, part q, warp w) -> ring stage i mod stages; the stage count is a
+    // multiple of 8, so a stage is always reused by the same warp.  The weights are constants:
+    // pieces that fit the ring are requested before the wait on the preceding kernel.
+    if (lane == 0) {
+      const int total = rounds * parts * kConsumerWarps;
+      for (int i = 0; i < total; ++i) {
+        const int w = i & (kConsumerWarps - 1), rq = i >> 3, r = rq / parts, q = rq - r * parts;
+        const int j = r * kConsumerWarps + w;
+        if (j >= n_blk) continue;
+        const int s = i % p.stages;
+        if (i >= p.stages && !mbar_wait_bounded(&empty[s], ((i / p.stages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT)) break;
+        const int ng = min(kPieceGroups, L - q * kPieceGroups);
+        const uint32_t bytes = (uint32_t)ng * XQ_GROUP_BYTES;
+        const unsigned char* src = p.W + ((size_t)(b0 + j) * p.k_groups + g0 + q * kPieceGroups) * XQ_GROUP_BYTES;
+        mbar_expect_tx(&full[s], bytes);
+        bulk_g2s(ring + (size_t)s * kStageBytes, src, bytes, &full[s]);
       }
-      return true;
-    };
-    const int first = min(chunks, p.stages);
-    if (lane == 0)
-      for (int ci = 0; ci < first; ++ci) issue(ci);
-    pdl_wait();
-    if (!PRESPLIT) {
-      const uint32_t row_bytes = (uint32_t)(p.Kp / 2);
-      if (lane == 0) mbar_expect_tx(actbar, row_bytes * (uint32_t)p.M);
-      __syncwarp();
-      if (lane < p.M) bulk_g2s(act + (size_t)lane * p.act_pitch, p.Xq + (size_t)lane * row_bytes, row_bytes, actbar);
     }
-    if (lane == 0)
-      for (int ci = first; ci < chunks; ++ci)
-        if (!issue(ci)) break;
-    return;
-  }
-
-  // ---------------- consumers ------------------------------------------------------------------
-  for (int i = tid; i < p.max_tiles * 16 * TP; i += kConsumerThreads) tiles[i] = 0;
-  if (PRESPLIT) {
+  } else {
+    // ---------------- consumers ----------------------------------------------------------------
     // token rows beyond M are zero
     for (int i = tid; i < (MT - p.M) * (p.act_pitch / 16); i += kConsumerThreads)
       reinterpret_cast<uint4*>(act + (size_t)p.M * p.act_pitch)[i] = make_uint4(0, 0, 0, 0);
     pdl_wait();
-    // expand the packed tokens once: a 16-byte piece (words w0..w3) becomes 32 bytes
-    // {even(w0), odd(w0), even(w1), odd(w1) | even(w2), odd(w2), even(w3), odd(w3)}
-    const int pieces = p.Kp / 32;
-    for (int m = warp; m < p.M; m += kConsumerWarps) {
-      const uint4* srow = reinterpret_cast<const uint4*>(p.Xq + (size_t)m * (p.Kp / 2));
-      uint4* drow = reinterpret_cast<uint4*>(act + (size_t)m * p.act_pitch);
-      for (int c = lane; c < pieces; c += 32) {
-        const uint4 v = __ldg(srow + c);
-        uint4 lo, hi;
-        split16(v.x, lo.x, lo.y);
-        split16(v.y, lo.z, lo.w);
-        split16(v.z, hi.x, hi.y);
-        split16(v.w, hi.z, hi.w);
-        drow[2 * c] = lo;
-        drow[2 * c + 1] = hi;
+    // Expand this CTA's K slice of the packed tokens once, in fragment order: chunk c of four
+    // groups takes 128 bytes per token, word t of group i (even codes, odd codes) at
+    // c * 128 + t * 32 + i * 8.
+    {
+      const int total = p.M * L;
+      constexpr int kBatch = 4;
+      for (int base = tid; base < total; base += kBatch * kConsumerThreads) {
+        uint4 v[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const int i = base + u * kConsumerThreads;
+          if (i < total) {
+            const int m = i / L, l = i - m * L;
+            v[u] = __ldg(reinterpret_cast<const uint4*>(p.Xq + (size_t)m * (p.Kp / 2)) + g0 + l);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const int i = base + u * kConsumerThreads;
+          if (i < total) {
+            const int m = i / L, l = i - m * L;
+            unsigned char* d = act + (size_t)m * p.act_pitch + (size_t)(l >> 2) * 128 + (size_t)(l & 3) * 8;
+            uint2 e;
+            split16(v[u].x, e.x, e.y);
+            *reinterpret_cast<uint2*>(d) = e;
+            split16(v[u].y, e.x, e.y);
+            *reinterpret_cast<uint2*>(d + 32) = e;
+            split16(v[u].z, e.x, e.y);
+            *reinterpret_cast<uint2*>(d + 64) = e;
+            split16(v[u].w, e.x, e.y);
+            *reinterpret_cast<uint2*>(d + 96) = e;
+          }
+        }
       }
     }
-  } else {
-    pdl_wait();  // the workspace (partial slots, counters) may still be in use by the kernel before
-    for (int i = tid; i < (MT - p.M) * (p.act_pitch / 16); i += kConsumerThreads)
-      reinterpret_cast<uint4*>(act + (size_t)p.M * p.act_pitch)[i] = make_uint4(0, 0, 0, 0);
-    mbar_wait_bounded(actbar, 0, flags, p.status, (int)XQ_ERR_TIMEOUT);
-  }
-  bar_sync(1, kConsumerThreads);
+    bar_sync(1, kConsumerThreads);
 
-  const int g = lane >> 2, t = lane & 3;
-  {
-    int acc[NT][2][4];
-#pragma unroll
-    for (int j = 0; j < NT; ++j)
-#pragma unroll
-      for (int c = 0; c < 2; ++c) acc[j][c][0] = acc[j][c][1] = acc[j][c][2] = acc[j][c][3] = 0;
-    auto flush = [&](int tile_index) {
-      int* tl = tiles + (size_t)tile_index * 16 * TP;
-#pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        atomicAdd(&tl[g * TP + 8 * j + 2 * t], acc[j][0][0] + acc[j][1][0]);
-        atomicAdd(&tl[g * TP + 8 * j + 2 * t + 1], acc[j][0][1] + acc[j][1][1]);
-        atomicAdd(&tl[(g + 8) * TP + 8 * j + 2 * t], acc[j][0][2] + acc[j][1][2]);
-        atomicAdd(&tl[(g + 8) * TP + 8 * j + 2 * t + 1], acc[j][0][3] + acc[j][1][3]);
-#pragma unroll
-        for (int c = 0; c < 2; ++c) acc[j][c][0] = acc[j][c][1] = acc[j][c][2] = acc[j][c][3] = 0;
-      }
-    };
-
-    // this warp's units: local index warp, warp + 8, ...; (rb, kb) follow incrementally
-    int kb = (u0 - rbA * p.KB) + warp, rb = rbA;
-    while (kb >= p.KB) {
-      kb -= p.KB;
-      ++rb;
-    }
-    int cur_rb = rb, s = 0;
-    uint32_t phase = 0;
+    const int ag = lane >> 2, at = lane & 3;  // MMA fragment coordinates: channel / token row, word
     bool ok = true;
-    for (int ul = warp; ul < n_units; ul += kChunkUnits) {
-      if (rb != cur_rb) {
-        flush(cur_rb - rbA);
-        cur_rb = rb;
-      }
-      ok = mbar_wait_bounded(&full[s], phase, flags, p.status, (int)XQ_ERR_TIMEOUT);
-      if (!ok) break;
-      const unsigned char* unit = ring + (size_t)s * kChunkBytes + warp * XQ_BLOCK_BYTES;
-      const uint4 w0 = *reinterpret_cast<const uint4*>(unit + g * 64 + t * 16);        // row g, codes 32t..32t+31
-      const uint4 w1 = *reinterpret_cast<const uint4*>(unit + (g + 8) * 64 + t * 16);  // row g+8
-      uint32_t a[4][4];
-      split16(w0.x, a[0][0], a[0][2]);
-      split16(w1.x, a[0][1], a[0][3]);
-      split16(w0.y, a[1][0], a[1][2]);
-      split16(w1.y, a[1][1], a[1][3]);
-      split16(w0.z, a[2][0], a[2][2]);
-      split16(w1.z, a[2][1], a[2][3]);
-      split16(w0.w, a[3][0], a[3][2]);
-      split16(w1.w, a[3][1], a[3][3]);
+    for (int r = 0; r < rounds && ok; ++r) {
+      const int j = r * kConsumerWarps + warp;
+      if (j >= n_blk) break;
+      int acc[NT][2][4];
 #pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        uint32_t b[4][2];
-        if (PRESPLIT) {
-          const uint4* xr = reinterpret_cast<const uint4*>(act + (size_t)(8 * j + g) * p.act_pitch + kb * 128 + t * 32);
-          const uint4 x0 = xr[0], x1 = xr[1];
-          b[0][0] = x0.x; b[0][1] = x0.y; b[1][0] = x0.z; b[1][1] = x0.w;
-          b[2][0] = x1.x; b[2][1] = x1.y; b[3][0] = x1.z; b[3][1] = x1.w;
-        } else {
-          const uint4 x = *reinterpret_cast<const uint4*>(act + (size_t)(8 * j + g) * p.act_pitch + kb * 64 + t * 16);
-          split16(x.x, b[0][0], b[0][1]);
-          split16(x.y, b[1][0], b[1][1]);
-          split16(x.z, b[2][0], b[2][1]);
-          split16(x.w, b[3][0], b[3][1]);
+      for (int a = 0; a < NT; ++a)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) acc[a][c][0] = acc[a][c][1] = acc[a][c][2] = acc[a][c][3] = 0;
+      for (int q = 0; q < parts && ok; ++q) {
+        const int i = (r * parts + q) * kConsumerWarps + warp;
+        const int s = i % p.stages;
+        ok = mbar_wait_bounded(&full[s], (i / p.stages) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+        if (!ok) break;
+        const int ng = min(kPieceGroups, L - q * kPieceGroups);
+        const unsigned char* wp = ring + (size_t)s * kStageBytes + lane * 4;  // channel ag, word at of group 0
+        for (int gq = 0; gq < ng; gq += 4, wp += 4 * XQ_GROUP_BYTES) {
+          const int nv = min(4, ng - gq);  // groups of this chunk that exist
+          uint32_t b[4][2];
+#pragma unroll
+          for (int i4 = 0; i4 < 4; ++i4) {
+            const uint32_t wv = i4 < nv ? *reinterpret_cast<const uint32_t*>(wp + i4 * XQ_GROUP_BYTES) : 0u;
+            split16(wv, b[i4][0], b[i4][1]);
+          }
+          const size_t coff = (size_t)(q * (kPieceGroups / 4) + (gq >> 2)) * 128 + (size_t)at * 32;
+#pragma unroll
+          for (int a = 0; a < NT; ++a) {
+            const uint4* lo = reinterpret_cast<const uint4*>(act + (size_t)(16 * a + ag) * p.act_pitch + coff);
+            const uint4* hi = reinterpret_cast<const uint4*>(act + (size_t)(16 * a + ag + 8) * p.act_pitch + coff);
+            const uint4 x0 = lo[0], x1 = lo[1], y0 = hi[0], y1 = hi[1];
+            const uint32_t a0[4] = {x0.x, y0.x, x0.y, y0.y};
+            const uint32_t a1[4] = {x0.z, y0.z, x0.w, y0.w};
+            const uint32_t a2[4] = {x1.x, y1.x, x1.y, y1.y};
+            const uint32_t a3[4] = {x1.z, y1.z, x1.w, y1.w};
+            mma_s8_16x8x32(acc[a][0], a0, b[0][0], b[0][1]);
+            mma_s8_16x8x32(acc[a][1], a1, b[1][0], b[1][1]);
+            mma_s8_16x8x32(acc[a][0], a2, b[2][0], b[2][1]);
+            mma_s8_16x8x32(acc[a][1], a3, b[3][0], b[3][1]);
+          }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);
+      }
+      // D fragment: (token ag, channels 2 at, 2 at + 1), (token ag + 8, same channels)
+      int* tl = tiles + (size_t)j * MT * 8;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) mma_s8_16x8x32(acc[j][i & 1], a[i], b[i][0], b[i][1]);
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[s]);
-      if (++s == p.stages) {
-        s = 0;
-        phase ^= 1u;
-      }
-      kb += kChunkUnits;
-      while (kb >= p.KB) {
-        kb -= p.KB;
-        ++rb;
+      for (int a = 0; a < NT; ++a) {
+        *reinterpret_cast<int2*>(&tl[(16 * a + ag) * 8 + 2 * at]) = make_int2(acc[a][0][0] + acc[a][1][0], acc[a][0][1] + acc[a][1][1]);
+        *reinterpret_cast<int2*>(&tl[(16 * a + ag + 8) * 8 + 2 * at]) = make_int2(acc[a][0][2] + acc[a][1][2], acc[a][0][3] + acc[a][1][3]);
       }
     }
-    if (n_units > warp) flush(cur_rb - rbA);
   }
-  bar_sync(1, kConsumerThreads);
 
-  // ---------------- finish or hand over every row block of the range -----------------------------
-  const int rbB = (u1 - 1) / p.KB;
-  const bool active = tid < MT * 8;
-  const int m = tid >> 3, np = tid & 7;  // token, pair of output channels
-  for (int rb = rbA; rb <= rbB && n_units > 0; ++rb) {
-    const int* tl = tiles + (size_t)(rb - rbA) * 16 * TP;
-    int v0 = 0, v1 = 0;
-    if (active) {
-      v0 = tl[(2 * np) * TP + m];
-      v1 = tl[(2 * np + 1) * TP + m];
-    }
-    const bool whole = (long long)rb * p.KB >= u0 && (long long)(rb + 1) * p.KB <= u1;
-    bool finish = whole;
-    if (!whole) {
-      // contributors of this row block: CTAs c_first..c_last (c(u) = largest c with u0(c) <= u)
-      const long long ua = (long long)rb * p.KB, ub = (long long)(rb + 1) * p.KB - 1;
-      const int c_first = (int)(((ua + 1) * G - 1) / p.U), c_last = (int)(((ub + 1) * G - 1) / p.U);
-      int32_t* slot = p.partial + ((size_t)rb + cta) * kSlotInts;
-      if (active) *reinterpret_cast<int2*>(&slot[2 * tid]) = make_int2(v0, v1);
-      bar_sync(1, kConsumerThreads);
-      if (tid == 0) {
-        __threadfence();  // cumulative: publishes the whole CTA's slot (ordered by the barrier)
-        const int old = atomicAdd(&p.counters[rb], 1);
-        __threadfence();
-        flags[1] = (old == c_last - c_first) ? 1 : 0;
+  // ---------------- meet the other K slices and finish ------------------------------------------
+  if (C > 1) cluster_sync_all(); else __syncthreads();
+  if (warp < kConsumerWarps && !*failed) {
+    // CTA `rank` finishes blocks j = rank, rank + C, ...: one thread per (block, token)
+    const int mine = (n_blk - rank + C - 1) / C;
+    for (int idx = tid; idx < mine * p.M; idx += kConsumerThreads) {
+      const int jj = idx / p.M, m = idx - jj * p.M;
+      const int j = rank + jj * C;
+      const int* row = tiles + ((size_t)j * MT + m) * 8;
+      int4 lo = *reinterpret_cast<const int4*>(row), hi = *reinterpret_cast<const int4*>(row + 4);
+#pragma unroll
+      for (int o = 1; o < C; ++o) {
+        const uint32_t peer = (uint32_t)((rank + o) % C);
+        const int4 l2 = ld_cluster_v4(row, peer), h2 = ld_cluster_v4(row + 4, peer);
+        lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
+        hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
       }
-      bar_sync(1, kConsumerThreads);
-      finish = flags[1] != 0;
-      if (finish) {
-        if (active) {
-          for (int c = c_first; c <= c_last; ++c) {
-            if (c == cta) continue;
-            const int2 o = __ldcg(reinterpret_cast<const int2*>(p.partial + ((size_t)rb + c) * kSlotInts + 2 * tid));
-            v0 += o.x;
-            v1 += o.y;
-          }
-        }
-        if (tid == 0) p.counters[rb] = 0;  // ready for the next launch
-      }
-      bar_sync(1, kConsumerThreads);  // flags[1] is reused by the next partial row block
-    }
-    if (finish && active && m < p.M) {
-      v0 >>= 8;  // every product carries 16 x 16
-      v1 >>= 8;
-      const int n0 = rb * 16 + 2 * np;
+      const int v[8] = {lo.x >> 8, lo.y >> 8, lo.z >> 8, lo.w >> 8, hi.x >> 8, hi.y >> 8, hi.z >> 8, hi.w >> 8};  // every product carries 16 x 16
+      const int n0 = (b0 + j) * 8;
       const float sxm = p.sx[m];
-      if (n0 < p.N) {
-        const size_t o = (size_t)m * p.N + n0;
-        if (p.acc_opt) p.acc_opt[o] = v0;
-        const __nv_bfloat16 h0 = __float2bfloat16_rn((float)v0 * sxm * p.sw[n0]);
-        if (n0 + 1 < p.N) {
-          if (p.acc_opt) p.acc_opt[o + 1] = v1;
-          const __nv_bfloat16 h1 = __float2bfloat16_rn((float)v1 * sxm * p.sw[n0 + 1]);
-          if ((p.N & 1) == 0) {
-            *reinterpret_cast<__nv_bfloat162*>(p.out + o) = __halves2bfloat162(h0, h1);
-          } else {
-            p.out[o] = h0;
-            p.out[o + 1] = h1;
-          }
-        } else {
-          p.out[o] = h0;
+      const size_t o = (size_t)m * p.N + n0;
+      if (n0 + 8 <= p.N && (p.N & 7) == 0) {
+        const float4 s0 = *reinterpret_cast<const float4*>(p.sw + n0), s1 = *reinterpret_cast<const float4*>(p.sw + n0 + 4);
+        const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+        uint32_t h[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const __nv_bfloat162 b2 = __halves2bfloat162(__float2bfloat16_rn((float)v[2 * e] * sxm * sc[2 * e]),
+                                                       __float2bfloat16_rn((float)v[2 * e + 1] * sxm * sc[2 * e + 1]));
+          h[e] = *reinterpret_cast<const uint32_t*>(&b2);
         }
+        *reinterpret_cast<uint4*>(p.out + o) = make_uint4(h[0], h[1], h[2], h[3]);
+        if (p.acc_opt) {
+          *reinterpret_cast<int4*>(p.acc_opt + o) = make_int4(v[0], v[1], v[2], v[3]);
+          *reinterpret_cast<int4*>(p.acc_opt + o + 4) = make_int4(v[4], v[5], v[6], v[7]);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (n0 + e < p.N) {
+            p.out[o + e] = __float2bfloat16_rn((float)v[e] * sxm * p.sw[n0 + e]);
+            if (p.acc_opt) p.acc_opt[o + e] = v[e];
+          }
       }
     }
   }
+  if (C > 1) cluster_sync_all();  // nobody leaves while a peer may still read its tiles
 }
 
 struct DecodePlan {
-  int nt, stages, act_pitch, max_tiles, grid;
-  bool presplit;
+  int nt, C, stages, act_pitch, max_blocks, grid;
   size_t smem;
 };
 
-// Shared-memory plan for M tokens on `sms` multiprocessors; stages == 0 means it does not fit.
-DecodePlan decode_plan(int M, const xq_weights* w, int sms) {
-  DecodePlan d = {};
-  d.nt = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
-  const int MT = 8 * d.nt, KB = w->Kp / 128;
-  const long long U = (long long)(w->Np / 16) * KB;
-  d.grid = (int)(U < sms ? U : sms);
-  const long long per_cta = (U + d.grid - 1) / d.grid;
-  d.max_tiles = (int)(per_cta / KB) + 2;
-  const size_t tiles = (size_t)d.max_tiles * 16 * (MT + 8) * 4;
-  const size_t misc = (2 * kMaxStages + 1) * 8 + 64 + 128;
-  const size_t cap = 227 * 1024;
-  const int want = (int)((per_cta + kChunkUnits - 1) / kChunkUnits);  // chunks of the longest range
-  // row pitches that keep the 128-bit fragment reads of eight token rows on distinct banks
-  const int pitch_split = w->Kp + 16, pitch_packed = w->Kp / 2 + ((w->Kp / 2) % 128 == 0 ? 64 : 0);
-  const size_t act_split = (size_t)MT * pitch_split, act_packed = (size_t)MT * pitch_packed;
-  const size_t min_ring = 4 * (size_t)kChunkBytes;
-  d.presplit = act_split + tiles + misc + min_ring <= cap;
-  const size_t actb = d.presplit ? act_split : act_packed;
-  d.act_pitch = d.presplit ? pitch_split : pitch_packed;
-  if (actb + tiles + misc + 2 * (size_t)kChunkBytes > cap) return d;  // stages == 0
-  int s = (int)((cap - actb - tiles - misc) / kChunkBytes);
-  if (s > kMaxStages) s = kMaxStages;
-  if (s > want) s = want < 2 ? 2 : want;
-  d.stages = s;
-  d.smem = actb + tiles + misc + (size_t)s * kChunkBytes;
-  return d;
-}
+// Cached answers of cudaOccupancyMaxActiveClusters, keyed by (device, variant, shared memory).
+struct ClusterCacheEntry {
+  int device, nt, C;
+  size_t smem;
+  int clusters;
+};
+std::mutex g_cache_mutex;
+ClusterCacheEntry g_cache[64];
+int g_cache_size = 0;
 
-template <int NT, bool PRESPLIT>
-cudaError_t launch_nt(const DecodeParams& p, int grid, size_t smem, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<NT, PRESPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+template <int NT, int C>
+cudaError_t launch_variant(const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
+  auto kern = gemm_decode_kernel<NT, C>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<NT, PRESPLIT>, p);
+  cfg.numAttrs = 2;
+  if (max_clusters) {  // occupancy query only
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3(C);
+    return cudaOccupancyMaxActiveClusters(max_clusters, kern, &cfg);
+  }
+  return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+cudaError_t dispatch(int nt, int C, const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
+  if (C == 2) {
+    if (nt == 1) return launch_variant<1, 2>(p, grid, smem, st, max_clusters);
+    return launch_variant<2, 2>(p, grid, smem, st, max_clusters);
+  }
+  if (nt == 1) return launch_variant<1, 4>(p, grid, smem, st, max_clusters);
+  return launch_variant<2, 4>(p, grid, smem, st, max_clusters);
+}
+
+int max_active_clusters(int device, int nt, int C, size_t smem) {
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
+  for (int i = 0; i < g_cache_size; ++i)
+    if (g_cache[i].device == device && g_cache[i].nt == nt && g_cache[i].C == C && g_cache[i].smem == smem) return g_cache[i].clusters;
+  int n = 0;
+  DecodeParams dummy = {};
+  if (dispatch(nt, C, dummy, C, smem, nullptr, &n) != cudaSuccess) {
+    cudaGetLastError();
+    n = 0;
+  }
+  if (g_cache_size < 64) g_cache[g_cache_size++] = {device, nt, C, smem, n};
+  return n;
+}
+
+// Shared-memory plan for M tokens; stages == 0 means the shape does not fit this kernel.
+DecodePlan decode_plan(int M, const xq_weights* w) {
+  DecodePlan d = {};
+  if (M < 1 || M > XQ_DECODE_MAX_M || w->Kp % XQ_K_GROUP != 0) return d;
+  d.nt = M <= 16 ? 1 : 2;
+  const int MT = 16 * d.nt, groups = w->Kp / XQ_K_GROUP, n_blocks = (w->N + 7) / 8;
+  const size_t cap = 227 * 1024;
+  for (int C = 2; C <= 4; C *= 2) {
+    if (groups < C) break;
+    const int Lmax = (groups + C - 1) / C;
+    const int chunks = (Lmax + 3) / 4;
+    const int pitch = chunks * 128 + 16;  // 16 (mod 128): conflict-free 128-bit fragment reads
+    const size_t act = (size_t)MT * pitch;
+    // a first guess of the cluster count sizes the tiles; refined below with the occupancy answer
+    for (int pass = 0, clusters = w->sms / C; pass < 2; ++pass) {
+      if (clusters < 1) break;
+      const int nc = clusters < n_blocks ? clusters : n_blocks;
+      const int max_blocks = (n_blocks + nc - 1) / nc;
+      const size_t tiles = (size_t)max_blocks * MT * 8 * 4;
+      const size_t misc = 2 * kMaxStages * 8 + 64 + 128;
+      if (act + tiles + misc + 8 * (size_t)kStageBytes > cap) break;
+      const int parts = (Lmax + kPieceGroups - 1) / kPieceGroups;
+      const int rounds = (max_blocks + kConsumerWarps - 1) / kConsumerWarps;
+      int s = (int)((cap - act - tiles - misc) / kStageBytes) / 8 * 8;
+      if (s > kMaxStages) s = kMaxStages;
+      const int want = (rounds * parts * kConsumerWarps + 7) / 8 * 8;
+      if (s > want) s = want;
+      const size_t smem = act + tiles + misc + (size_t)s * kStageBytes;
+      const int fit = max_active_clusters(w->device, d.nt, C, smem);
+      if (fit < 1) break;
+      if (pass == 1 || fit == clusters) {
+        d.C = C;
+        d.stages = s;
+        d.act_pitch = pitch;
+        d.max_blocks = max_blocks;
+        d.grid = nc * C;
+        d.smem = smem;
+        return d;
+      }
+      clusters = fit < clusters ? fit : clusters;
+    }
+  }
+  return d;
 }
 
 }  // namespace
 
-bool xq_decode_supported(int32_t M, const xq_weights* w) {
-  if (M < 1 || M > XQ_DECODE_MAX_M || w->Kp % 128 != 0) return false;
-  if ((long long)(w->Np / 16) * (w->Kp / 128) > 0x7fffffffLL) return false;
-  return decode_plan(M, w, w->sms).stages >= 2;
-}
-
-size_t xq_decode_ws_bytes(const xq_weights* w, int sms) {
-  const size_t rbs = (size_t)w->Np / 16;
-  return (rbs + sms) * kSlotInts * sizeof(int32_t);
-}
-
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
-                                  int32_t* acc_opt, int32_t* partial, int32_t* counters, int32_t* status, int sms,
-                                  cudaStream_t st) {
-  const DecodePlan d = decode_plan(M, w, sms);
+                                  int32_t* acc_opt, int32_t* status, cudaStream_t st) {
+  const DecodePlan d = decode_plan(M, w);
+  if (d.stages < 8) return cudaErrorNotSupported;
   DecodeParams p;
   p.W = w->packed;
   p.sw = w->s_w;
@@ -375,23 +392,14 @@ cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M,
   p.sx = sx;
   p.out = (__nv_bfloat16*)out;
   p.acc_opt = acc_opt;
-  p.partial = partial;
-  p.counters = counters;
   p.status = status;
-  p.KB = w->Kp / 128;
-  p.U = (w->Np / 16) * p.KB;
   p.M = M;
   p.N = w->N;
   p.Kp = w->Kp;
+  p.k_groups = w->Kpp / XQ_K_GROUP;
+  p.n_blocks = (w->N + 7) / 8;
   p.stages = d.stages;
   p.act_pitch = d.act_pitch;
-  p.max_tiles = d.max_tiles;
-  if (d.presplit) {
-    if (d.nt == 1) return launch_nt<1, true>(p, d.grid, d.smem, st);
-    if (d.nt == 2) return launch_nt<2, true>(p, d.grid, d.smem, st);
-    return launch_nt<4, true>(p, d.grid, d.smem, st);
-  }
-  if (d.nt == 1) return launch_nt<1, false>(p, d.grid, d.smem, st);
-  if (d.nt == 2) return launch_nt<2, false>(p, d.grid, d.smem, st);
-  return launch_nt<4, false>(p, d.grid, d.smem, st);
+  p.max_blocks = d.max_blocks;
+  return dispatch(d.nt, d.C, p, d.grid, d.smem, st, nullptr);
 }

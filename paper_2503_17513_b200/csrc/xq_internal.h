@@ -11,17 +11,21 @@
 // Prepared-weights device layout.
 //
 // Codes are packed two per byte exactly like the activation format (byte j of a row = code 2j in
-// bits 0-3, code 2j+1 in bits 4-7, two's complement).  Bytes are stored in units of 16 output
-// channels x 128 codes (1 KiB): inside a unit the 16 rows follow one another, 64 bytes each.
-// Units are ordered [row block][k block], k fastest, so all codes of 16 output channels are
-// contiguous (the decode kernel streams them linearly) and 16 consecutive row blocks at one k
-// block, fetched as 16 bulk copies, land in shared memory as a plain 256-row x 64-byte tile (the
-// prefill kernel expands that tile into the operand layout of tcgen05.mma).
+// bits 0-3, code 2j+1 in bits 4-7, two's complement).  The smallest piece is 16 bytes: 32
+// consecutive codes of one output channel.  Pieces are stored as
+//     [block of 8 output channels][group of 32 codes][channel within the block][16 bytes]
+// so that (a) the codes of 8 channels over any range of K that is a multiple of 32 are one
+// contiguous run (the decode kernel streams such runs and cuts K between the CTAs of a cluster),
+// (b) a warp-wide 128-bit load of 512 consecutive bytes gives lane 8t + g the codes 32t..32t+31
+// of channel g of a 128-code block -- the B fragments of four m16n8k32 MMAs after the nibble
+// split -- and (c) 32 consecutive channel blocks at one 128-code block, fetched as 32 bulk
+// copies of 512 bytes, form the 256-row tile the prefill kernel expands for tcgen05.mma.
 // Rows are padded to a multiple of 256 and K' to a multiple of 128 with zero codes.
 // ---------------------------------------------------------------------------------------------
-constexpr int XQ_ROW_BLOCK = 16;
+constexpr int XQ_ROW_BLOCK = 8;
+constexpr int XQ_K_GROUP = 32;                                   // codes per 16-byte piece
+constexpr int XQ_GROUP_BYTES = XQ_ROW_BLOCK * XQ_K_GROUP / 2;    // 128: one group of one block
 constexpr int XQ_K_BLOCK = 128;
-constexpr int XQ_BLOCK_BYTES = XQ_ROW_BLOCK * XQ_K_BLOCK / 2;  // 1024
 constexpr int XQ_ROW_PAD = 256;
 
 struct xq_weights {
@@ -34,25 +38,21 @@ struct xq_weights {
   int sms;             // multiprocessors of that device
 };
 
-// Byte offset of the 32-bit word holding codes 8*kg .. 8*kg+7 of row n.
-__host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_blocks) {
-  const int rb = n >> 4, r = n & 15, kb = kg >> 4, kin = kg & 15;
-  return ((size_t)rb * k_blocks + kb) * XQ_BLOCK_BYTES + (size_t)r * 64 + (size_t)kin * 4;
+// Byte offset of the 32-bit word holding codes 8*kg .. 8*kg+7 of row n (k_groups = K'' / 32).
+__host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_groups) {
+  const int blk = n >> 3, g = n & 7, grp = kg >> 2, word = kg & 3;
+  return ((size_t)blk * k_groups + grp) * XQ_GROUP_BYTES + (size_t)g * 16 + (size_t)word * 4;
 }
 
 // Workspace layout (all offsets multiples of 256 bytes).  The header is what xq_workspace_init
-// clears: word 0 is the sticky status, words 64.. are the split-K arrival counters (one per
-// 16-channel row block; kernels leave them at zero).
-constexpr size_t XQ_WS_HEADER_BYTES = 64 * 1024;
-constexpr int XQ_WS_COUNTER_OFFSET_WORDS = 64;
-constexpr int XQ_WS_MAX_ROW_BLOCKS = (int)(XQ_WS_HEADER_BYTES / 4) - XQ_WS_COUNTER_OFFSET_WORDS;
+// clears: word 0 is the sticky status.
+constexpr size_t XQ_WS_HEADER_BYTES = 256;
 struct xq_ws_layout {
   size_t header;   // XQ_WS_HEADER_BYTES
   size_t xq;       // M_max * Kp/2 bytes of packed activations
   size_t sx;       // M_max floats
   size_t xstage;   // M_max * K bf16 (host entry point)
   size_t ostage;   // M_max * N bf16 (host entry point)
-  size_t partial;  // split-K partial accumulators
   size_t total;
 };
 xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
@@ -70,11 +70,9 @@ cudaError_t xq_launch_relayout_from_blocks(const uint8_t* blocks, int32_t Np, in
                                            int32_t N, int32_t Kp, cudaStream_t st);
 cudaError_t xq_launch_pack_codes(const int8_t* codes, int64_t count_pairs, uint8_t* packed, cudaStream_t st);
 cudaError_t xq_launch_unpack_codes(const uint8_t* packed, int64_t count_pairs, int8_t* codes, cudaStream_t st);
-bool xq_decode_supported(int32_t M, const xq_weights* w);
-size_t xq_decode_ws_bytes(const xq_weights* w, int sms);
+// Decode path: returns cudaErrorNotSupported (nothing launched) when the shape does not fit it.
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
-                                  int32_t* acc_opt, int32_t* partial, int32_t* counters, int32_t* status, int sms,
-                                  cudaStream_t st);
+                                  int32_t* acc_opt, int32_t* status, cudaStream_t st);
 bool xq_prefill_supported(int32_t M, const xq_weights* w);
 cudaError_t xq_launch_gemm_prefill(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                                    int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st);

@@ -375,7 +375,7 @@ cudaError_t launch_tc_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq
 // ---------------------------------------------------------------------------------------------
 __global__ void relayout_to_blocks_kernel(const uint8_t* __restrict__ canon, int N, int Kp, uint32_t* __restrict__ blocks,
                                           int Np, int Kpp) {
-  const int k_blocks = Kpp / XQ_K_BLOCK, words_per_row = Kpp / 8, row_bytes = Kp / 2;
+  const int k_groups = Kpp / XQ_K_GROUP, words_per_row = Kpp / 8, row_bytes = Kp / 2;
   const long long total = (long long)Np * words_per_row;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const int n = (int)(i / words_per_row), kg = (int)(i % words_per_row);
@@ -387,17 +387,17 @@ __global__ void relayout_to_blocks_kernel(const uint8_t* __restrict__ canon, int
         if (byte < row_bytes) w |= (uint32_t)canon[(long long)n * row_bytes + byte] << (8 * b);
       }
     }
-    blocks[xq_weight_word_offset(n, kg, k_blocks) / 4] = w;
+    blocks[xq_weight_word_offset(n, kg, k_groups) / 4] = w;
   }
 }
 
 __global__ void relayout_from_blocks_kernel(const uint32_t* __restrict__ blocks, int Np, int Kpp, uint8_t* __restrict__ canon,
                                             int N, int Kp) {
-  const int k_blocks = Kpp / XQ_K_BLOCK, row_bytes = Kp / 2;
+  const int k_groups = Kpp / XQ_K_GROUP, row_bytes = Kp / 2;
   const long long total = (long long)N * row_bytes;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const int n = (int)(i / row_bytes), byte = (int)(i % row_bytes);
-    const uint32_t w = blocks[xq_weight_word_offset(n, byte >> 2, k_blocks) / 4];
+    const uint32_t w = blocks[xq_weight_word_offset(n, byte >> 2, k_groups) / 4];
     canon[i] = (uint8_t)(w >> (8 * (byte & 3)));
   }
 }
