@@ -13,10 +13,11 @@
 // of eight codes with one conflict-free 32-bit load, the nibble split turns it into the B
 // fragment of an m16n8k32 integer MMA (even codes in K slots 4t.., odd codes in 16+4t..), and the
 // A fragments (16 tokens) come from the token slice that the CTA expanded once into shared
-// memory in exactly that fragment order.  The C partial tiles of a
-// block meet through distributed shared memory: after one cluster barrier CTA s sums and
-// finishes the blocks j with j mod C == s (scales, bf16, 16-byte stores).  No global scratch,
-// no atomics, no CTA waits on another outside the two cluster barriers.
+// memory in exactly that fragment order.  Block j is finished by CTA j mod C
+// of the cluster: every CTA stores its partial tile of the block into that CTA's shared memory
+// (distributed shared memory), and after one cluster barrier the owner sums the C tiles and
+// applies the epilogue (scales, bf16, 16-byte stores).  No global scratch, no atomics, and no
+// CTA waits on another outside the cluster barrier.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -46,7 +47,7 @@ struct DecodeParams {
   int M, N, Kp;
   int k_groups;     // groups of 32 codes per channel block in the weight layout (K'' / 32)
   int n_blocks;     // channel blocks holding real channels: ceil(N / 8)
-  int stages;       // ring stages, a multiple of 8
+  int stages;       // ring stages: 8, 16 or 32
   int act_pitch;    // bytes between token rows of the expanded token slice
   int max_blocks;   // blocks in the longest cluster range
 };
@@ -56,18 +57,15 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
 }
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// 16 bytes from the shared memory of CTA `rank` of the cluster, at the address that `local_ptr`
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// 8 bytes into the shared memory of CTA `rank` of the cluster, at the address that `local_ptr`
 // has in this CTA.
-__device__ __forceinline__ int4 ld_cluster_v4(const void* local_ptr, uint32_t rank) {
+__device__ __forceinline__ void st_cluster_v2(void* local_ptr, uint32_t rank, int2 v) {
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(rank));
-  int4 v;
-  asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(remote) : "memory");
-  return v;
+  asm volatile("st.shared::cluster.v2.s32 [%0], {%1, %2};" ::"r"(remote), "r"(v.x), "r"(v.y) : "memory");
 }
 
 template <int NT, int C>  // NT token tiles of 16 (M <= 16 NT), clusters of C CTAs
@@ -80,8 +78,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
 
   unsigned char* ring = smem;
   unsigned char* act = ring + (size_t)p.stages * kStageBytes;
-  int* tiles = reinterpret_cast<int*>(act + (size_t)MT * p.act_pitch);   // [block][token][8 channels]
-  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)p.max_blocks * MT * 8);
+  // partial tiles of the blocks this CTA finishes: [owned block][source CTA][token][8 channels]
+  int* tiles = reinterpret_cast<int*>(act + (size_t)MT * p.act_pitch);
+  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)((p.max_blocks + C - 1) / C) * C * MT * 8);
   uint64_t* empty = full + p.stages;
   volatile int* failed = reinterpret_cast<volatile int*>(empty + p.stages);
 
@@ -101,28 +100,33 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   if (tid == 32) *failed = 0;
   mbar_fence_init();
   __syncthreads();
+  if (C > 1) cluster_arrive_relaxed();  // "this CTA runs": awaited before the first remote store
   pdl_launch_dependents();
+  const uint32_t smask = (uint32_t)p.stages - 1u;
+  const int sshift = 31 - __clz(p.stages);
 
   if (warp == kConsumerWarps) {
     // ---------------- producer ------------------------------------------------------------------
-    // Piece i = (round r, part q, warp w) -> ring stage i mod stages; the stage count is a
-    // multiple of 8, so a stage is always reused by the same warp.  The weights are constants:
-    // pieces that fit the ring are requested before the wait on the preceding kernel.
-    if (lane == 0) {
-      const int total = rounds * parts * kConsumerWarps;
-      for (int i = 0; i < total; ++i) {
-        const int w = i & (kConsumerWarps - 1), rq = i >> 3, r = rq / parts, q = rq - r * parts;
-        const int j = r * kConsumerWarps + w;
-        if (j >= n_blk) continue;
-        const int s = i % p.stages;
-        if (i >= p.stages && !mbar_wait_bounded(&empty[s], ((i / p.stages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT)) break;
-        const int ng = min(kPieceGroups, L - q * kPieceGroups);
-        const uint32_t bytes = (uint32_t)ng * XQ_GROUP_BYTES;
-        const unsigned char* src = p.W + ((size_t)(b0 + j) * p.k_groups + g0 + q * kPieceGroups) * XQ_GROUP_BYTES;
-        mbar_expect_tx(&full[s], bytes);
-        bulk_g2s(ring + (size_t)s * kStageBytes, src, bytes, &full[s]);
-      }
+    // Piece i = (round r, part q, warp w) -> ring stage i mod stages (a stage is always reused
+    // by the same consumer warp).  Lane l owns ring stage l and issues its pieces l, l + stages,
+    // ... in order, so it sees every phase of that stage's "empty" barrier in turn (a one-bit
+    // parity cannot tell phase n from phase n + 2); one lane alone would be far too slow to feed
+    // the copy engine.  The weights are constants: nothing here waits for the preceding kernel.
+    const int total = rounds * parts * kConsumerWarps;
+    for (int i = lane; i < total && lane < p.stages; i += p.stages) {
+      const int w = i & (kConsumerWarps - 1), rq = i >> 3, r = rq / parts, q = rq - r * parts;
+      const int j = r * kConsumerWarps + w;
+      if (j >= n_blk) continue;
+      const int s = i & smask;
+      if (i >= p.stages && !mbar_wait_bounded(&empty[s], ((i >> sshift) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT)) break;
+      const int ng = min(kPieceGroups, L - q * kPieceGroups);
+      const uint32_t bytes = (uint32_t)ng * XQ_GROUP_BYTES;
+      const unsigned char* src = p.W + ((size_t)(b0 + j) * p.k_groups + g0 + q * kPieceGroups) * XQ_GROUP_BYTES;
+      mbar_expect_tx(&full[s], bytes);
+      bulk_g2s(ring + (size_t)s * kStageBytes, src, bytes, &full[s]);
     }
+    __syncwarp();
+    if (C > 1) cluster_wait_acquire();
   } else {
     // ---------------- consumers ----------------------------------------------------------------
     // token rows beyond M are zero
@@ -165,6 +169,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       }
     }
     bar_sync(1, kConsumerThreads);
+    if (C > 1) cluster_wait_acquire();  // every CTA of the cluster has started: remote stores are legal
 
     const int ag = lane >> 2, at = lane & 3;  // MMA fragment coordinates: channel / token row, word
     bool ok = true;
@@ -178,11 +183,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         for (int c = 0; c < 2; ++c) acc[a][c][0] = acc[a][c][1] = acc[a][c][2] = acc[a][c][3] = 0;
       for (int q = 0; q < parts && ok; ++q) {
         const int i = (r * parts + q) * kConsumerWarps + warp;
-        const int s = i % p.stages;
-        ok = mbar_wait_bounded(&full[s], (i / p.stages) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+        const int s = i & smask;
+        ok = mbar_wait_bounded(&full[s], (i >> sshift) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
         if (!ok) break;
         const int ng = min(kPieceGroups, L - q * kPieceGroups);
         const unsigned char* wp = ring + (size_t)s * kStageBytes + lane * 4;  // channel ag, word at of group 0
+#pragma unroll 2
         for (int gq = 0; gq < ng; gq += 4, wp += 4 * XQ_GROUP_BYTES) {
           const int nv = min(4, ng - gq);  // groups of this chunk that exist
           uint32_t b[4][2];
@@ -210,30 +216,45 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[s]);
       }
-      // D fragment: (token ag, channels 2 at, 2 at + 1), (token ag + 8, same channels)
-      int* tl = tiles + (size_t)j * MT * 8;
+      // D fragment: (token ag, channels 2 at, 2 at + 1), (token ag + 8, same channels) -> the
+      // tile [j / C][rank] in the shared memory of CTA j mod C
+      const int owner = j % C;
+      int* tl = tiles + ((size_t)(j / C) * C + rank) * MT * 8;
 #pragma unroll
       for (int a = 0; a < NT; ++a) {
-        *reinterpret_cast<int2*>(&tl[(16 * a + ag) * 8 + 2 * at]) = make_int2(acc[a][0][0] + acc[a][1][0], acc[a][0][1] + acc[a][1][1]);
-        *reinterpret_cast<int2*>(&tl[(16 * a + ag + 8) * 8 + 2 * at]) = make_int2(acc[a][0][2] + acc[a][1][2], acc[a][0][3] + acc[a][1][3]);
+        const int2 v0 = make_int2(acc[a][0][0] + acc[a][1][0], acc[a][0][1] + acc[a][1][1]);
+        const int2 v1 = make_int2(acc[a][0][2] + acc[a][1][2], acc[a][0][3] + acc[a][1][3]);
+        int* d0 = &tl[(16 * a + ag) * 8 + 2 * at];
+        int* d1 = &tl[(16 * a + ag + 8) * 8 + 2 * at];
+        if (owner == rank) {
+          *reinterpret_cast<int2*>(d0) = v0;
+          *reinterpret_cast<int2*>(d1) = v1;
+        } else {
+          st_cluster_v2(d0, (uint32_t)owner, v0);
+          st_cluster_v2(d1, (uint32_t)owner, v1);
+        }
       }
     }
   }
 
   // ---------------- meet the other K slices and finish ------------------------------------------
-  if (C > 1) cluster_sync_all(); else __syncthreads();
+  if (C > 1) {
+    cluster_arrive_release();
+    cluster_wait_acquire();
+  } else {
+    __syncthreads();
+  }
   if (warp < kConsumerWarps && !*failed) {
-    // CTA `rank` finishes blocks j = rank, rank + C, ...: one thread per (block, token)
+    // this CTA finishes blocks j = rank, rank + C, ...: one thread per (block, token)
     const int mine = (n_blk - rank + C - 1) / C;
     for (int idx = tid; idx < mine * p.M; idx += kConsumerThreads) {
       const int jj = idx / p.M, m = idx - jj * p.M;
       const int j = rank + jj * C;
-      const int* row = tiles + ((size_t)j * MT + m) * 8;
+      const int* row = tiles + ((size_t)jj * C * MT + m) * 8;
       int4 lo = *reinterpret_cast<const int4*>(row), hi = *reinterpret_cast<const int4*>(row + 4);
 #pragma unroll
       for (int o = 1; o < C; ++o) {
-        const uint32_t peer = (uint32_t)((rank + o) % C);
-        const int4 l2 = ld_cluster_v4(row, peer), h2 = ld_cluster_v4(row + 4, peer);
+        const int4 l2 = *reinterpret_cast<const int4*>(row + o * MT * 8), h2 = *reinterpret_cast<const int4*>(row + o * MT * 8 + 4);
         lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
         hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
       }
@@ -266,7 +287,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       }
     }
   }
-  if (C > 1) cluster_sync_all();  // nobody leaves while a peer may still read its tiles
 }
 
 struct DecodePlan {
@@ -352,15 +372,15 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
       if (clusters < 1) break;
       const int nc = clusters < n_blocks ? clusters : n_blocks;
       const int max_blocks = (n_blocks + nc - 1) / nc;
-      const size_t tiles = (size_t)max_blocks * MT * 8 * 4;
+      const size_t tiles = (size_t)((max_blocks + C - 1) / C) * C * MT * 8 * 4;
       const size_t misc = 2 * kMaxStages * 8 + 64 + 128;
       if (act + tiles + misc + 8 * (size_t)kStageBytes > cap) break;
       const int parts = (Lmax + kPieceGroups - 1) / kPieceGroups;
       const int rounds = (max_blocks + kConsumerWarps - 1) / kConsumerWarps;
-      int s = (int)((cap - act - tiles - misc) / kStageBytes) / 8 * 8;
-      if (s > kMaxStages) s = kMaxStages;
-      const int want = (rounds * parts * kConsumerWarps + 7) / 8 * 8;
-      if (s > want) s = want;
+      const int room = (int)((cap - act - tiles - misc) / kStageBytes);
+      const int want = rounds * parts * kConsumerWarps;
+      int s = 8;
+      while (2 * s <= kMaxStages && 2 * s <= room && s < want) s *= 2;
       const size_t smem = act + tiles + misc + (size_t)s * kStageBytes;
       const int fit = max_active_clusters(w->device, d.nt, C, smem);
       if (fit < 1) break;
