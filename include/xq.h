@@ -130,6 +130,37 @@ xq_status xq_expanded_linear(const void* X_bf16_dev, int32_t M, int64_t ldx, con
 xq_status xq_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_weights* w,
                                   void* out_bf16_host, void* ws_dev, size_t ws_bytes, void* stream);
 
+/* The whole layer for callers that cannot allocate device memory.  (No counterpart in the paper:
+ * this is a deployment variant of xq_expanded_linear, same arithmetic, same kernels.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host
+ * application that owns the whole memory pool and hands out nothing at run time, a real-time
+ * loop that may not take the allocator's locks or its implicit synchronization, a process
+ * that already sits at its memory limit.  Such a caller has buffers for its inputs and outputs
+ * but nowhere to put the workspace that xq_expanded_linear asks for.
+ *
+ * Here the intermediate results (packed INT4 codes of the M tokens, their M scales, the status
+ * word) are kept in a fixed 4 MiB array that is part of the library image; every GPU on which
+ * the library is used holds those 4 MiB until the process exits.  The call itself performs no
+ * allocation of any kind: it looks up the array, clears the status word and enqueues the same
+ * two kernels as xq_expanded_linear on `stream`.
+ *
+ * Limit: 256 + roundup256(M * Kp / 2) + roundup256(4 * M) bytes must fit in 4 MiB (about 3800
+ * tokens at Kp = 2176, 540 at Kp = 15360); larger calls return XQ_ERR_WORKSPACE and launch
+ * nothing.
+ * First call on each device: it asks the runtime for the array's device address (with that
+ * device current) and remembers it; make this first call outside any stream capture.
+ * Sharing: all calls on one device use the same array, which keeps the previous call's
+ * contents.  Calls that may overlap on the GPU (different streams, or the same stream with
+ * programmatic overlap you arranged yourself) race on it: serialize them.  Calls issued one
+ * after another on one stream are safe.
+ * A device-side time-out of this path cannot be read with xq_poll_status (there is no
+ * caller-visible workspace); X, out, w as in xq_expanded_linear.
+ * Errors: INVALID_ARG (null or misaligned pointer, bad ldx, device index above 63), WORKSPACE
+ * (does not fit the array), CUDA (a runtime call or launch failed). */
+xq_status xq_expanded_linear_static(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w,
+                                    void* out_bf16_dev, void* stream);
+
 /* Synchronizes `stream` and returns the sticky device status stored in the workspace (XQ_OK,
  * XQ_ERR_TIMEOUT or XQ_ERR_BOUNDS), or XQ_ERR_CUDA if the stream itself reports an error. */
 xq_status xq_poll_status(const void* ws_dev, void* stream);

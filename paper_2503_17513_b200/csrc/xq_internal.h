@@ -57,6 +57,9 @@ struct xq_ws_layout {
 };
 xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
 
+// Size of the built-in scratch array of xq_expanded_linear_static.
+constexpr size_t XQ_STATIC_SCRATCH_BYTES = 4u << 20;
+
 constexpr int XQ_MAX_P = 256;
 constexpr int XQ_DECODE_MAX_M = 32;
 

@@ -36,7 +36,7 @@ class HadamardPlan(ctypes.Structure):
 EXPORTS = [
     "xq_status_string", "xq_hadamard_plan", "xq_prepare_weights", "xq_weights_import", "xq_weights_export",
     "xq_weights_info", "xq_weights_free", "xq_workspace_bytes", "xq_workspace_init", "xq_rotate_quant",
-    "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status",
+    "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status", "xq_expanded_linear_static",
 ]
 
 
@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         L.xq_expanded_linear.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_poll_status.argtypes = [vp, vp]
+        L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes"):
                 getattr(L, name).restype = ctypes.c_int
@@ -194,6 +195,15 @@ def xq_expanded_linear_host(X_host, w: Weights, out_host, ws, M=None, stream=Non
     _check(lib().xq_expanded_linear_host(ctypes.c_void_p(X_host.data_ptr()), M, w.handle,
                                          ctypes.c_void_p(out_host.data_ptr()), _dp(ws), ws.numel() * ws.element_size(),
                                          _stream(stream)), "xq_expanded_linear_host")
+
+
+def xq_expanded_linear_static(X, w: Weights, out, M=None, ldx=None, stream=None) -> None:
+    """The layer without a caller workspace: intermediates live in the library's built-in 4 MiB
+    device array (for callers that must not allocate).  Calls share that array: do not overlap them."""
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_expanded_linear_static(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _stream(stream)),
+           "xq_expanded_linear_static")
 
 
 def xq_poll_status(ws, stream=None) -> int:
