@@ -98,11 +98,25 @@ def test_plan_factors_the_workload_and_paper_sizes(oracle):
         oracle.plan(4, 6)  # 6 = 3 * 2: no Hadamard matrix of order 6
 
 
-def test_table1_layer_sizes_are_down_proj_in_channels():
-    """Table 1: growing the 16 (1B) / 32 (8B) down projections from 8192 to 8960 (14336 to
-    15360) input channels accounts for the printed model-size increase, so 'layer size' is K'."""
-    assert abs((1.235e9 + 16 * 2048 * (8960 - 8192)) / 1e9 - 1.260) < 1e-3
-    assert abs((7.504e9 + 32 * 4096 * (15360 - 14336)) / 1e9 - 7.638) < 1e-3
+def test_table1_layer_sizes_are_down_proj_in_channels(oracle):
+    """Table 1 (values in tests/golden/table1_sizes.txt): the printed model sizes grow by exactly
+    layers x hidden x (channels - base channels), so the 'layer size' column is the K' of the down
+    projection, and every printed K' is an order the plan function can factor."""
+    import os
+
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "table1_sizes.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                m, layers, hidden, base, ch, size = line.split()
+                rows.append((m, int(layers), int(hidden), int(base), int(ch), float(size)))
+    assert len(rows) == 15
+    base_size = {m: size for m, _, _, base, ch, size in rows if base == ch}
+    for m, layers, hidden, base, ch, size in rows:
+        predicted = base_size[m] + layers * hidden * (ch - base) / 1e9
+        assert abs(predicted - size) < 1.5e-3, (m, ch, predicted, size)  # printed to three decimals
+        pl = oracle.plan(base, ch)
+        assert pl.p * (1 << pl.log2n) == ch
 
 
 @pytest.mark.parametrize("K,Kp", [(100, 136), (200, 240), (130, 144), (64, 64), (2048, 2176)])
