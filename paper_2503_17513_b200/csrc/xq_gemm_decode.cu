@@ -2,22 +2,26 @@
 // packed INT4 weights once from HBM (paper Sec. 3: the quantized product Q(XR) Q(W~) computed at
 // inference; here the case where the weight stream, not the arithmetic, sets the time).
 //
-// Decomposition.  Output channels are handled in blocks of 8; a thread-block cluster of C CTAs
+// Decomposition.  Output channels are handled in blocks of 16; a thread-block cluster of C CTAs
 // owns a contiguous range of blocks and cuts K between its CTAs in multiples of 32 codes, so a
-// CTA needs only its K slice of the quantized tokens.  In the weight layout the K slice of one
-// block is one contiguous run of bytes; a producer warp fetches runs with bulk copies (pieces of
-// at most 4 KiB) into a shared-memory ring, the first ring-full before the kernel waits for its
-// predecessor in the stream.  Each of the eight consumer warps owns whole blocks (block j of
-// the range goes to warp j mod 8), so a block's partial sums stay in one warp's registers:
-// MMA i of a chunk of four 32-code groups takes group i; lane (channel g, word t) loads its word
-// of eight codes with one conflict-free 32-bit load, the nibble split turns it into the B
-// fragment of an m16n8k32 integer MMA (even codes in K slots 4t.., odd codes in 16+4t..), and the
-// A fragments (16 tokens) come from the token slice that the CTA expanded once into shared
-// memory in exactly that fragment order.  Block j is finished by CTA j mod C
-// of the cluster: every CTA stores its partial tile of the block into that CTA's shared memory
-// (distributed shared memory), and after one cluster barrier the owner sums the C tiles and
-// applies the epilogue (scales, bf16, 16-byte stores).  No global scratch, no atomics, and no
-// CTA waits on another outside the cluster barrier.
+// CTA needs only its K slice of the quantized tokens.  Inside a CTA the slice of a block is cut
+// once more into S sub-slices so that there are about as many work items (block, sub-slice) as
+// consumer warps; item t goes to warp t mod 16 and its partial sums stay in that warp's
+// registers.  In the weight layout an item is one contiguous run of bytes; a producer warp
+// fetches it in P pieces of at most 4 KiB with bulk copies into a shared-memory ring (lane l owns
+// stage l), the first ring-full before the kernel waits for its predecessor in the stream.
+//
+// Arithmetic.  The weights are the 16-row A operand of m16n8k32 integer MMAs and eight tokens the
+// B operand: shared-memory traffic per weight byte is what bounds this kernel after HBM, and this
+// orientation reads the fewest token bytes.  MMA i of a chunk of four 32-code groups takes group
+// i; lane (g, t) loads word t (eight codes) of channels g and g + 8 with two conflict-free 32-bit
+// loads, the nibble split (16 x code in each byte) puts the even codes in K slots 4t.. and the odd
+// codes in 16+4t..; the token fragments come from the token slice that the CTA expanded once into
+// shared memory in exactly that order.  Block j is finished by CTA j mod C of the cluster: every
+// warp stores the partial tile of its item into that CTA's shared memory (distributed shared
+// memory), and after one cluster barrier the owner sums the C * S tiles and applies the epilogue
+// (exact >> 8, scales, bf16, 16-byte stores).  No global scratch, no atomics, and no CTA waits on
+// another outside the cluster barrier.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -29,12 +33,13 @@ using namespace xqptx;
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = 16;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;
-constexpr int kPieceGroups = 32;                               // 32-code groups per ring stage
-constexpr int kStageBytes = kPieceGroups * XQ_GROUP_BYTES;     // 4 KiB
-constexpr int kMaxStages = 32;
+constexpr int kChunkBytes = 4 * XQ_GROUP_BYTES;              // 1 KiB: 16 channels x 128 codes
+constexpr int kPieceChunks = 4;                              // chunks per ring stage
+constexpr int kStageBytes = kPieceChunks * kChunkBytes;      // 4 KiB
+constexpr int kMaxStages = 48;
 
 struct DecodeParams {
   const uint8_t* W;
@@ -46,10 +51,12 @@ struct DecodeParams {
   int32_t* status;
   int M, N, Kp;
   int k_groups;     // groups of 32 codes per channel block in the weight layout (K'' / 32)
-  int n_blocks;     // channel blocks holding real channels: ceil(N / 8)
-  int stages;       // ring stages: 8, 16 or 32
+  int n_blocks;     // channel blocks holding real channels: ceil(N / 16)
+  int stages;       // ring stages: 16, 32 or 48
   int act_pitch;    // bytes between token rows of the expanded token slice
   int max_blocks;   // blocks in the longest cluster range
+  int log2S;        // sub-slices per block and CTA: S = 1 << log2S
+  int P;            // ring pieces per work item
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -68,19 +75,20 @@ __device__ __forceinline__ void st_cluster_v2(void* local_ptr, uint32_t rank, in
   asm volatile("st.shared::cluster.v2.s32 [%0], {%1, %2};" ::"r"(remote), "r"(v.x), "r"(v.y) : "memory");
 }
 
-template <int NT, int C>  // NT token tiles of 16 (M <= 16 NT), clusters of C CTAs
+template <int NT, int C>  // NT token tiles of 8 (M <= 8 NT), clusters of C CTAs
 __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  constexpr int MT = 16 * NT;  // padded token count
-  const int rank = C == 1 ? 0 : (int)cluster_ctarank();
+  constexpr int MT = 8 * NT;  // padded token count
+  const int rank = (int)cluster_ctarank();
   const int cid = blockIdx.x / C, n_clusters = gridDim.x / C;
 
   unsigned char* ring = smem;
   unsigned char* act = ring + (size_t)p.stages * kStageBytes;
-  // partial tiles of the blocks this CTA finishes: [owned block][source CTA][token][8 channels]
+  // partial tiles of the blocks this CTA finishes: [owned block][source CTA, sub-slice][16 channels][MT tokens]
+  const int S = 1 << p.log2S, srcs = C * S;
   int* tiles = reinterpret_cast<int*>(act + (size_t)MT * p.act_pitch);
-  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)((p.max_blocks + C - 1) / C) * C * MT * 8);
+  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)((p.max_blocks + C - 1) / C) * srcs * 16 * MT);
   uint64_t* empty = full + p.stages;
   volatile int* failed = reinterpret_cast<volatile int*>(empty + p.stages);
 
@@ -89,46 +97,108 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   const int n_blk = b1 - b0;
   const int groups = p.Kp / XQ_K_GROUP;
   const int g0 = rank * groups / C, g1 = (rank + 1) * groups / C;
-  const int L = g1 - g0;                                  // groups in the slice
-  const int parts = (L + kPieceGroups - 1) / kPieceGroups;  // ring pieces per block
-  const int rounds = (n_blk + kConsumerWarps - 1) / kConsumerWarps;
+  const int L = g1 - g0;               // groups in the slice
+  const int n_chunks = (L + 3) >> 2;   // chunks of four groups
+  const int n_items = n_blk << p.log2S, parts = p.P;
+  const int rounds = (n_items + kConsumerWarps - 1) / kConsumerWarps;
+  // item t = (block t >> log2S, sub-slice u = t & (S - 1)) covers chunks [u n_chunks / S, (u + 1) n_chunks / S);
+  // its piece q covers chunks [lo + q len / P, lo + (q + 1) len / P)
+  auto piece_range = [&](int u, int q, int& c_lo, int& c_hi) {
+    const int lo = (u * n_chunks) >> p.log2S, len = (((u + 1) * n_chunks) >> p.log2S) - lo;
+    if (parts == 1) {
+      c_lo = lo;
+      c_hi = lo + len;
+    } else {
+      c_lo = lo + q * len / parts;
+      c_hi = lo + (q + 1) * len / parts;
+    }
+  };
 
   if (tid < p.stages) {
     mbar_init(&full[tid], 1);
     mbar_init(&empty[tid], 1);
   }
+  if (tid == 33) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.sx));
   if (tid == 32) *failed = 0;
   mbar_fence_init();
   __syncthreads();
-  if (C > 1) cluster_arrive_relaxed();  // "this CTA runs": awaited before the first remote store
+  cluster_arrive_relaxed();  // "this CTA runs": awaited before the first remote store
   pdl_launch_dependents();
-  const uint32_t smask = (uint32_t)p.stages - 1u;
-  const int sshift = 31 - __clz(p.stages);
 
   if (warp == kConsumerWarps) {
     // ---------------- producer ------------------------------------------------------------------
-    // Piece i = (round r, part q, warp w) -> ring stage i mod stages (a stage is always reused
-    // by the same consumer warp).  Lane l owns ring stage l and issues its pieces l, l + stages,
-    // ... in order, so it sees every phase of that stage's "empty" barrier in turn (a one-bit
-    // parity cannot tell phase n from phase n + 2); one lane alone would be far too slow to feed
-    // the copy engine.  The weights are constants: nothing here waits for the preceding kernel.
-    const int total = rounds * parts * kConsumerWarps;
-    for (int i = lane; i < total && lane < p.stages; i += p.stages) {
-      const int w = i & (kConsumerWarps - 1), rq = i >> 3, r = rq / parts, q = rq - r * parts;
-      const int j = r * kConsumerWarps + w;
-      if (j >= n_blk) continue;
-      const int s = i & smask;
-      if (i >= p.stages && !mbar_wait_bounded(&empty[s], ((i >> sshift) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT)) break;
-      const int ng = min(kPieceGroups, L - q * kPieceGroups);
-      const uint32_t bytes = (uint32_t)ng * XQ_GROUP_BYTES;
-      const unsigned char* src = p.W + ((size_t)(b0 + j) * p.k_groups + g0 + q * kPieceGroups) * XQ_GROUP_BYTES;
-      mbar_expect_tx(&full[s], bytes);
-      bulk_g2s(ring + (size_t)s * kStageBytes, src, bytes, &full[s]);
+    // Warp w's n-th piece (n = round * P + part) goes to ring stage w + 16 (n mod slots), slots =
+    // stages / 16.  Every stage is served by one lane, which issues that stage's pieces in order
+    // and so sees every phase of its "empty" barrier in turn (a one-bit parity cannot tell phase
+    // n from phase n + 2).  The lanes poll together with the
+    // non-blocking probe: a lane suspended inside a blocking wait would hold up the lanes whose
+    // stages are already free.  The weights are constants: nothing here waits for the preceding
+    // kernel.
+    // Lane l serves the stages l and (with 48 stages) l + 32, one after the other in piece order.
+    const int w = lane & (kConsumerWarps - 1);
+    const int per_round = p.stages / kConsumerWarps;   // ring slots per warp: 1, 2 or 3
+    // this lane's k-th piece has slot index n(k) in its warp's sequence of (round, part) pairs:
+    // slots with n mod per_round == lane / 16 (and == 2 for lanes 0..15 when per_round == 3)
+    int n = lane >> 4;                                 // index into the warp's piece sequence
+    uint32_t use_a = 0, use_b = 0;                     // fills so far of stage lane and stage lane + 32
+    bool active = (lane >> 4) < per_round;
+    const int total_n = rounds * parts;                // pieces of one warp, counting missing items
+    auto exists = [&](int nn) { return nn < total_n && (nn / parts) * kConsumerWarps + w < n_items; };
+    auto next_n = [&](int nn) {                        // the next slot this lane serves after nn
+      if (per_round == 3 && lane < 16) return (nn % 3 == 0) ? nn + 2 : nn + 1;  // residues 0 and 2
+      if (per_round == 3) return nn + 3;                                         // residue 1
+      return nn + per_round;
+    };
+    if (active && !exists(n)) active = false;
+    uint32_t idle = 0;
+    uint64_t t_idle = 0;
+    while (__any_sync(0xffffffffu, active)) {
+      bool ready = false;
+      int stage = 0;
+      if (active) {
+        const bool second = (per_round == 3 && lane < 16 && n % 3 == 2);
+        stage = second ? lane + 32 : lane;
+        const uint32_t use = second ? use_b : use_a;
+        ready = use == 0 || mbar_test(&empty[stage], (use - 1) & 1);
+      }
+      if (ready) {
+        const int r = n / parts, q = n - r * parts;
+        const int t = r * kConsumerWarps + w;
+        int c_lo, c_hi;
+        piece_range(t & (S - 1), q, c_lo, c_hi);
+        const int ng = min(4 * c_hi, L) - 4 * c_lo;
+        const uint32_t bytes = (uint32_t)ng * XQ_GROUP_BYTES;
+        const unsigned char* src = p.W + ((size_t)(b0 + (t >> p.log2S)) * p.k_groups + g0 + 4 * c_lo) * XQ_GROUP_BYTES;
+        mbar_expect_tx(&full[stage], bytes);
+        bulk_g2s(ring + (size_t)stage * kStageBytes, src, bytes, &full[stage]);
+        if (stage == lane) ++use_a; else ++use_b;
+        n = next_n(n);
+        if (!exists(n)) active = false;
+      }
+      if (__any_sync(0xffffffffu, ready)) {
+        idle = 0;
+      } else {
+        __nanosleep(40);
+        if ((++idle & 255u) == 0u) {  // nothing moved for a while: bounded, like every other wait
+          const uint64_t now = globaltimer_ns();
+          if (idle == 256u) t_idle = now;
+          if (*failed || now - t_idle > 1000000000ull) {
+            if (lane == 0 && !*failed) {
+              *failed = 1;
+              atomicExch(p.status, (int)XQ_ERR_TIMEOUT);
+            }
+            break;
+          }
+        }
+      }
     }
     __syncwarp();
-    if (C > 1) cluster_wait_acquire();
+    cluster_wait_acquire();
   } else {
     // ---------------- consumers ----------------------------------------------------------------
+    // the epilogue's channel scales: bring them into L2 now, they are constants
+    for (int i = tid * 32; i < n_blk * 16; i += kConsumerThreads * 32)
+      if (b0 * 16 + i < p.N) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.sw + b0 * 16 + i));
     // token rows beyond M are zero
     for (int i = tid; i < (MT - p.M) * (p.act_pitch / 16); i += kConsumerThreads)
       reinterpret_cast<uint4*>(act + (size_t)p.M * p.act_pitch)[i] = make_uint4(0, 0, 0, 0);
@@ -169,63 +239,67 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       }
     }
     bar_sync(1, kConsumerThreads);
-    if (C > 1) cluster_wait_acquire();  // every CTA of the cluster has started: remote stores are legal
+    cluster_wait_acquire();  // every CTA of the cluster has started: remote stores are legal
 
-    const int ag = lane >> 2, at = lane & 3;  // MMA fragment coordinates: channel / token row, word
+    const int ag = lane >> 2, at = lane & 3;  // MMA fragment coordinates: channel row / token column, word
     bool ok = true;
     for (int r = 0; r < rounds && ok; ++r) {
-      const int j = r * kConsumerWarps + warp;
-      if (j >= n_blk) break;
-      int acc[NT][2][4];
+      const int t = r * kConsumerWarps + warp;
+      if (t >= n_items) break;
+      const int j = t >> p.log2S, u = t & (S - 1);
+      int acc[NT][4][4];  // one chain per MMA of a chunk: the integer MMA has a long latency
 #pragma unroll
       for (int a = 0; a < NT; ++a)
 #pragma unroll
-        for (int c = 0; c < 2; ++c) acc[a][c][0] = acc[a][c][1] = acc[a][c][2] = acc[a][c][3] = 0;
+        for (int c = 0; c < 4; ++c) acc[a][c][0] = acc[a][c][1] = acc[a][c][2] = acc[a][c][3] = 0;
       for (int q = 0; q < parts && ok; ++q) {
-        const int i = (r * parts + q) * kConsumerWarps + warp;
-        const int s = i & smask;
-        ok = mbar_wait_bounded(&full[s], (i >> sshift) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+        // this warp's n-th piece sits in ring stage warp + 16 (n mod slots), in its (n / slots)-th use
+        const int n = r * parts + q, per_round = p.stages / kConsumerWarps;
+        const int s = warp + kConsumerWarps * (n % per_round);
+        ok = mbar_wait_bounded(&full[s], (n / per_round) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
         if (!ok) break;
-        const int ng = min(kPieceGroups, L - q * kPieceGroups);
-        const unsigned char* wp = ring + (size_t)s * kStageBytes + lane * 4;  // channel ag, word at of group 0
+        int c_lo, c_hi;
+        piece_range(u, q, c_lo, c_hi);
+        const int ng = min(4 * c_hi, L) - 4 * c_lo;
+        const unsigned char* wp = ring + (size_t)s * kStageBytes + lane * 4;  // channel ag (and ag + 8 at +128), word at
+        const unsigned char* ap = act + (size_t)ag * p.act_pitch + (size_t)c_lo * 128 + (size_t)at * 32;
 #pragma unroll 2
-        for (int gq = 0; gq < ng; gq += 4, wp += 4 * XQ_GROUP_BYTES) {
+        for (int gq = 0; gq < ng; gq += 4, wp += kChunkBytes, ap += 128) {
           const int nv = min(4, ng - gq);  // groups of this chunk that exist
-          uint32_t b[4][2];
+          uint32_t a[4][4];
 #pragma unroll
           for (int i4 = 0; i4 < 4; ++i4) {
-            const uint32_t wv = i4 < nv ? *reinterpret_cast<const uint32_t*>(wp + i4 * XQ_GROUP_BYTES) : 0u;
-            split16(wv, b[i4][0], b[i4][1]);
+            uint32_t lo = 0u, hi = 0u;
+            if (i4 < nv) {
+              lo = *reinterpret_cast<const uint32_t*>(wp + i4 * XQ_GROUP_BYTES);
+              hi = *reinterpret_cast<const uint32_t*>(wp + i4 * XQ_GROUP_BYTES + 128);
+            }
+            split16(lo, a[i4][0], a[i4][2]);  // channel ag: even codes -> K slots 4 at.., odd -> 16 + 4 at..
+            split16(hi, a[i4][1], a[i4][3]);  // channel ag + 8
           }
-          const size_t coff = (size_t)(q * (kPieceGroups / 4) + (gq >> 2)) * 128 + (size_t)at * 32;
 #pragma unroll
-          for (int a = 0; a < NT; ++a) {
-            const uint4* lo = reinterpret_cast<const uint4*>(act + (size_t)(16 * a + ag) * p.act_pitch + coff);
-            const uint4* hi = reinterpret_cast<const uint4*>(act + (size_t)(16 * a + ag + 8) * p.act_pitch + coff);
-            const uint4 x0 = lo[0], x1 = lo[1], y0 = hi[0], y1 = hi[1];
-            const uint32_t a0[4] = {x0.x, y0.x, x0.y, y0.y};
-            const uint32_t a1[4] = {x0.z, y0.z, x0.w, y0.w};
-            const uint32_t a2[4] = {x1.x, y1.x, x1.y, y1.y};
-            const uint32_t a3[4] = {x1.z, y1.z, x1.w, y1.w};
-            mma_s8_16x8x32(acc[a][0], a0, b[0][0], b[0][1]);
-            mma_s8_16x8x32(acc[a][1], a1, b[1][0], b[1][1]);
-            mma_s8_16x8x32(acc[a][0], a2, b[2][0], b[2][1]);
-            mma_s8_16x8x32(acc[a][1], a3, b[3][0], b[3][1]);
+          for (int n = 0; n < NT; ++n) {
+            const uint4* xp = reinterpret_cast<const uint4*>(ap + (size_t)(8 * n) * p.act_pitch);
+            const uint4 x0 = xp[0], x1 = xp[1];  // token 8 n + ag: (even, odd) of word at of groups 0..3
+            mma_s8_16x8x32(acc[n][0], a[0], x0.x, x0.y);
+            mma_s8_16x8x32(acc[n][1], a[1], x0.z, x0.w);
+            mma_s8_16x8x32(acc[n][2], a[2], x1.x, x1.y);
+            mma_s8_16x8x32(acc[n][3], a[3], x1.z, x1.w);
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[s]);
       }
-      // D fragment: (token ag, channels 2 at, 2 at + 1), (token ag + 8, same channels) -> the
-      // tile [j / C][rank] in the shared memory of CTA j mod C
+      // D fragment: (channel ag, tokens 2 at, 2 at + 1), (channel ag + 8, same tokens) -> the
+      // tile [j / C][rank * S + u] in the shared memory of CTA j mod C
       const int owner = j % C;
-      int* tl = tiles + ((size_t)(j / C) * C + rank) * MT * 8;
+      int* tl = tiles + ((size_t)(j / C) * srcs + rank * S + u) * 16 * MT;
 #pragma unroll
-      for (int a = 0; a < NT; ++a) {
-        const int2 v0 = make_int2(acc[a][0][0] + acc[a][1][0], acc[a][0][1] + acc[a][1][1]);
-        const int2 v1 = make_int2(acc[a][0][2] + acc[a][1][2], acc[a][0][3] + acc[a][1][3]);
-        int* d0 = &tl[(16 * a + ag) * 8 + 2 * at];
-        int* d1 = &tl[(16 * a + ag + 8) * 8 + 2 * at];
+      for (int n = 0; n < NT; ++n) {
+        const int2 v0 = make_int2(acc[n][0][0] + acc[n][1][0] + acc[n][2][0] + acc[n][3][0], acc[n][0][1] + acc[n][1][1] + acc[n][2][1] + acc[n][3][1]);
+        const int2 v1 = make_int2(acc[n][0][2] + acc[n][1][2] + acc[n][2][2] + acc[n][3][2], acc[n][0][3] + acc[n][1][3] + acc[n][2][3] + acc[n][3][3]);
+        int* d0 = &tl[ag * MT + 8 * n + 2 * at];
+        int* d1 = &tl[(ag + 8) * MT + 8 * n + 2 * at];
         if (owner == rank) {
           *reinterpret_cast<int2*>(d0) = v0;
           *reinterpret_cast<int2*>(d1) = v1;
@@ -238,41 +312,39 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   }
 
   // ---------------- meet the other K slices and finish ------------------------------------------
-  if (C > 1) {
-    cluster_arrive_release();
-    cluster_wait_acquire();
-  } else {
-    __syncthreads();
-  }
+  cluster_arrive_release();
+  cluster_wait_acquire();
   if (warp < kConsumerWarps && !*failed) {
-    // this CTA finishes blocks j = rank, rank + C, ...: one thread per (block, token)
+    // this CTA finishes blocks j = rank, rank + C, ...: one thread per (block, token, half of the channels)
     const int mine = (n_blk - rank + C - 1) / C;
-    for (int idx = tid; idx < mine * p.M; idx += kConsumerThreads) {
-      const int jj = idx / p.M, m = idx - jj * p.M;
+    for (int idx = tid; idx < mine * p.M * 2; idx += kConsumerThreads) {
+      const int h = idx & 1, bm = idx >> 1;
+      const int jj = bm / p.M, m = bm - jj * p.M;
       const int j = rank + jj * C;
-      const int* row = tiles + ((size_t)jj * C * MT + m) * 8;
-      int4 lo = *reinterpret_cast<const int4*>(row), hi = *reinterpret_cast<const int4*>(row + 4);
+      const int* col = tiles + (size_t)jj * srcs * 16 * MT + (8 * h) * MT + m;
+      int v[8];
 #pragma unroll
-      for (int o = 1; o < C; ++o) {
-        const int4 l2 = *reinterpret_cast<const int4*>(row + o * MT * 8), h2 = *reinterpret_cast<const int4*>(row + o * MT * 8 + 4);
-        lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
-        hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
+      for (int e = 0; e < 8; ++e) v[e] = col[e * MT];
+      for (int o = 1; o < srcs; ++o) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] += col[o * 16 * MT + e * MT];
       }
-      const int v[8] = {lo.x >> 8, lo.y >> 8, lo.z >> 8, lo.w >> 8, hi.x >> 8, hi.y >> 8, hi.z >> 8, hi.w >> 8};  // every product carries 16 x 16
-      const int n0 = (b0 + j) * 8;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] >>= 8;  // every product carries 16 x 16
+      const int n0 = (b0 + j) * 16 + 8 * h;
       const float sxm = p.sx[m];
       const size_t o = (size_t)m * p.N + n0;
       if (n0 + 8 <= p.N && (p.N & 7) == 0) {
         const float4 s0 = *reinterpret_cast<const float4*>(p.sw + n0), s1 = *reinterpret_cast<const float4*>(p.sw + n0 + 4);
         const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-        uint32_t h[4];
+        uint32_t hw[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const __nv_bfloat162 b2 = __halves2bfloat162(__float2bfloat16_rn((float)v[2 * e] * sxm * sc[2 * e]),
                                                        __float2bfloat16_rn((float)v[2 * e + 1] * sxm * sc[2 * e + 1]));
-          h[e] = *reinterpret_cast<const uint32_t*>(&b2);
+          hw[e] = *reinterpret_cast<const uint32_t*>(&b2);
         }
-        *reinterpret_cast<uint4*>(p.out + o) = make_uint4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<uint4*>(p.out + o) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
         if (p.acc_opt) {
           *reinterpret_cast<int4*>(p.acc_opt + o) = make_int4(v[0], v[1], v[2], v[3]);
           *reinterpret_cast<int4*>(p.acc_opt + o + 4) = make_int4(v[4], v[5], v[6], v[7]);
@@ -290,7 +362,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
 }
 
 struct DecodePlan {
-  int nt, C, stages, act_pitch, max_blocks, grid;
+  int nt, C, stages, act_pitch, max_blocks, grid, log2S, P;
   size_t smem;
 };
 
@@ -334,10 +406,12 @@ cudaError_t launch_variant(const DecodeParams& p, int grid, size_t smem, cudaStr
 cudaError_t dispatch(int nt, int C, const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
   if (C == 2) {
     if (nt == 1) return launch_variant<1, 2>(p, grid, smem, st, max_clusters);
-    return launch_variant<2, 2>(p, grid, smem, st, max_clusters);
+    if (nt == 2) return launch_variant<2, 2>(p, grid, smem, st, max_clusters);
+    return launch_variant<4, 2>(p, grid, smem, st, max_clusters);
   }
   if (nt == 1) return launch_variant<1, 4>(p, grid, smem, st, max_clusters);
-  return launch_variant<2, 4>(p, grid, smem, st, max_clusters);
+  if (nt == 2) return launch_variant<2, 4>(p, grid, smem, st, max_clusters);
+  return launch_variant<4, 4>(p, grid, smem, st, max_clusters);
 }
 
 int max_active_clusters(int device, int nt, int C, size_t smem) {
@@ -358,13 +432,13 @@ int max_active_clusters(int device, int nt, int C, size_t smem) {
 DecodePlan decode_plan(int M, const xq_weights* w) {
   DecodePlan d = {};
   if (M < 1 || M > XQ_DECODE_MAX_M || w->Kp % XQ_K_GROUP != 0) return d;
-  d.nt = M <= 16 ? 1 : 2;
-  const int MT = 16 * d.nt, groups = w->Kp / XQ_K_GROUP, n_blocks = (w->N + 7) / 8;
+  d.nt = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
+  const int MT = 8 * d.nt, groups = w->Kp / XQ_K_GROUP, n_blocks = (w->N + 15) / 16;
   const size_t cap = 227 * 1024;
   for (int C = 2; C <= 4; C *= 2) {
-    if (groups < C) break;
-    const int Lmax = (groups + C - 1) / C;
-    const int chunks = (Lmax + 3) / 4;
+    if (groups < 4 * C) break;
+    const int Lmax = (groups + C - 1) / C, Lmin = groups / C;
+    const int chunks = (Lmax + 3) / 4, chunks_min = (Lmin + 3) / 4;
     const int pitch = chunks * 128 + 16;  // 16 (mod 128): conflict-free 128-bit fragment reads
     const size_t act = (size_t)MT * pitch;
     // a first guess of the cluster count sizes the tiles; refined below with the occupancy answer
@@ -372,28 +446,36 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
       if (clusters < 1) break;
       const int nc = clusters < n_blocks ? clusters : n_blocks;
       const int max_blocks = (n_blocks + nc - 1) / nc;
-      const size_t tiles = (size_t)((max_blocks + C - 1) / C) * C * MT * 8 * 4;
+      // sub-slices: as few as give most consumer warps an item in the first round (long items keep
+      // several ring pieces in flight per warp), each item at least one chunk long
+      int log2S = 0;
+      while ((max_blocks << log2S) < 12 && (2 << log2S) <= chunks_min && log2S < 4) ++log2S;
+      const int S = 1 << log2S;
+      const int item_chunks_max = (chunks + S - 1) / S, item_chunks_min = chunks_min / S;
+      int P = (item_chunks_max + kPieceChunks - 1) / kPieceChunks;
+      while (P <= item_chunks_min && (item_chunks_max + P - 1) / P > kPieceChunks) ++P;  // uneven cuts: keep pieces <= 4 KiB
+      if (P < 1 || P > item_chunks_min) break;  // every piece holds at least one chunk
+      const size_t tiles = (size_t)((max_blocks + C - 1) / C) * C * S * 16 * MT * 4;
       const size_t misc = 2 * kMaxStages * 8 + 64 + 128;
-      if (act + tiles + misc + 8 * (size_t)kStageBytes > cap) break;
-      const int parts = (Lmax + kPieceGroups - 1) / kPieceGroups;
-      const int rounds = (max_blocks + kConsumerWarps - 1) / kConsumerWarps;
+      if (act + tiles + misc + 16 * (size_t)kStageBytes > cap) break;
       const int room = (int)((cap - act - tiles - misc) / kStageBytes);
-      const int want = rounds * parts * kConsumerWarps;
-      int s = 8;
-      while (2 * s <= kMaxStages && 2 * s <= room && s < want) s *= 2;
-      const size_t smem = act + tiles + misc + (size_t)s * kStageBytes;
+      const int want = ((max_blocks << log2S) + kConsumerWarps - 1) / kConsumerWarps * P * kConsumerWarps;
+      const int stg = (room >= 48 && want > 32) ? 48 : ((room >= 32 && want > 16) ? 32 : 16);
+      const size_t smem = act + tiles + misc + (size_t)stg * kStageBytes;
       const int fit = max_active_clusters(w->device, d.nt, C, smem);
       if (fit < 1) break;
-      if (pass == 1 || fit == clusters) {
+      if (pass == 1 || fit >= clusters) {
         d.C = C;
-        d.stages = s;
+        d.stages = stg;
         d.act_pitch = pitch;
         d.max_blocks = max_blocks;
         d.grid = nc * C;
         d.smem = smem;
+        d.log2S = log2S;
+        d.P = P;
         return d;
       }
-      clusters = fit < clusters ? fit : clusters;
+      clusters = fit;
     }
   }
   return d;
@@ -404,7 +486,7 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                                   int32_t* acc_opt, int32_t* status, cudaStream_t st) {
   const DecodePlan d = decode_plan(M, w);
-  if (d.stages < 8) return cudaErrorNotSupported;
+  if (d.stages < 16) return cudaErrorNotSupported;
   DecodeParams p;
   p.W = w->packed;
   p.sw = w->s_w;
@@ -417,9 +499,11 @@ cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M,
   p.N = w->N;
   p.Kp = w->Kp;
   p.k_groups = w->Kpp / XQ_K_GROUP;
-  p.n_blocks = (w->N + 7) / 8;
+  p.n_blocks = (w->N + 15) / 16;
   p.stages = d.stages;
   p.act_pitch = d.act_pitch;
   p.max_blocks = d.max_blocks;
+  p.log2S = d.log2S;
+  p.P = d.P;
   return dispatch(d.nt, d.C, p, d.grid, d.smem, st, nullptr);
 }

@@ -4,8 +4,8 @@
 // Tile: 128 tokens x 256 output channels, K in blocks of 128 codes.  A persistent CTA per SM
 // walks its tiles with four kinds of warps:
 //   producer (1 warp)   TMA: the packed activation tile (tensor map over the [M, K'/2] byte
-//                       matrix, out-of-range rows and columns read as zero) and 32 bulk copies
-//                       of 512 bytes of packed weights per K block, into a ring of packed stages;
+//                       matrix, out-of-range rows and columns read as zero) and 16 bulk copies
+//                       of 1 KiB of packed weights per K block, into a ring of packed stages;
 //   unpack   (8 warps)  expand packed nibbles to signed bytes (16 x the code: the nibble moved
 //                       to the top of its byte) and write them into the 128-byte-swizzled
 //                       K-major operand stages that tcgen05.mma reads;
@@ -121,8 +121,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
       const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-      // lane l fetches channel block l of the tile: 8 channels x 128 codes = 512 contiguous bytes
-      const unsigned char* wsrc = p.W + ((size_t)(tn * (BN / XQ_ROW_BLOCK) + lane) * p.KB) * (4 * XQ_GROUP_BYTES);
+      // lane l < 16 fetches channel block l of the tile: 16 channels x 128 codes = 1 KiB contiguous
+      const unsigned char* wsrc = p.W + ((size_t)(tn * (BN / XQ_ROW_BLOCK) + (lane & 15)) * p.KB) * (4 * XQ_GROUP_BYTES);
       for (int kb = 0; kb < p.KB; ++kb, ++it) {
         const int s = it % kPkStages;
         if (it >= (uint32_t)kPkStages) {
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
           tma_load_2d(stage, &mapA, kb * 64, tm * BM, &pk_full[s]);
         }
         __syncwarp();
-        bulk_g2s(stage + kPkABytes + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
+        if (lane < 16) bulk_g2s(stage + kPkABytes + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
       }
     }
   } else if (warp == 1) {
@@ -240,8 +240,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
           ok = mbar_wait_bounded(&i8_empty[u], ((it / kI8Stages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
           if (!ok) break;
         }
-        // A: 128 rows of 64 bytes.  B: 32 channel blocks of 512 bytes, piece 8t + g of a block =
-        // codes 32t..32t+31 of channel g.
+        // A: 128 rows of 64 bytes.  B: 16 channel blocks of 1 KiB, piece 16t + r of a block =
+        // codes 32t..32t+31 of channel r.
         const unsigned char* src = pk + (size_t)s * kPkStageBytes;
         unsigned char* dstA = i8 + (size_t)u * kI8StageBytes;
         unsigned char* dstB = dstA + kI8ABytes;
@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
             expand_store(v[i], dstA, piece >> 2, piece & 3);
           } else {
             const int q = piece - BM * 4;
-            expand_store(v[i], dstB, ((q >> 5) << 3) + (q & 7), (q >> 3) & 3);
+            expand_store(v[i], dstB, ((q >> 6) << 4) + (q & 15), (q >> 4) & 3);
           }
         }
         fence_proxy_async_smem();

@@ -13,18 +13,19 @@
 // Codes are packed two per byte exactly like the activation format (byte j of a row = code 2j in
 // bits 0-3, code 2j+1 in bits 4-7, two's complement).  The smallest piece is 16 bytes: 32
 // consecutive codes of one output channel.  Pieces are stored as
-//     [block of 8 output channels][group of 32 codes][channel within the block][16 bytes]
-// so that (a) the codes of 8 channels over any range of K that is a multiple of 32 are one
+//     [block of 16 output channels][group of 32 codes][channel within the block][16 bytes]
+// so that (a) the codes of 16 channels over any range of K that is a multiple of 32 are one
 // contiguous run (the decode kernel streams such runs and cuts K between the CTAs of a cluster),
-// (b) a warp-wide 128-bit load of 512 consecutive bytes gives lane 8t + g the codes 32t..32t+31
-// of channel g of a 128-code block -- the B fragments of four m16n8k32 MMAs after the nibble
-// split -- and (c) 32 consecutive channel blocks at one 128-code block, fetched as 32 bulk
-// copies of 512 bytes, form the 256-row tile the prefill kernel expands for tcgen05.mma.
+// (b) inside a 256-byte group lane 4g + t of a warp finds word t (8 codes) of channels g and g + 8
+// at byte offsets 4 * lane and 128 + 4 * lane -- conflict-free 32-bit loads that become the A
+// fragment of one m16n8k32 MMA after the nibble split -- and (c) 16 consecutive channel blocks at
+// one 128-code block, fetched as 16 bulk copies of 1 KiB, form the 256-row tile the prefill
+// kernel expands for tcgen05.mma.
 // Rows are padded to a multiple of 256 and K' to a multiple of 128 with zero codes.
 // ---------------------------------------------------------------------------------------------
-constexpr int XQ_ROW_BLOCK = 8;
+constexpr int XQ_ROW_BLOCK = 16;
 constexpr int XQ_K_GROUP = 32;                                   // codes per 16-byte piece
-constexpr int XQ_GROUP_BYTES = XQ_ROW_BLOCK * XQ_K_GROUP / 2;    // 128: one group of one block
+constexpr int XQ_GROUP_BYTES = XQ_ROW_BLOCK * XQ_K_GROUP / 2;    // 256: one group of one block
 constexpr int XQ_K_BLOCK = 128;
 constexpr int XQ_ROW_PAD = 256;
 
@@ -40,8 +41,8 @@ struct xq_weights {
 
 // Byte offset of the 32-bit word holding codes 8*kg .. 8*kg+7 of row n (k_groups = K'' / 32).
 __host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_groups) {
-  const int blk = n >> 3, g = n & 7, grp = kg >> 2, word = kg & 3;
-  return ((size_t)blk * k_groups + grp) * XQ_GROUP_BYTES + (size_t)g * 16 + (size_t)word * 4;
+  const int blk = n >> 4, r = n & 15, grp = kg >> 2, word = kg & 3;
+  return ((size_t)blk * k_groups + grp) * XQ_GROUP_BYTES + (size_t)r * 16 + (size_t)word * 4;
 }
 
 // Workspace layout (all offsets multiples of 256 bytes).  The header is what xq_workspace_init
