@@ -1,0 +1,69 @@
+// Device helpers shared by the rotate + quantize kernels: the order-p Paley factor from the
+// quadratic-character table of GF(q), block-wide maximum, transposing matrix loads.
+#pragma once
+
+#include <stdint.h>
+
+namespace xqhad {
+
+// ---------------------------------------------------------------------------------------------
+// Sign of entry (a, a2) of the order-p Paley factor from the quadratic-character table of GF(q).
+// chi2 is indexed by d + q for d in (-q, q): chi2[d + q] = chi(d mod q), chi(0) = 0.
+// Paley-I:  first row +1, first column -1 below it, core chi(i - j) + identity.
+// Paley-II: symmetric S of order q + 1 (zero diagonal, border +1, core chi(i - j)); each entry s
+//           becomes s * [[1, 1], [1, -1]], each diagonal zero becomes [[1, -1], [-1, -1]].
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int paley_sign(int kind, int q, const int8_t* chi2, int a, int a2) {
+  if (kind == 1) {
+    if (a == 0) return 1;
+    if (a2 == 0) return -1;
+    const int d = a - a2;
+    return d == 0 ? 1 : chi2[d + q];
+  }
+  const int i = a >> 1, u = a & 1, j = a2 >> 1, v = a2 & 1;
+  if (i == j) return (u | v) ? -1 : 1;
+  int s = (i == 0 || j == 0) ? 1 : chi2[i - j + q];
+  return (u & v) ? -s : s;
+}
+
+// Fill chi2 (2q + 1 entries) cooperatively; `sq` is q scratch bytes.
+__device__ __forceinline__ void build_chi(int q, int8_t* chi2, int8_t* sq) {
+  for (int i = threadIdx.x; i < q; i += blockDim.x) sq[i] = 0;
+  __syncthreads();
+  for (int i = 1 + threadIdx.x; i <= (q - 1) / 2; i += blockDim.x) sq[(i * i) % q] = 1;
+  __syncthreads();
+  for (int d = threadIdx.x; d < 2 * q + 1; d += blockDim.x) {
+    int r = (d - q) % q;
+    if (r < 0) r += q;
+    chi2[d] = r == 0 ? 0 : (sq[r] ? 1 : -1);
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ float block_max(float v, float* red) {
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float r = lane < nw ? red[lane] : 0.f;
+  for (int o = 16; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, o));
+  __syncthreads();
+  return r;
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_ptr) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_ptr) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+
+__device__ __forceinline__ uint32_t sign_bf16(int s) { return s > 0 ? 0x3F80u : (s < 0 ? 0xBF80u : 0u); }
+
+}  // namespace xqhad

@@ -68,6 +68,11 @@ constexpr int XQ_DECODE_MAX_M = 32;
 // A8opt (optional): byte-per-code copy of the codes in the operand format of the tcgen05 GEMM, [M, Kp].
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl,
                                    uint8_t* Xq, float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st);
+// Throughput form for many rows (several independent row groups per CTA, double-buffered loads).
+bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl);
+cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
+                                  float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st);
+constexpr int XQ_ROTATE_ROWS_MIN_M = 48;  // below this the one-CTA-per-row kernel has the shorter latency
 cudaError_t xq_launch_relayout_to_blocks(const uint8_t* canon, int32_t N, int32_t Kp, uint8_t* blocks,
                                          int32_t Np, int32_t Kpp, cudaStream_t st);
 cudaError_t xq_launch_relayout_from_blocks(const uint8_t* blocks, int32_t Np, int32_t Kpp, uint8_t* canon,

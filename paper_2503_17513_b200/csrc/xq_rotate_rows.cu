@@ -1,0 +1,278 @@
+// Online step of the expanded layer for many rows (paper Sec. 3: X_hat = X H_hat; Sec. 4:
+// per-token 4-bit): the throughput form of the fused pad + Kronecker Hadamard + quantize kernel.
+//
+// One persistent CTA per SM holds H_p^T as a bf16 matrix in shared memory and runs G independent
+// row groups of Wr warps each; a group streams its rows through a double-buffered cp.async stage
+// (the next row lands while the current one is computed) and never meets the other groups: the
+// only synchronisation is a named barrier inside the group (a warp-level one when Wr == 1).
+// With the row viewed as V[a][b] (a < p, b < n = 2^k) the layer needs Y = H_p^T V S_n.  The outer
+// factor goes first, on the raw bf16 inputs -- +-1 times bf16 is exact and the sums accumulate
+// in fp32 -- as m16n8k16 MMAs: A fragments with ldmatrix from the shared H_p^T, B fragments with
+// a transposing ldmatrix from the staged row.  A warp owns MTW tiles of 16 rows a' and all n
+// columns, so the Sylvester butterflies along b stay inside the warp.  In the accumulator layout
+// a thread holds columns b = 8j + 2t + e of its rows: bits 0 and 3.. of b are butterflied in
+// registers; for bits 1-2 (the lane bits t) eight rows at a time pass through a small per-warp
+// shared-memory tile and come back with all eight columns 8j..8j+7 of one row in one thread --
+// the warp shuffle unit would otherwise be the bottleneck -- which is also exactly one packed
+// word of eight codes.  Per-row absmax (five shuffles, then Wr values through shared memory),
+// scale 1/sqrt(K') folded into the quantizer's multiplier, round-to-nearest-even by the
+// magic-number add, nibble packing and coalesced 32-bit stores follow.
+#include <cuda_bf16.h>
+
+#include "xq_internal.h"
+#include "xq_hadamard.cuh"
+#include "xq_ptx.cuh"
+
+using namespace xqhad;
+
+namespace {
+
+constexpr int kMaxWarps = 16;
+
+__device__ __forceinline__ void group_sync(int group, int Wr) {
+  if (Wr == 1) __syncwarp();
+  else xqptx::bar_sync(1 + group, 32 * Wr);
+}
+
+template <int LOG2N, int KS, int MTW>
+__global__ void __launch_bounds__(kMaxWarps * 32, 1)
+    rotate_quant_rows_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx, xq_hadamard_plan_t pl, float gamma,
+                             uint8_t* __restrict__ Xq, float* __restrict__ sx, float* __restrict__ Yopt, uint8_t* __restrict__ A8opt,
+                             int Wr, int G) {
+  constexpr int n = 1 << LOG2N, NT8 = n / 8;
+  constexpr int xpitch = n + 8;        // bf16 elements per staged row (conflict-free ldmatrix)
+  constexpr int hpitch = KS * 16 + 8;  // bf16 elements per row of H_p^T
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int K = pl.K, Kp = pl.Kp, p = pl.p, q = pl.q;
+  const int MT = (p + 15) / 16;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int group = warp / Wr, wg = warp - group * Wr, tg = tid - group * Wr * 32, gthreads = Wr * 32;
+
+  __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(smem_raw);                       // [MT * 16][hpitch]
+  __nv_bfloat16* Xs_all = Hs + MT * 16 * hpitch;                                        // [G][2][KS * 16][xpitch]
+  constexpr int tpitch = n + 8;        // floats per row of the transpose tile
+  float* tr_all = reinterpret_cast<float*>(Xs_all + (size_t)G * 2 * KS * 16 * xpitch);  // [warps][8][tpitch]
+  float* red_all = tr_all + (size_t)G * Wr * 8 * tpitch;                                // [G][Wr] + 32 spare
+  int8_t* chi2 = reinterpret_cast<int8_t*>(red_all + G * Wr + 32);
+  int8_t* sq = chi2 + 2 * q + 1;
+
+  build_chi(q, chi2, sq);
+  xqptx::pdl_launch_dependents();
+  // H_p^T: row a' (output index), column a (input index); zero outside p x p
+  for (int i = tid; i < MT * 16 * KS * 16; i += blockDim.x) {
+    const int a2 = i / (KS * 16), a = i - a2 * (KS * 16);
+    const int s = (a2 < p && a < p) ? paley_sign(pl.paley_kind, q, chi2, a, a2) : 0;
+    Hs[a2 * hpitch + a] = __ushort_as_bfloat16((unsigned short)sign_bf16(s));
+  }
+  // zero the staged rows once: rows past the data and the tail of a partial last row stay zero
+  for (int i = tid; i < G * 2 * KS * 16 * xpitch / 8; i += blockDim.x) reinterpret_cast<uint4*>(Xs_all)[i] = make_uint4(0, 0, 0, 0);
+  xqptx::pdl_wait();
+  __syncthreads();
+  if (group >= G) return;
+
+  __nv_bfloat16* Xs = Xs_all + (size_t)group * 2 * KS * 16 * xpitch;
+  float* tr = tr_all + (size_t)warp * 8 * tpitch;
+  float* red = red_all + group * Wr;
+  constexpr int TPL = NT8 / 4;  // (row, j) tuples of eight columns per lane and pass of eight rows
+  const int chunks = K / 8;  // 16-byte pieces of a row
+  const int stride = gridDim.x * G;
+  auto issue_load = [&](int row, int buf) {
+    const __nv_bfloat16* x = X + (long long)row * ldx;
+    __nv_bfloat16* dst = Xs + (size_t)buf * KS * 16 * xpitch;
+    for (int i = tg; i < chunks; i += gthreads) {
+      const int c = 8 * i, a = c >> LOG2N, b = c & (n - 1);
+      xqptx::cp_async16(dst + a * xpitch + b, x + c);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  int row = blockIdx.x * G + group, buf = 0;
+  if (row < M) issue_load(row, 0);
+  for (; row < M; row += stride, buf ^= 1) {
+    if (row + stride < M) {
+      issue_load(row + stride, buf ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    group_sync(group, Wr);
+    const __nv_bfloat16* xb = Xs + (size_t)buf * KS * 16 * xpitch;
+
+    float acc[MTW][NT8][4];
+#pragma unroll
+    for (int m = 0; m < MTW; ++m)
+#pragma unroll
+      for (int j = 0; j < NT8; ++j) acc[m][j][0] = acc[m][j][1] = acc[m][j][2] = acc[m][j][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      uint32_t bfr[NT8][2];
+      const __nv_bfloat16* base = xb + (16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8) * xpitch + ((lane >> 4) & 1) * 8;
+#pragma unroll
+      for (int jp = 0; jp < NT8 / 2; ++jp) {
+        uint32_t r4[4];
+        ldmatrix_x4_trans(r4, base + 16 * jp);
+        bfr[2 * jp][0] = r4[0];
+        bfr[2 * jp][1] = r4[1];
+        bfr[2 * jp + 1][0] = r4[2];
+        bfr[2 * jp + 1][1] = r4[3];
+      }
+#pragma unroll
+      for (int m = 0; m < MTW; ++m) {
+        const int mt = wg * MTW + m;
+        if (mt < MT) {
+          uint32_t afr[4];
+          ldmatrix_x4(afr, Hs + (16 * mt + (lane & 15)) * hpitch + 16 * ks + (lane >> 4) * 8);
+#pragma unroll
+          for (int j = 0; j < NT8; ++j) xqptx::mma_bf16_16x8x16(acc[m][j], afr, bfr[j][0], bfr[j][1]);
+        }
+      }
+    }
+    // Sylvester butterflies along b = 8 j + 2 t + e: bit 0 (e) and bits 3.. (j) in registers
+#pragma unroll
+    for (int m = 0; m < MTW; ++m) {
+#pragma unroll
+      for (int j = 0; j < NT8; ++j) {
+        const float u0 = acc[m][j][0], u1 = acc[m][j][1], u2 = acc[m][j][2], u3 = acc[m][j][3];
+        acc[m][j][0] = u0 + u1; acc[m][j][1] = u0 - u1; acc[m][j][2] = u2 + u3; acc[m][j][3] = u2 - u3;
+      }
+#pragma unroll
+      for (int s = 1; s < NT8; s <<= 1)
+#pragma unroll
+        for (int j = 0; j < NT8; ++j)
+          if (!(j & s)) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float u = acc[m][j][e], w = acc[m][j | s][e];
+              acc[m][j][e] = u + w;
+              acc[m][j | s][e] = u - w;
+            }
+          }
+    }
+    // bits 1-2 (t): eight rows at a time through the warp's tile; afterwards fin[m][h][k][0..7] are
+    // the columns 8 jj .. 8 jj + 7 of row a' = 16 (wg MTW + m) + 8 h + r, (r, jj) = tuple lane + 32 k
+    float fin[MTW][2][TPL][8];
+    float amax = 0.f;
+#pragma unroll
+    for (int m = 0; m < MTW; ++m)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+#pragma unroll
+        for (int j = 0; j < NT8; ++j) *reinterpret_cast<float2*>(tr + g * tpitch + 8 * j + 2 * t) = make_float2(acc[m][j][2 * h], acc[m][j][2 * h + 1]);
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < TPL; ++k) {
+          const int id = lane + 32 * k, r = id / NT8, jj = id % NT8;
+          const float4 v0 = *reinterpret_cast<const float4*>(tr + r * tpitch + 8 * jj);
+          const float4 v1 = *reinterpret_cast<const float4*>(tr + r * tpitch + 8 * jj + 4);
+          // index i = 2 t + e inside the eight: bit 1 pairs (i, i ^ 2), bit 2 pairs (i, i ^ 4)
+          const float a0 = v0.x + v0.z, a1 = v0.y + v0.w, a2 = v0.x - v0.z, a3 = v0.y - v0.w;
+          const float a4 = v1.x + v1.z, a5 = v1.y + v1.w, a6 = v1.x - v1.z, a7 = v1.y - v1.w;
+          float* f = fin[m][h][k];
+          f[0] = a0 + a4; f[1] = a1 + a5; f[2] = a2 + a6; f[3] = a3 + a7;
+          f[4] = a0 - a4; f[5] = a1 - a5; f[6] = a2 - a6; f[7] = a3 - a7;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(f[i]));
+        }
+        __syncwarp();
+      }
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if (Wr > 1) {
+      if (lane == 0) red[wg] = amax;
+      group_sync(group, Wr);
+      for (int i = 0; i < Wr; ++i) amax = fmaxf(amax, red[i]);
+    }
+    amax *= gamma;  // the maximum of the scaled values: scaling is monotone
+    float s = amax > 0.f ? __fdiv_rn(amax, 7.f) : 1.f;
+    if (!(s > 0.f)) s = 1.f;
+    const float mult = gamma * __frcp_rn(s);
+    if (tg == 0) sx[row] = s;
+    // quantize (round to nearest even through the 1.5 * 2^23 add: the low mantissa bits are the
+    // two's-complement integer; |y / s| <= 7, so no clamp is needed), pack eight codes per word
+    uint32_t* xq_row = reinterpret_cast<uint32_t*>(Xq + (long long)row * (Kp / 2));
+#pragma unroll
+    for (int m = 0; m < MTW; ++m)
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int k = 0; k < TPL; ++k) {
+          const int id = lane + 32 * k, r = id / NT8, jj = id % NT8;
+          const int a2 = 16 * (wg * MTW + m) + 8 * h + r;
+          const float* f = fin[m][h][k];
+          uint32_t w = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) w |= ((uint32_t)__float_as_int(fmaf(f[i], mult, 12582912.f)) & 0xFu) << (4 * i);
+          if (a2 < p) {
+            xq_row[a2 * NT8 + jj] = w;
+            if (A8opt) {
+              uint2 e8;
+              xqptx::split16(w, e8.x, e8.y);
+              *reinterpret_cast<uint2*>(A8opt + (long long)row * Kp + (long long)a2 * n + 8 * jj) = e8;
+            }
+            if (Yopt) {
+              float4* y = reinterpret_cast<float4*>(Yopt + (long long)row * Kp + (long long)a2 * n + 8 * jj);
+              y[0] = make_float4(f[0] * gamma, f[1] * gamma, f[2] * gamma, f[3] * gamma);
+              y[1] = make_float4(f[4] * gamma, f[5] * gamma, f[6] * gamma, f[7] * gamma);
+            }
+          }
+        }
+    // every warp of the group is done with the stage before its reuse two loads from now
+    group_sync(group, Wr);
+  }
+}
+
+template <int LOG2N, int KS, int MTW>
+cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
+                        float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+  constexpr int n = 1 << LOG2N;
+  const int MT = (pl.p + 15) / 16, Wr = (MT + MTW - 1) / MTW;
+  int G = kMaxWarps / Wr;
+  const size_t fixed = (size_t)MT * 16 * (KS * 16 + 8) * 2 + 32 * 4 + (size_t)(3 * pl.q + 1) + 64;
+  const size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 4;
+  while (G > 1 && fixed + G * per_group > 200 * 1024) --G;
+  const size_t smem = fixed + G * per_group;
+  auto kern = rotate_quant_rows_kernel<LOG2N, KS, MTW>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const int want = (M + G - 1) / G;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(want < sms ? want : sms);
+  cfg.blockDim = dim3(32 * Wr * G);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, Wr, G);
+}
+
+template <int LOG2N, int MTW>
+cudaError_t launch_rows_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
+                           float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+  switch (ks) {
+    case 1: return launch_rows<LOG2N, 1, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 2: return launch_rows<LOG2N, 2, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 3: return launch_rows<LOG2N, 3, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    default: return launch_rows<LOG2N, 4, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+  }
+}
+
+}  // namespace
+
+bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
+  const int n = 1 << pl.log2n, rows_a = (pl.K + n - 1) / n, MT = (pl.p + 15) / 16;
+  return pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 7 && pl.K % 8 == 0 && rows_a <= 64 && MT <= 15 && pl.Kp % 32 == 0;
+}
+
+cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
+                                  float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+  const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
+  const int n = 1 << pl.log2n, rows_a = (pl.K + n - 1) / n, ks = (rows_a + 15) / 16;
+  // tiles of 16 output rows per warp: 80 accumulator registers at n = 32, 64 at n = 64 and 128
+  switch (pl.log2n) {
+    case 5: return launch_rows_ks<5, 5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 6: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    default: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+  }
+}

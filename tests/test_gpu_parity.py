@@ -77,6 +77,8 @@ ROTATE_CASES = [
     (5, 100, 136), (3, 200, 240), (4, 130, 144), (7, 70, 80), (2, 64, 64), (3, 40, 48), (3, 50, 56), (2, 250, 280),
     (2, 8, 8), (16, 2048, 2176), (3, 8192, 8704), (3, 4096, 4352), (2, 14336, 15360), (3, 4096, 4608),
     (3, 4096, 5120), (3, 4096, 4096), (33, 2048, 2176),
+    # many rows: the multi-row-group kernel (several rows per CTA, ragged last pass), every n it takes
+    (300, 2048, 2176), (333, 100, 160), (150, 4096, 4352), (100, 8192, 8704), (70, 1000, 1152), (49, 4096, 4608),
 ]
 
 
