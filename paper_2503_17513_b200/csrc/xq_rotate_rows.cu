@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     const float mult = gamma * __frcp_rn(s);
     if (tg == 0) sx[row] = s;
     // quantize (round to nearest even through the 1.5 * 2^23 add: the low mantissa bits are the
-    // two's-complement integer; |y / s| <= 7, so no clamp is needed), pack eight codes per word
+    // integer; |y / s| <= 7, so no clamp is needed), pack eight codes per word
     uint32_t* xq_row = reinterpret_cast<uint32_t*>(Xq + (long long)row * (Kp / 2));
 #pragma unroll
     for (int m = 0; m < MTW; ++m)
@@ -198,9 +198,13 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
           const int id = lane + 32 * k, r = id / NT8, jj = id % NT8;
           const int a2 = 16 * (wg * MTW + m) + 8 * h + r;
           const float* f = fin[m][h][k];
+          // Horner over the raw bit patterns 0x4B400008 + code (the add also biases the code by 8):
+          // the constant parts sum to a fixed word that is removed once, and offset-binary
+          // nibbles become two's complement by flipping their top bits.
           uint32_t w = 0;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) w |= ((uint32_t)__float_as_int(fmaf(f[i], mult, 12582912.f)) & 0xFu) << (4 * i);
+          for (int i = 7; i >= 0; --i) w = w * 16u + (uint32_t)__float_as_int(fmaf(f[i], mult, 12582920.f));
+          w = (w - 0x4B400000u * 0x11111111u) ^ 0x88888888u;
           if (a2 < p) {
             xq_row[a2 * NT8 + jj] = w;
             if (A8opt) {
