@@ -117,10 +117,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   if (tid < p.stages) {
     mbar_init(&full[tid], 1);
     mbar_init(&empty[tid], 1);
+    mbar_fence_init();  // only the initialising threads: a cluster-scope fence in every thread is costly
   }
-  if (tid == 33) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.sx));
-  if (tid == 32) *failed = 0;
-  mbar_fence_init();
+  if (tid == 64) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.sx));
+  if (tid == 65) *failed = 0;
   __syncthreads();
   cluster_arrive_relaxed();  // "this CTA runs": awaited before the first remote store
   pdl_launch_dependents();
@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         const int ng = min(4 * c_hi, L) - 4 * c_lo;
         const unsigned char* wp = ring + (size_t)s * kStageBytes + lane * 4;  // channel ag (and ag + 8 at +128), word at
         const unsigned char* ap = act + (size_t)ag * p.act_pitch + (size_t)c_lo * 128 + (size_t)at * 32;
-#pragma unroll 2
+#pragma unroll 1
         for (int gq = 0; gq < ng; gq += 4, wp += kChunkBytes, ap += 128) {
           const int nv = min(4, ng - gq);  // groups of this chunk that exist
           uint32_t a[4][4];
