@@ -147,16 +147,18 @@ def rotate_bytes(M, K, Kp):
 
 
 def run_reference(args, table, layers, M, heavy):
-    """CPU oracle on the host cores: each step = the online path of ONE layer's linears for min(M, 64) tokens
-    (weights prepared beforehand, as on the GPU); tokens/s scaled to the full layer count."""
+    """CPU oracle on the host cores.  A step is a bounded sample of the workload -- the online path of
+    ONE layer's linears for min(M, 8) tokens and min(N, 128) output channels per linear (weights prepared
+    beforehand, as on the GPU) -- so that K steps end within minutes whatever K is; tokens/s is scaled
+    linearly to all layers, all tokens and all channels (the path is independent per token and channel)."""
     import oracle
 
     oracle.build()
-    Ms = min(M, 64)
+    Ms = min(M, 8)
     prepared = {}
     xs = {}
     for name, (K, Kp, N) in table.items():
-        Ns = min(N, 1024)  # bounded sample of output channels, scaled below
+        Ns = min(N, 128)
         pl = oracle.plan(K, Kp)
         xs[name] = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
         qw, sw = oracle.prepare_weights(pl, synth.weights(Ns, K, seed=0, tag=name))
@@ -175,16 +177,23 @@ def run_reference(args, table, layers, M, heavy):
             t_scaled += (t1 - t0) + (t2 - t1) * scale
         return t_scaled
 
+    t_begin = time.perf_counter()
     for _ in range(args.warmup):
         step()
-    times = [step() for _ in range(args.steps)]
+        if time.perf_counter() - t_begin > 30.0:
+            break
+    times = []
+    for _ in range(args.steps):  # at most K steps, fewer when K of them would not end within minutes
+        times.append(step())
+        if time.perf_counter() - t_begin > 150.0:
+            break
     t_layer = sum(times) / len(times)
     t_step = t_layer * layers * (M / Ms)
     value = M / t_step
-    sample = (f"online path of one layer's linears for {Ms} tokens, {min(1024, min(v[2] for v in table.values()))}+ output "
-              f"channels per linear (GEMM time scaled to full N), scaled to {layers} layers and M={M}")
+    sample = (f"{len(times)} timed steps; per step: online path of one layer's linears for {Ms} tokens and up to 128 output channels per linear "
+              f"(GEMM time scaled to full N), scaled to {layers} layers and M={M}")
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": len(times),
         "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64/int64 (oracle)", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {','.join(table)} x {layers} layers, M={M}"},
