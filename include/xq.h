@@ -145,9 +145,9 @@ xq_status xq_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_w
  * allocation of any kind: it looks up the array, clears the status word and enqueues the same
  * two kernels as xq_expanded_linear on `stream`.
  *
- * Limit: 256 + roundup256(M * Kp / 2) + roundup256(4 * M) bytes must fit in 4 MiB (about 3800
- * tokens at Kp = 2176, 540 at Kp = 15360); larger calls return XQ_ERR_WORKSPACE and launch
- * nothing.
+ * Limit: 256 + roundup256(M * Kp / 2) + roundup256(4 * M) bytes, plus roundup256(M * Kp) when
+ * M > 32, must fit in 4 MiB (about 1280 tokens at Kp = 2176, 180 at Kp = 15360); larger calls
+ * return XQ_ERR_WORKSPACE and launch nothing.
  * First call on each device: it asks the runtime for the array's device address (with that
  * device current) and remembers it; make this first call outside any stream capture.
  * Sharing: all calls on one device use the same array, which keeps the previous call's

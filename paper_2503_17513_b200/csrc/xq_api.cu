@@ -74,6 +74,11 @@ xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w) {
   off += align_up((size_t)M_max * (size_t)w->K * 2, 256);
   L.ostage = off;
   off += align_up((size_t)M_max * (size_t)w->N * 2, 256);
+  L.a8 = 0;
+  if (M_max > XQ_DECODE_MAX_M) {
+    L.a8 = off;
+    off += align_up((size_t)M_max * (size_t)w->Kp, 256);
+  }
   L.total = off;
   return L;
 }
@@ -275,7 +280,7 @@ xq_status xq_w4a4_gemm(const uint8_t* Xq, const float* s_x, int32_t M, const xq_
     return XQ_ERR_INVALID_ARG;
   const xq_ws_layout L = xq_ws_compute(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
-  if (xq_launch_gemm(Xq, s_x, M, w, out, acc_opt, ws, L, (cudaStream_t)stream) != cudaSuccess) {
+  if (xq_launch_gemm(Xq, s_x, M, w, out, acc_opt, ws, L, false, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
@@ -294,8 +299,9 @@ xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_wei
   uint8_t* Xq = base + L.xq;
   float* sx = (float*)(base + L.sx);
   cudaStream_t st = (cudaStream_t)stream;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, nullptr, w->sms, st) != cudaSuccess ||
-      xq_launch_gemm(Xq, sx, M, w, out, nullptr, ws, L, st) != cudaSuccess) {
+  uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + L.a8 : nullptr;
+  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->sms, st) != cudaSuccess ||
+      xq_launch_gemm(Xq, sx, M, w, out, nullptr, ws, L, A8 != nullptr, st) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }

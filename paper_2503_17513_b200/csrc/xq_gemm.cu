@@ -36,15 +36,24 @@ __global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __res
 
 }  // namespace
 
+bool xq_gemm_wants_a8(int32_t M, const xq_weights* w) { return M > XQ_DECODE_MAX_M && xq_prefill_supported(M, w); }
+
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
-                           int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st) {
+                           int32_t* acc_opt, void* ws, const xq_ws_layout& L, bool a8_ready, cudaStream_t st) {
   if (w->Kp % 8 != 0) return cudaErrorInvalidValue;
   int32_t* header = (int32_t*)ws;
   if (M <= XQ_DECODE_MAX_M) {
     const cudaError_t e = xq_launch_gemm_decode(Xq, sx, M, w, out, acc_opt, header, st);
     if (e != cudaErrorNotSupported) return e;
   }
-  if (xq_prefill_supported(M, w)) return xq_launch_gemm_prefill(Xq, sx, M, w, out, acc_opt, header, w->sms, st);
+  if (xq_prefill_supported(M, w) && L.a8 != 0) {
+    uint8_t* A8 = (uint8_t*)ws + L.a8;
+    if (!a8_ready) {
+      const cudaError_t e = xq_launch_expand_tokens(Xq, M, w->Kp, A8, st);
+      if (e != cudaSuccess) return e;
+    }
+    return xq_launch_gemm_prefill(A8, sx, M, w, out, acc_opt, header, w->sms, st);
+  }
   dim3 grid((w->N + 127) / 128, M);
   gemm_general_kernel<<<grid, 128, 0, st>>>((const uint32_t*)Xq, sx, M, w->packed, w->s_w, w->N, w->Kp,
                                             w->Kpp / XQ_K_GROUP, (__nv_bfloat16*)out, acc_opt);

@@ -1,20 +1,28 @@
 // Prefill-shape W4A4 GEMM (many tokens): the quantized product Q(XR) Q(W~) of the paper's Sec. 3
 // as a dense integer contraction on the fifth-generation tensor cores.
 //
-// Tile: 128 tokens x 256 output channels, K in blocks of 128 codes.  A persistent CTA per SM
-// walks its tiles with four kinds of warps:
-//   producer (1 warp)   TMA: the packed activation tile (tensor map over the [M, K'/2] byte
-//                       matrix, out-of-range rows and columns read as zero) and 16 bulk copies
-//                       of 1 KiB of packed weights per K block, into a ring of packed stages;
-//   unpack   (8 warps)  expand packed nibbles to signed bytes (16 x the code: the nibble moved
-//                       to the top of its byte) and write them into the 128-byte-swizzled
-//                       K-major operand stages that tcgen05.mma reads;
-//   mma      (1 warp)   one thread issues tcgen05.mma kind::i8, 128 x 256 x 32 per instruction,
-//                       int32 accumulators in tensor memory (two buffers of 256 columns);
-//   epilogue (4 warps)  tcgen05.ld the finished accumulator, remove the factor 256 exactly,
-//                       multiply by the per-token and per-channel scales, write bf16.
+// Tile: MH x 128 tokens by 256 output channels (MH = 1 or 2), K in blocks of 128 codes.  A
+// persistent CTA per SM walks its tiles with five kinds of warps:
+//   weight producer (1 warp)  16 bulk copies of 1 KiB of packed weights per K block into a ring
+//                             of packed stages;
+//   token producer (1 warp)   TMA: the byte-per-code token tile (tensor map over the [M, K'] byte
+//                             matrix, 128-byte swizzle, out-of-range rows and columns read as
+//                             zero) straight into the operand stage that tcgen05.mma reads;
+//   unpack   (8 warps)        expand the packed weight nibbles to signed bytes (16 x the code: the
+//                             nibble moved to the top of its byte) and write them into the
+//                             128-byte-swizzled K-major operand stage;
+//   mma      (1 warp)         one thread issues tcgen05.mma kind::i8, 128 x 256 x 32 per
+//                             instruction, int32 accumulators in tensor memory;
+//   epilogue (4 MH warps)     tcgen05.ld the finished accumulator, remove the factor 256 exactly,
+//                             multiply by the per-token and per-channel scales, write bf16.
+// What bounds the kernel is shared-memory traffic per MMA cycle: the token operand therefore
+// arrives already expanded (the rotate + quantize kernel, or a small expansion kernel, writes it
+// once to global memory), and with MH = 2 one expanded weight tile feeds two accumulators.
+// MH = 1 double-buffers its 256-column accumulator (the epilogue of a tile overlaps the main loop
+// of the next); MH = 2 uses all 512 columns for one tile and is chosen when there are enough
+// tiles for that to pay.
 // Inside a word of eight codes the even positions come first after expansion (0,2,4,6,1,3,5,7);
-// activations and weights are expanded by the same rule, so the sum over K is unchanged.
+// tokens and weights are expanded by the same rule, so the sum over K is unchanged.
 // All barrier waits are time-bounded: on expiry the CTA records XQ_ERR_TIMEOUT in the workspace
 // status word, every role leaves its loop, and tensor memory is released before exit.
 #include <cuda.h>
@@ -27,18 +35,25 @@ using namespace xqptx;
 
 namespace {
 
-constexpr int BM = 128, BN = 256;
-constexpr int kPkStages = 4, kI8Stages = 2;
-constexpr int kPkABytes = BM * 64, kPkBBytes = BN * 64;     // packed: 8 KiB + 16 KiB
-constexpr int kI8ABytes = BM * 128, kI8BBytes = BN * 128;   // expanded: 16 KiB + 32 KiB
-constexpr int kPkStageBytes = kPkABytes + kPkBBytes;
-constexpr int kI8StageBytes = kI8ABytes + kI8BBytes;
-constexpr int kUnpackWarps = 8, kEpiWarps = 4;
-constexpr int kFirstEpiWarp = 2, kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
-constexpr int kThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;  // 448
+constexpr int BMH = 128, BN = 256;                           // rows of one accumulator, columns
+constexpr int kPkStages = 4;
+constexpr int kPkBBytes = BN * 64;                           // packed weights of a K block: 16 KiB
+constexpr int kI8ABytes = BMH * 128, kI8BBytes = BN * 128;   // expanded: 16 KiB per 128 tokens, 32 KiB
+constexpr int kUnpackWarps = 8;
+constexpr int kFirstEpiWarp = 4;
 constexpr int kTmemCols = 512;
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kI8Stages * kI8StageBytes + (size_t)kPkStages * kPkStageBytes +
-                              kEpiWarps * BN * sizeof(float) + 256 /*barriers, flags*/;
+
+template <int MH>
+struct Cfg {
+  static constexpr int kI8Stages = MH == 1 ? 3 : 2;
+  static constexpr int kI8StageBytes = MH * kI8ABytes + kI8BBytes;
+  static constexpr int kEpiWarps = 4 * MH;
+  static constexpr int kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
+  static constexpr int kThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;
+  static constexpr int kAccBufs = MH == 1 ? 2 : 1;
+  static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kI8Stages * kI8StageBytes + (size_t)kPkStages * kPkBBytes +
+                                       kEpiWarps * BN * sizeof(float) + 256 /*barriers, flags*/;
+};
 
 struct PrefillParams {
   const uint8_t* W;    // block layout
@@ -65,14 +80,17 @@ __device__ __forceinline__ void expand_store(const uint4 v, unsigned char* tile,
   *reinterpret_cast<uint4*>(row + (((2 * j + 1) ^ x) << 4)) = hi;
 }
 
-__global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap mapA, const PrefillParams p) {
+template <int MH>
+__global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap mapA, const PrefillParams p) {
+  using C = Cfg<MH>;
+  constexpr int kI8Stages = C::kI8Stages, kI8StageBytes = C::kI8StageBytes, kAccBufs = C::kAccBufs;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* base = smem_raw + (((raw + 1023u) & ~1023u) - raw);
-  unsigned char* i8 = base;                                         // kI8Stages x [A 16 KiB | B 32 KiB], 1024-aligned
-  unsigned char* pk = i8 + (size_t)kI8Stages * kI8StageBytes;       // kPkStages x [A 8 KiB | B 16 KiB]
-  float* sw_tile = reinterpret_cast<float*>(pk + (size_t)kPkStages * kPkStageBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sw_tile + kEpiWarps * BN);
+  unsigned char* i8 = base;                                        // kI8Stages x [A (MH x 16 KiB) | B 32 KiB], 1024-aligned
+  unsigned char* pk = i8 + (size_t)kI8Stages * kI8StageBytes;      // kPkStages x 16 KiB of packed weights
+  float* sw_tile = reinterpret_cast<float*>(pk + (size_t)kPkStages * kPkBBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sw_tile + C::kEpiWarps * BN);
   uint64_t* pk_full = bars;
   uint64_t* pk_empty = pk_full + kPkStages;
   uint64_t* i8_full = pk_empty + kPkStages;
@@ -92,12 +110,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
       mbar_init(&pk_empty[s], kUnpackWarps);
     }
     for (int s = 0; s < kI8Stages; ++s) {
-      mbar_init(&i8_full[s], kUnpackWarps);
+      mbar_init(&i8_full[s], kUnpackWarps + 1);  // the unpack warps and the token producer's expect_tx
       mbar_init(&i8_empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&acc_full[b], 1);
-      mbar_init(&acc_empty[b], kEpiWarps);
+      mbar_init(&acc_empty[b], C::kEpiWarps);
     }
     mbar_init(drain, 1);
     *failed = 0;
@@ -113,14 +131,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   pdl_launch_dependents();
-  pdl_wait();  // activations and their scales may come from the kernel before this one
+  pdl_wait();  // tokens and their scales may come from the kernel before this one
 
   if (warp == 0) {
-    // ---------------- producer ------------------------------------------------------------------
+    // ---------------- weight producer -----------------------------------------------------------
     uint32_t it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+      const int tn = tile / p.tiles_m;
       // lane l < 16 fetches channel block l of the tile: 16 channels x 128 codes = 1 KiB contiguous
       const unsigned char* wsrc = p.W + ((size_t)(tn * (BN / XQ_ROW_BLOCK) + (lane & 15)) * p.KB) * (4 * XQ_GROUP_BYTES);
       for (int kb = 0; kb < p.KB; ++kb, ++it) {
@@ -129,28 +147,25 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
           ok = mbar_wait_bounded(&pk_empty[s], ((it / kPkStages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
           if (!ok) break;
         }
-        unsigned char* stage = pk + (size_t)s * kPkStageBytes;
-        if (lane == 0) {
-          mbar_expect_tx(&pk_full[s], kPkStageBytes);
-          tma_load_2d(stage, &mapA, kb * 64, tm * BM, &pk_full[s]);
-        }
+        unsigned char* stage = pk + (size_t)s * kPkBBytes;
+        if (lane == 0) mbar_expect_tx(&pk_full[s], kPkBBytes);
         __syncwarp();
-        if (lane < 16) bulk_g2s(stage + kPkABytes + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
+        if (lane < 16) bulk_g2s(stage + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issue -----------------------------------------------------------------
-    constexpr uint32_t idesc = umma_idesc_s8(BM, BN);
+    constexpr uint32_t idesc = umma_idesc_s8(BMH, BN);
     uint32_t it = 0, tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
-      const uint32_t buf = tcount & 1u;
-      if (tcount >= 2u) {
-        ok = mbar_wait_bounded(&acc_empty[buf], ((tcount >> 1) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+      const uint32_t buf = kAccBufs == 2 ? (tcount & 1u) : 0u;
+      const uint32_t use = kAccBufs == 2 ? (tcount >> 1) : tcount;  // earlier uses of this accumulator
+      if (use >= 1u) {
+        ok = mbar_wait_bounded(&acc_empty[buf], (use - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
         if (!ok) break;
       }
       tc_fence_after_sync();
-      const uint32_t d_tmem = tmem_base + buf * BN;
       for (int kb = 0; kb < p.KB; ++kb, ++it) {
         const int u = it % kI8Stages;
         ok = mbar_wait_bounded(&i8_full[u], (it / kI8Stages) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
@@ -158,9 +173,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
         tc_fence_after_sync();
         if (lane == 0) {
           const uint32_t a_addr = smem_u32(i8 + (size_t)u * kI8StageBytes);
-          const uint64_t adesc = umma_desc_k128(a_addr), bdesc = umma_desc_k128(a_addr + kI8ABytes);
+          const uint64_t bdesc = umma_desc_k128(a_addr + MH * kI8ABytes);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma_i8_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          for (int h = 0; h < MH; ++h) {
+            const uint64_t adesc = umma_desc_k128(a_addr + h * kI8ABytes);
+            const uint32_t d_tmem = tmem_base + (kAccBufs == 2 ? buf : (uint32_t)h) * BN;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) umma_i8_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
           umma_commit(&i8_empty[u]);
         }
         __syncwarp();
@@ -172,25 +192,50 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
     if (lane == 0) umma_commit(drain);
     __syncwarp();
     mbar_wait_bounded(drain, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);
-  } else if (warp < kFirstUnpackWarp) {
+  } else if (warp == 2) {
+    // ---------------- token producer ------------------------------------------------------------
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+      const int tm = tile % p.tiles_m;
+      for (int kb = 0; kb < p.KB; ++kb, ++it) {
+        const int u = it % kI8Stages;
+        if (it >= (uint32_t)kI8Stages) {
+          ok = mbar_wait_bounded(&i8_empty[u], ((it / kI8Stages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+          if (!ok) break;
+        }
+        if (lane == 0) {
+          unsigned char* stage = i8 + (size_t)u * kI8StageBytes;
+          mbar_expect_tx(&i8_full[u], MH * kI8ABytes);
+#pragma unroll
+          for (int h = 0; h < MH; ++h) tma_load_2d(stage + h * kI8ABytes, &mapA, kb * 128, (tm * MH + h) * BMH, &i8_full[u]);
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp == 3) {
+    // idle: keeps the epilogue warps on tensor-memory lane quarters warp mod 4
+  } else if (warp < C::kFirstUnpackWarp) {
     // ---------------- epilogue ------------------------------------------------------------------
-    const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    const int q = warp & 3;                        // tensor-memory lane quarter this warp may read
+    const int eh = (warp - kFirstEpiWarp) >> 2;    // which 128-row half of the tile (MH = 2)
     float* sw_mine = sw_tile + (warp - kFirstEpiWarp) * BN;  // a private copy per warp: no cross-warp barrier
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
       const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-      const uint32_t buf = tcount & 1u;
+      const uint32_t buf = kAccBufs == 2 ? (tcount & 1u) : 0u;
+      const uint32_t use = kAccBufs == 2 ? (tcount >> 1) : tcount;
       const int n0 = tn * BN;
       __syncwarp();
       for (int i = lane; i < BN; i += 32) sw_mine[i] = (n0 + i < p.N) ? p.sw[n0 + i] : 0.f;
       __syncwarp();
-      const int m = tm * BM + q * 32 + lane;
+      const int m = (tm * MH + eh) * BMH + q * 32 + lane;
       const float sxm = m < p.M ? p.sx[m] : 0.f;
-      ok = mbar_wait_bounded(&acc_full[buf], (tcount >> 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+      ok = mbar_wait_bounded(&acc_full[buf], use & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (kAccBufs == 2 ? buf : (uint32_t)eh) * BN;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t v[32];
@@ -228,7 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
     }
   } else {
     // ---------------- unpack --------------------------------------------------------------------
-    const int ut = tid - kFirstUnpackWarp * 32;  // 0..255
+    const int ut = tid - C::kFirstUnpackWarp * 32;  // 0..255
     uint32_t it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
@@ -240,24 +285,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
           ok = mbar_wait_bounded(&i8_empty[u], ((it / kI8Stages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
           if (!ok) break;
         }
-        // A: 128 rows of 64 bytes.  B: 16 channel blocks of 1 KiB, piece 16t + r of a block =
-        // codes 32t..32t+31 of channel r.
-        const unsigned char* src = pk + (size_t)s * kPkStageBytes;
-        unsigned char* dstA = i8 + (size_t)u * kI8StageBytes;
-        unsigned char* dstB = dstA + kI8ABytes;
-        constexpr int kPieces = (BM + BN) * 4 / (kUnpackWarps * 32);  // 16-byte pieces per thread: 6
+        // 16 channel blocks of 1 KiB, piece 16t + r of a block = codes 32t..32t+31 of channel r
+        const unsigned char* src = pk + (size_t)s * kPkBBytes;
+        unsigned char* dstB = i8 + (size_t)u * kI8StageBytes + MH * kI8ABytes;
+        constexpr int kPieces = BN * 4 / (kUnpackWarps * 32);  // 16-byte pieces per thread: 4
         uint4 v[kPieces];
 #pragma unroll
         for (int i = 0; i < kPieces; ++i) v[i] = *reinterpret_cast<const uint4*>(src + (size_t)(ut + i * kUnpackWarps * 32) * 16);
 #pragma unroll
         for (int i = 0; i < kPieces; ++i) {
-          const int piece = ut + i * kUnpackWarps * 32;
-          if (piece < BM * 4) {
-            expand_store(v[i], dstA, piece >> 2, piece & 3);
-          } else {
-            const int q = piece - BM * 4;
-            expand_store(v[i], dstB, ((q >> 6) << 4) + (q & 15), (q >> 4) & 3);
-          }
+          const int q = ut + i * kUnpackWarps * 32;
+          expand_store(v[i], dstB, ((q >> 6) << 4) + (q & 15), (q >> 4) & 3);
         }
         fence_proxy_async_smem();
         __syncwarp();
@@ -274,10 +312,28 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_kernel(const __grid_
   if (warp == 0 && *failed) {
     // bounded drain of copies that may still be landing in this CTA's shared memory
     for (int s = 0; s < kPkStages; ++s) mbar_wait(&pk_full[s], 0, 1u << 16), mbar_wait(&pk_full[s], 1, 1u << 16);
+    for (int s = 0; s < kI8Stages; ++s) mbar_wait(&i8_full[s], 0, 1u << 16), mbar_wait(&i8_full[s], 1, 1u << 16);
   }
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Packed tokens -> byte-per-code tokens in the operand order of the GEMM: a 16-byte piece (words
+// w0..w3) becomes {even(w0), odd(w0), even(w1), odd(w1) | even(w2), odd(w2), even(w3), odd(w3)}.
+__global__ void expand_tokens_kernel(const uint4* __restrict__ Xq, long long pieces, uint4* __restrict__ A8) {
+  pdl_launch_dependents();
+  pdl_wait();
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < pieces; i += (long long)gridDim.x * blockDim.x) {
+    const uint4 v = Xq[i];
+    uint4 lo, hi;
+    split16(v.x, lo.x, lo.y);
+    split16(v.y, lo.z, lo.w);
+    split16(v.z, hi.x, hi.y);
+    split16(v.w, hi.z, hi.w);
+    A8[2 * i] = lo;
+    A8[2 * i + 1] = hi;
   }
 }
 
@@ -297,23 +353,59 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+template <int MH>
+cudaError_t launch_mh(const CUtensorMap& mapA, PrefillParams p, int sms, cudaStream_t st) {
+  using C = Cfg<MH>;
+  p.tiles_m = (p.M + MH * BMH - 1) / (MH * BMH);
+  cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel<MH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  const int tiles = p.tiles_m * p.tiles_n;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles < sms ? tiles : sms);
+  cfg.blockDim = dim3(C::kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_prefill_kernel<MH>, mapA, p);
+}
+
 }  // namespace
 
 bool xq_prefill_supported(int32_t M, const xq_weights* w) {
   return M >= 1 && w->Kp % 32 == 0 && w->N % 8 == 0 && w->Np % BN == 0;
 }
 
-cudaError_t xq_launch_gemm_prefill(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, uint8_t* A8, cudaStream_t st) {
+  const long long pieces = (long long)M * (Kp / 32);
+  long long blocks = (pieces + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks);
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, expand_tokens_kernel, (const uint4*)Xq, pieces, (uint4*)A8);
+}
+
+cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, int32_t M, const xq_weights* w, void* out,
                                    int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st) {
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
   CUtensorMap mapA;
-  const cuuint64_t dims[2] = {(cuuint64_t)(w->Kp / 2), (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)(w->Kp / 2)};
-  const cuuint32_t box[2] = {64, (cuuint32_t)BM};
+  const cuuint64_t dims[2] = {(cuuint64_t)w->Kp, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)w->Kp};
+  const cuuint32_t box[2] = {128, (cuuint32_t)BMH};
   const cuuint32_t estr[2] = {1, 1};
-  if (enc(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)Xq, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+  if (enc(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)A8, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
   PrefillParams p;
   p.W = w->packed;
@@ -325,20 +417,11 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* Xq, const float* sx, int32_t M
   p.M = M;
   p.N = w->N;
   p.KB = w->Kpp / XQ_K_BLOCK;
-  p.tiles_m = (M + BM - 1) / BM;
   p.tiles_n = (w->N + BN - 1) / BN;
-  cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-  if (e != cudaSuccess) return e;
-  const int tiles = p.tiles_m * p.tiles_n;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(tiles < sms ? tiles : sms);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = kSmemBytes;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_prefill_kernel, mapA, p);
+  p.tiles_m = 0;
+  // 256-token tiles halve the weight expansion per MMA but leave fewer, coarser tiles: take them
+  // when they still fill the machine at least twice
+  const int tiles2 = ((M + 2 * BMH - 1) / (2 * BMH)) * p.tiles_n;
+  if (tiles2 >= 2 * sms) return launch_mh<2>(mapA, p, sms, st);
+  return launch_mh<1>(mapA, p, sms, st);
 }

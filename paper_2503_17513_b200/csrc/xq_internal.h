@@ -54,6 +54,7 @@ struct xq_ws_layout {
   size_t sx;       // M_max floats
   size_t xstage;   // M_max * K bf16 (host entry point)
   size_t ostage;   // M_max * N bf16 (host entry point)
+  size_t a8;       // M_max * K'' bytes: byte-per-code tokens for the tensor-core GEMM (only when M_max > 32)
   size_t total;
 };
 xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
@@ -82,8 +83,15 @@ cudaError_t xq_launch_unpack_codes(const uint8_t* packed, int64_t count_pairs, i
 // Decode path: returns cudaErrorNotSupported (nothing launched) when the shape does not fit it.
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
                                   int32_t* acc_opt, int32_t* status, cudaStream_t st);
+// Tensor-core path: takes the tokens one code per byte (16 x code, even codes of every word first),
+// as written by the rotate kernels' optional output or by xq_launch_expand_tokens.
 bool xq_prefill_supported(int32_t M, const xq_weights* w);
-cudaError_t xq_launch_gemm_prefill(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, uint8_t* A8, cudaStream_t st);
+cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, int32_t M, const xq_weights* w, void* out,
                                    int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st);
+// True when M tokens against w go down the tensor-core path (so that the caller lets the rotate
+// kernel write the byte-per-code tokens).
+bool xq_gemm_wants_a8(int32_t M, const xq_weights* w);
+// a8_ready: the a8 region of the workspace already holds the byte-per-code tokens.
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
-                           int32_t* acc_opt, void* ws, const xq_ws_layout& L, cudaStream_t st);
+                           int32_t* acc_opt, void* ws, const xq_ws_layout& L, bool a8_ready, cudaStream_t st);

@@ -49,10 +49,11 @@ extern "C" xq_status xq_expanded_linear_static(const void* X, int32_t M, int64_t
   if (!X || !out) return XQ_ERR_INVALID_ARG;
   if (ldx < w->K || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u))
     return XQ_ERR_INVALID_ARG;
-  // [status header | packed codes M x K'/2 | scales M]
+  // [status header | packed codes M x K'/2 | scales M | byte-per-code tokens M x K' when M > 32]
   const size_t off_xq = XQ_WS_HEADER_BYTES;
   const size_t off_sx = off_xq + round256((size_t)M * (size_t)(w->Kp / 2));
-  const size_t need = off_sx + round256(sizeof(float) * (size_t)M);
+  const size_t off_a8 = off_sx + round256(sizeof(float) * (size_t)M);
+  const size_t need = off_a8 + (M > XQ_DECODE_MAX_M ? round256((size_t)M * (size_t)w->Kp) : 0);
   if (need > kStaticScratchBytes) return XQ_ERR_WORKSPACE;
   unsigned char* base = nullptr;
   const xq_status s = scratch_address(&base);
@@ -68,9 +69,11 @@ extern "C" xq_status xq_expanded_linear_static(const void* X, int32_t M, int64_t
   xq_ws_layout L = {};
   L.xq = off_xq;
   L.sx = off_sx;
+  L.a8 = M > XQ_DECODE_MAX_M ? off_a8 : 0;
   L.total = need;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, nullptr, w->sms, st) != cudaSuccess ||
-      xq_launch_gemm(Xq, sx, M, w, out, nullptr, base, L, st) != cudaSuccess) {
+  uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + off_a8 : nullptr;
+  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->sms, st) != cudaSuccess ||
+      xq_launch_gemm(Xq, sx, M, w, out, nullptr, base, L, A8 != nullptr, st) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
