@@ -422,6 +422,6 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, int32_t M
   // 256-token tiles halve the weight expansion per MMA but leave fewer, coarser tiles: take them
   // when they still fill the machine at least twice
   const int tiles2 = ((M + 2 * BMH - 1) / (2 * BMH)) * p.tiles_n;
-  if (tiles2 >= 2 * sms) return launch_mh<2>(mapA, p, sms, st);
+  if (5 * tiles2 >= 3 * sms) return launch_mh<2>(mapA, p, sms, st);
   return launch_mh<1>(mapA, p, sms, st);
 }
