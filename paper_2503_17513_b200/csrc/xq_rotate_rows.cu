@@ -17,6 +17,9 @@
 // word of eight codes.  Per-row absmax (five shuffles, then Wr values through shared memory),
 // scale 1/sqrt(K') folded into the quantizer's multiplier, round-to-nearest-even by the
 // magic-number add, nibble packing and coalesced 32-bit stores follow.
+// Orders with n = 256 run as n = 128 with the top Sylvester bit folded into the outer factor:
+// H_p (x) S_256 = (H_p (x) S_2) (x) S_128, and channel a 256 + b = (2a + b7) 128 + b', so the same
+// code applies with a factor of order 2p whose signs carry one extra (-1)^(b7 b7').
 #include <cuda_bf16.h>
 
 #include "xq_internal.h"
@@ -38,12 +41,12 @@ template <int LOG2N, int KS, int MTW>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     rotate_quant_rows_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx, xq_hadamard_plan_t pl, float gamma,
                              uint8_t* __restrict__ Xq, float* __restrict__ sx, float* __restrict__ Yopt, uint8_t* __restrict__ A8opt,
-                             int Wr, int G) {
+                             int Wr, int G, int fold) {
   constexpr int n = 1 << LOG2N, NT8 = n / 8;
   constexpr int xpitch = n + 8;        // bf16 elements per staged row (conflict-free ldmatrix)
   constexpr int hpitch = KS * 16 + 8;  // bf16 elements per row of H_p^T
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int K = pl.K, Kp = pl.Kp, p = pl.p, q = pl.q;
+  const int K = pl.K, Kp = pl.Kp, p = pl.p << fold, q = pl.q;  // p: order of the (folded) outer factor
   const int MT = (p + 15) / 16;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int group = warp / Wr, wg = warp - group * Wr, tg = tid - group * Wr * 32, gthreads = Wr * 32;
@@ -61,7 +64,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
   // H_p^T: row a' (output index), column a (input index); zero outside p x p
   for (int i = tid; i < MT * 16 * KS * 16; i += blockDim.x) {
     const int a2 = i / (KS * 16), a = i - a2 * (KS * 16);
-    const int s = (a2 < p && a < p) ? paley_sign(pl.paley_kind, q, chi2, a, a2) : 0;
+    int s = (a2 < p && a < p) ? paley_sign(pl.paley_kind, q, chi2, a >> fold, a2 >> fold) : 0;
+    if (fold && (a & a2 & 1)) s = -s;
     Hs[a2 * hpitch + a] = __ushort_as_bfloat16((unsigned short)sign_bf16(s));
   }
   // zero the staged rows once: rows past the data and the tail of a partial last row stay zero
@@ -228,11 +232,12 @@ template <int LOG2N, int KS, int MTW>
 cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
                         float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
   constexpr int n = 1 << LOG2N;
-  const int MT = (pl.p + 15) / 16, Wr = (MT + MTW - 1) / MTW;
+  const int fold = pl.log2n - LOG2N;  // Sylvester bits folded into the outer factor
+  const int MT = ((pl.p << fold) + 15) / 16, Wr = (MT + MTW - 1) / MTW;
   int G = kMaxWarps / Wr;
   const size_t fixed = (size_t)MT * 16 * (KS * 16 + 8) * 2 + 32 * 4 + (size_t)(3 * pl.q + 1) + 64;
   const size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 4;
-  while (G > 1 && fixed + G * per_group > 200 * 1024) --G;
+  while (G > 1 && fixed + G * per_group > 224 * 1024) --G;
   const size_t smem = fixed + G * per_group;
   auto kern = rotate_quant_rows_kernel<LOG2N, KS, MTW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -248,7 +253,7 @@ cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, Wr, G);
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, Wr, G, fold);
 }
 
 template <int LOG2N, int MTW>
@@ -262,21 +267,43 @@ cudaError_t launch_rows_ks(int ks, const void* X, int32_t M, int64_t ldx, const 
   }
 }
 
+// n = 256 folded to 128: up to 112 staged rows
+cudaError_t launch_rows_folded(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
+                               float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+  switch (ks) {
+    case 5: return launch_rows<7, 5, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 6: return launch_rows<7, 6, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 7: return launch_rows<7, 7, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 8: return launch_rows<7, 8, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    default: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+  }
+}
+
 }  // namespace
 
 bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
-  const int n = 1 << pl.log2n, rows_a = (pl.K + n - 1) / n, MT = (pl.p + 15) / 16;
-  return pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 7 && pl.K % 8 == 0 && rows_a <= 64 && MT <= 15 && pl.Kp % 32 == 0;
+  if (pl.p <= 1 || pl.log2n < 5 || pl.log2n > 8 || pl.K % 8 != 0 || pl.Kp % 32 != 0) return false;
+  const int log2n = pl.log2n > 7 ? 7 : pl.log2n, fold = pl.log2n - log2n;
+  const int n = 1 << log2n, rows_a = (pl.K + n - 1) / n, MT = ((pl.p << fold) + 15) / 16;
+  if (rows_a > (fold ? 128 : 64) || MT > 15) return false;
+  if (fold) {  // the CTA must hold at least one row group
+    const int ks = (rows_a + 15) / 16;
+    const size_t need = (size_t)MT * 16 * (ks * 16 + 8) * 2 + (size_t)2 * ks * 16 * (n + 8) * 2 + (size_t)MT * 8 * (n + 8) * 4 + 4096;
+    if (need > 224 * 1024) return false;
+  }
+  return true;
 }
 
 cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
                                   float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
-  const int n = 1 << pl.log2n, rows_a = (pl.K + n - 1) / n, ks = (rows_a + 15) / 16;
+  const int log2n = pl.log2n > 7 ? 7 : pl.log2n;
+  const int n = 1 << log2n, rows_a = (pl.K + n - 1) / n, ks = (rows_a + 15) / 16;
   // tiles of 16 output rows per warp: 80 accumulator registers at n = 32, 64 at n = 64 and 128
   switch (pl.log2n) {
     case 5: return launch_rows_ks<5, 5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
     case 6: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    default: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 7: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    default: return launch_rows_folded(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
   }
 }

@@ -79,6 +79,7 @@ ROTATE_CASES = [
     (3, 4096, 5120), (3, 4096, 4096), (33, 2048, 2176),
     # many rows: the multi-row-group kernel (several rows per CTA, ragged last pass), every n it takes
     (300, 2048, 2176), (333, 100, 160), (150, 4096, 4352), (100, 8192, 8704), (70, 1000, 1152), (49, 4096, 4608),
+    (60, 14336, 15360), (100, 4096, 5120), (80, 5000, 5120),
 ]
 
 
