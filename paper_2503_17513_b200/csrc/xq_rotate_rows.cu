@@ -17,9 +17,10 @@
 // word of eight codes.  Per-row absmax (five shuffles, then Wr values through shared memory),
 // scale 1/sqrt(K') folded into the quantizer's multiplier, round-to-nearest-even by the
 // magic-number add, nibble packing and coalesced 32-bit stores follow.
-// Orders with n = 256 run as n = 128 with the top Sylvester bit folded into the outer factor:
-// H_p (x) S_256 = (H_p (x) S_2) (x) S_128, and channel a 256 + b = (2a + b7) 128 + b', so the same
-// code applies with a factor of order 2p whose signs carry one extra (-1)^(b7 b7').
+// Orders with n = 2^k > 128 run as n = 128 with the top f = k - 7 Sylvester bits folded into the
+// outer factor: H_p (x) S_{2^k} = (H_p (x) S_{2^f}) (x) S_128, and channel a 2^k + b =
+// (a 2^f + b_hi) 128 + b_lo, so the same code applies with a factor of order p 2^f whose signs
+// carry one extra (-1)^popcount(b_hi & b_hi').  A pure Sylvester order (p = 1) is the case H_1 = [1].
 #include <cuda_bf16.h>
 
 #include "xq_internal.h"
@@ -59,13 +60,16 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
   int8_t* chi2 = reinterpret_cast<int8_t*>(red_all + G * Wr + 32);
   int8_t* sq = chi2 + 2 * q + 1;
 
-  build_chi(q, chi2, sq);
+  if (pl.p > 1) build_chi(q, chi2, sq);
   xqptx::pdl_launch_dependents();
   // H_p^T: row a' (output index), column a (input index); zero outside p x p
   for (int i = tid; i < MT * 16 * KS * 16; i += blockDim.x) {
     const int a2 = i / (KS * 16), a = i - a2 * (KS * 16);
-    int s = (a2 < p && a < p) ? paley_sign(pl.paley_kind, q, chi2, a >> fold, a2 >> fold) : 0;
-    if (fold && (a & a2 & 1)) s = -s;
+    int s = 0;
+    if (a2 < p && a < p) {
+      s = pl.p > 1 ? paley_sign(pl.paley_kind, q, chi2, a >> fold, a2 >> fold) : 1;
+      if (__popc(a & a2 & ((1 << fold) - 1)) & 1) s = -s;
+    }
     Hs[a2 * hpitch + a] = __ushort_as_bfloat16((unsigned short)sign_bf16(s));
   }
   // zero the staged rows once: rows past the data and the tail of a partial last row stay zero
@@ -267,7 +271,7 @@ cudaError_t launch_rows_ks(int ks, const void* X, int32_t M, int64_t ldx, const 
   }
 }
 
-// n = 256 folded to 128: up to 112 staged rows
+// n > 128 folded to 128: up to 128 staged rows
 cudaError_t launch_rows_folded(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
                                float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
   switch (ks) {
@@ -282,7 +286,8 @@ cudaError_t launch_rows_folded(int ks, const void* X, int32_t M, int64_t ldx, co
 }  // namespace
 
 bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
-  if (pl.p <= 1 || pl.log2n < 5 || pl.log2n > 8 || pl.K % 8 != 0 || pl.Kp % 32 != 0) return false;
+  if (pl.log2n < 5 || pl.K % 8 != 0 || pl.Kp % 32 != 0) return false;
+  if (pl.p == 1 && pl.log2n < 9) return false;  // small pure Sylvester orders: the general kernel
   const int log2n = pl.log2n > 7 ? 7 : pl.log2n, fold = pl.log2n - log2n;
   const int n = 1 << log2n, rows_a = (pl.K + n - 1) / n, MT = ((pl.p << fold) + 15) / 16;
   if (rows_a > (fold ? 128 : 64) || MT > 15) return false;

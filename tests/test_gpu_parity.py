@@ -80,6 +80,8 @@ ROTATE_CASES = [
     # many rows: the multi-row-group kernel (several rows per CTA, ragged last pass), every n it takes
     (300, 2048, 2176), (333, 100, 160), (150, 4096, 4352), (100, 8192, 8704), (70, 1000, 1152), (49, 4096, 4608),
     (60, 14336, 15360), (100, 4096, 5120), (80, 5000, 5120),
+    # n > 256 and pure Sylvester orders through the folded outer factor
+    (50, 4096, 4096), (50, 8192, 12288), (64, 1000, 1024),
 ]
 
 
