@@ -165,6 +165,13 @@ xq_status xq_expanded_linear_static(const void* X_bf16_dev, int32_t M, int64_t l
  * XQ_ERR_TIMEOUT or XQ_ERR_BOUNDS), or XQ_ERR_CUDA if the stream itself reports an error. */
 xq_status xq_poll_status(const void* ws_dev, void* stream);
 
+/* Self-test of the failure path (no counterpart in the paper): enqueues a one-warp kernel that
+ * waits, with the same time-bounded wait every pipelined kernel uses, on a barrier that nothing
+ * ever signals.  After about one second the wait gives up, the kernel records XQ_ERR_TIMEOUT in
+ * the workspace status word and returns normally; xq_poll_status then reports XQ_ERR_TIMEOUT and
+ * the CUDA context stays usable.  xq_workspace_init clears the status again. */
+xq_status xq_selftest_wait_timeout(void* ws_dev, size_t ws_bytes, void* stream);
+
 const char* xq_status_string(xq_status s);
 
 #ifdef __cplusplus

@@ -336,6 +336,15 @@ xq_status xq_expanded_linear_host(const void* X_host, int32_t M, const xq_weight
   return XQ_OK;
 }
 
+xq_status xq_selftest_wait_timeout(void* ws, size_t ws_bytes, void* stream) {
+  if (!ws || ws_bytes < XQ_WS_HEADER_BYTES || !aligned16(ws)) return XQ_ERR_WORKSPACE;
+  if (xq_launch_selftest_wait_timeout((int32_t*)ws, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
 xq_status xq_poll_status(const void* ws, void* stream) {
   if (!ws) return XQ_ERR_WORKSPACE;
   int32_t word = 0;

@@ -34,7 +34,26 @@ __global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __res
   out[(long long)m * N + n] = __float2bfloat16_rn((float)acc * sx[m] * sw[n]);
 }
 
+// One warp waits on a barrier that nobody arrives at: exercises the bounded wait and the status
+// word without any fault, trap or endless loop.
+__global__ void selftest_wait_timeout_kernel(int32_t* status) {
+  __shared__ uint64_t bar;
+  __shared__ int failed;
+  if (threadIdx.x == 0) {
+    xqptx::mbar_init(&bar, 1);
+    failed = 0;
+    xqptx::mbar_fence_init();
+  }
+  __syncwarp();
+  xqptx::mbar_wait_bounded(&bar, 0, &failed, status, (int)XQ_ERR_TIMEOUT);
+}
+
 }  // namespace
+
+cudaError_t xq_launch_selftest_wait_timeout(int32_t* status, cudaStream_t st) {
+  selftest_wait_timeout_kernel<<<1, 32, 0, st>>>(status);
+  return cudaGetLastError();
+}
 
 bool xq_gemm_wants_a8(int32_t M, const xq_weights* w) { return M > XQ_DECODE_MAX_M && xq_prefill_supported(M, w); }
 

@@ -91,6 +91,7 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, int32_t M
                                    int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st);
 // True when M tokens against w go down the tensor-core path (so that the caller lets the rotate
 // kernel write the byte-per-code tokens).
+cudaError_t xq_launch_selftest_wait_timeout(int32_t* status, cudaStream_t st);
 bool xq_gemm_wants_a8(int32_t M, const xq_weights* w);
 // a8_ready: the a8 region of the workspace already holds the byte-per-code tokens.
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,

@@ -37,6 +37,7 @@ EXPORTS = [
     "xq_status_string", "xq_hadamard_plan", "xq_prepare_weights", "xq_weights_import", "xq_weights_export",
     "xq_weights_info", "xq_weights_free", "xq_workspace_bytes", "xq_workspace_init", "xq_rotate_quant",
     "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status", "xq_expanded_linear_static",
+    "xq_selftest_wait_timeout",
 ]
 
 
@@ -68,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
+        L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
         for name in EXPORTS:
             if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes"):
                 getattr(L, name).restype = ctypes.c_int
@@ -204,6 +206,11 @@ def xq_expanded_linear_static(X, w: Weights, out, M=None, ldx=None, stream=None)
     ldx = X.stride(0) if ldx is None else ldx
     _check(lib().xq_expanded_linear_static(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _stream(stream)),
            "xq_expanded_linear_static")
+
+
+def xq_selftest_wait_timeout(ws, stream=None) -> None:
+    """Enqueue the self-test kernel whose bounded wait runs out after about a second."""
+    _check(lib().xq_selftest_wait_timeout(_dp(ws), ws.numel() * ws.element_size(), _stream(stream)), "xq_selftest_wait_timeout")
 
 
 def xq_poll_status(ws, stream=None) -> int:

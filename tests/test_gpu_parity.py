@@ -248,3 +248,62 @@ def test_argument_errors_on_device(xq):
     xq.xq_w4a4_gemm(Xq, sx, 0, w, out, ws)
     xq.xq_expanded_linear(X, w, out, ws, M=0)
     assert xq.xq_poll_status(ws) == xq.OK
+
+
+def test_bounded_wait_times_out_cleanly(xq):
+    """A wait on a barrier nobody signals gives up after about a second, records XQ_ERR_TIMEOUT in
+    the workspace status word and leaves the context usable; re-initialising clears the status."""
+    K, Kp, N, M = 64, 64, 32, 4
+    w = xq.xq_weights_import(synth.int4_codes(N, Kp), synth.scales(N), K)
+    ws = xq.new_workspace(M, w)
+    assert xq.xq_poll_status(ws) == xq.OK
+    xq.xq_selftest_wait_timeout(ws)
+    assert xq.xq_poll_status(ws) == xq.ERR_TIMEOUT
+    assert xq.xq_poll_status(ws) == xq.ERR_TIMEOUT  # sticky
+    xq.xq_workspace_init(ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    # the context still works
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    xq.xq_w4a4_gemm(torch.zeros((M, Kp // 2), dtype=torch.uint8, device="cuda"), torch.ones(M, device="cuda"), M, w, out, ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    assert not out.any()
+
+
+# Full sizes of the benchmark workloads, in the launch configuration bench.py times (xq_expanded_linear,
+# all N, all M): the oracle computes every output of a seeded sample of token rows.
+FULL_CASES = [
+    # (tag, M, N, K, Kp, heavy, sampled rows)
+    ("1b-qkv-m32", 32, 3072, 2048, 2176, False, 32), ("1b-gate-m8", 8, 8192, 2048, 2176, False, 8),
+    ("1b-down-m32", 32, 2048, 8192, 8704, False, 8), ("1b-o-m1", 1, 2048, 2048, 2176, False, 1),
+    ("1b-up-m2048", 2048, 8192, 2048, 2176, True, 12), ("1b-down-m2048", 2048, 2048, 8192, 8704, True, 6),
+    ("8b-qkv-m16", 16, 6144, 4096, 4352, False, 6), ("8b-down-m16", 16, 4096, 14336, 15360, False, 3),
+    ("8b-gate-m4096", 4096, 14336, 4096, 4352, True, 4), ("sweep-kp5120-m8192", 8192, 4096, 4096, 5120, True, 6),
+    ("sweep-kp4096-m1", 1, 4096, 4096, 4096, False, 1),
+]
+
+
+@pytest.mark.parametrize("tag,M,N,K,Kp,heavy,nsample", FULL_CASES, ids=[c[0] for c in FULL_CASES])
+def test_full_size_sampled_rows(xq, oracle, tag, M, N, K, Kp, heavy, nsample):
+    x = synth.activations(M, K, seed=0, tag=tag, heavy_tail=heavy)
+    wb = synth.weights(N, K, seed=0, tag=tag)
+    w = xq.xq_prepare_weights(wb, Kp)
+    ws = xq.new_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    xq.xq_expanded_linear(dev(x), w, out, ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    rows = np.sort(np.random.default_rng(11).choice(M, size=min(nsample, M), replace=False))
+    if M > 1:
+        rows[-1] = M - 1  # the last (possibly ragged-tile) row is always checked
+    pl = oracle.plan(K, Kp)
+    qw, s_w = oracle.prepare_weights(pl, wb)
+    _, qx, s_x = oracle.rotate_quant(pl, x[rows])
+    want_bits = oracle.epilogue(oracle.gemm_i64(qx, qw), s_x, s_w)
+    got = synth.bf16_bits_to_f32(host_u16(out[torch.from_numpy(rows).cuda()]))
+    want = synth.bf16_bits_to_f32(want_bits)
+    for i in range(len(rows)):
+        assert rel_l2(got[i], want[i]) <= E2E_REL_L2, (tag, int(rows[i]))
+    # weights as prepared on the GPU: the same +-1 / 0.01 % bound as the activations
+    codes, s_back = xq.xq_weights_export(w)
+    diff = codes.astype(np.int32) - qw.astype(np.int32)
+    assert np.abs(diff).max() <= 1 and np.count_nonzero(diff) / diff.size <= CODE_MISMATCH_FRAC
+    assert np.allclose(s_back, s_w, rtol=2e-6)
