@@ -20,6 +20,32 @@ bool prime(int v) {
   return true;
 }
 
+// Quadratic character of GF(q), q prime: 0 for 0, +1 for non-zero squares, -1 otherwise.
+int host_chi(int a, int q) {
+  a %= q;
+  if (a < 0) a += q;
+  if (a == 0) return 0;
+  for (int i = 1; i <= (q - 1) / 2; ++i)
+    if ((i * i) % q == a) return 1;
+  return -1;
+}
+
+// Entry (a, a2) of the order-p Paley factor (the construction the device kernels use: Paley-I has a
+// first row of +1, a first column of -1 below it and the core chi(i - j) + identity; Paley-II
+// expands the symmetric conference matrix of order q + 1 into 2 x 2 blocks).
+int host_paley_sign(const xq_hadamard_plan_t& pl, int a, int a2) {
+  const int q = pl.q;
+  if (pl.paley_kind == 1) {
+    if (a == 0) return 1;
+    if (a2 == 0) return -1;
+    return a == a2 ? 1 : host_chi(a - a2, q);
+  }
+  const int i = a >> 1, u = a & 1, j = a2 >> 1, v = a2 & 1;
+  if (i == j) return (u | v) ? -1 : 1;
+  const int s = (i == 0 || j == 0) ? 1 : host_chi(i - j, q);
+  return (u & v) ? -s : s;
+}
+
 struct DevBuf {  // scoped device allocation for the offline calls
   void* p = nullptr;
   cudaError_t alloc(size_t bytes) { return cudaMalloc(&p, bytes ? bytes : 1); }
@@ -43,6 +69,7 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
   w->plan = pl;
   w->packed = nullptr;
   w->s_w = nullptr;
+  w->hp_signs = nullptr;
   if (cudaGetDevice(&w->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&w->sms, cudaDevAttrMultiProcessorCount, w->device) != cudaSuccess) {
     delete w;
@@ -54,6 +81,26 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
     cudaGetLastError();
     xq_weights_free(w);
     return XQ_ERR_ALLOC;
+  }
+  if (pl.p > 1) {
+    // bf16 image of H_p^T (row a', column a) for the rotate kernel: a constant of the plan
+    const int P16 = (pl.p + 15) / 16 * 16, pitch = P16 + 8;
+    uint16_t* img = (uint16_t*)calloc((size_t)P16 * pitch, sizeof(uint16_t));
+    if (!img) {
+      xq_weights_free(w);
+      return XQ_ERR_ALLOC;
+    }
+    for (int a2 = 0; a2 < pl.p; ++a2)
+      for (int a = 0; a < pl.p; ++a) img[(size_t)a2 * pitch + a] = host_paley_sign(pl, a, a2) > 0 ? 0x3F80 : 0xBF80;
+    const size_t img_bytes = (size_t)P16 * pitch * sizeof(uint16_t);
+    const bool ok = cudaMalloc((void**)&w->hp_signs, img_bytes) == cudaSuccess &&
+                    cudaMemcpy(w->hp_signs, img, img_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+    free(img);
+    if (!ok) {
+      cudaGetLastError();
+      xq_weights_free(w);
+      return XQ_ERR_ALLOC;
+    }
   }
   *out = w;
   return XQ_OK;
@@ -132,6 +179,7 @@ void xq_weights_free(xq_weights* w) {
   if (!w) return;
   if (w->packed) cudaFree(w->packed);
   if (w->s_w) cudaFree(w->s_w);
+  if (w->hp_signs) cudaFree(w->hp_signs);
   delete w;
 }
 
@@ -164,7 +212,7 @@ xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t K
                                     cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(w->s_w, 0, sizeof(float) * (size_t)w->Np, st);
   if (e == cudaSuccess)
-    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, nullptr, w->sms, st);
+    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, nullptr, w->hp_signs, w->sms, st);
   if (e == cudaSuccess)
     e = xq_launch_relayout_to_blocks((const uint8_t*)dCanon.p, N, Kp, w->packed, w->Np, w->Kpp, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -263,7 +311,7 @@ xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadama
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
-  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, nullptr, sms, (cudaStream_t)stream) != cudaSuccess) {
+  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, nullptr, nullptr, sms, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
@@ -300,7 +348,7 @@ xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_wei
   float* sx = (float*)(base + L.sx);
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + L.a8 : nullptr;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->sms, st) != cudaSuccess ||
+  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->hp_signs, w->sms, st) != cudaSuccess ||
       xq_launch_gemm(Xq, sx, M, w, out, nullptr, ws, L, A8 != nullptr, st) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;

@@ -35,6 +35,7 @@ struct xq_weights {
   xq_hadamard_plan_t plan;
   uint8_t* packed;     // device, Np * Kpp / 2 bytes, block layout above
   float* s_w;          // device, Np floats (padding rows hold 0)
+  uint16_t* hp_signs;  // device, bf16 image of H_p^T for the rotate kernel ([P16][P16 + 8]); NULL when p == 1
   int device;
   int sms;             // multiprocessors of that device
 };
@@ -67,8 +68,11 @@ constexpr int XQ_DECODE_MAX_M = 32;
 
 // Launchers (each returns the CUDA error of its launch).
 // A8opt (optional): byte-per-code copy of the codes in the operand format of the tcgen05 GEMM, [M, Kp].
+// Hsigns (optional): device image of H_p^T as bf16, [P16][P16 + 8] with P16 = p rounded up to 16
+// (xq_weights::hp_signs); without it the kernel derives the signs itself.
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl,
-                                   uint8_t* Xq, float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st);
+                                   uint8_t* Xq, float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms,
+                                   cudaStream_t st);
 // Throughput form for many rows (several independent row groups per CTA, double-buffered loads).
 bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl);
 cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,

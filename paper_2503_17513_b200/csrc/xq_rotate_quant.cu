@@ -110,7 +110,7 @@ template <int LOG2NB, int KS>
 __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx,
                                                               xq_hadamard_plan_t pl, float gamma, uint8_t* __restrict__ Xq,
                                                               float* __restrict__ sx, float* __restrict__ Yopt,
-                                                              uint8_t* __restrict__ A8opt) {
+                                                              uint8_t* __restrict__ A8opt, const __nv_bfloat16* __restrict__ Hsigns) {
   constexpr int NB = 1 << LOG2NB;  // columns per warp
   constexpr int NT8 = NB / 8;      // n-tiles per warp
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -126,12 +126,28 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
   float* red = reinterpret_cast<float*>(outp + Kp / 8);               // 32 floats
   int8_t* chi2 = reinterpret_cast<int8_t*>(red + 32);
   int8_t* sq = chi2 + 2 * q + 1;
-  float* exch = reinterpret_cast<float*>(smem_raw + (((size_t)(sq + q - reinterpret_cast<int8_t*>(smem_raw)) + 15) & ~(size_t)15));
+  // shared image of H_p^T (only when the caller has one ready in global memory), then the exchange buffer
+  const int P16 = (p + 15) / 16 * 16, hpitch = P16 + 8;
+  __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(smem_raw + (((size_t)(sq + q - reinterpret_cast<int8_t*>(smem_raw)) + 15) & ~(size_t)15));
+  float* exch = reinterpret_cast<float*>(Hs + (Hsigns ? P16 * hpitch : 0));
 
-  build_chi(q, chi2, sq);
   xqptx::pdl_launch_dependents();
   // A = H_p^T, rows a' = 16 mt + {g, g+8}, k = a = 16 ks + {2t, 2t+1, 2t+8, 2t+9}
   uint32_t afrag[KS][4];
+  if (Hsigns) {
+    // the sign matrix was prepared with the weights (it is a constant of the plan): fetch the
+    // image and read the fragments with ldmatrix -- a few hundred nanoseconds instead of the
+    // table build and 8 KS sign evaluations per thread below
+    for (int i = tid; i < P16 * hpitch / 8; i += nthreads) xqptx::cp_async16(Hs + 8 * i, Hsigns + 8 * i);
+    xqptx::cp_async_wait_all();
+    __syncthreads();
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      if (16 * ks < P16) ldmatrix_x4(afrag[ks], Hs + (16 * mt + (lane & 15)) * hpitch + 16 * ks + (lane >> 4) * 8);
+      else afrag[ks][0] = afrag[ks][1] = afrag[ks][2] = afrag[ks][3] = 0u;
+    }
+  } else {
+  build_chi(q, chi2, sq);
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks) {
 #pragma unroll
@@ -145,6 +161,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
       }
       afrag[ks][r] = lo | (hi << 16);
     }
+  }
   }
   // zero the staged rows once: rows past the data and the tail of a partial last row stay zero
   for (int i = tid; i < KS * 16 * pitch / 8; i += nthreads) reinterpret_cast<uint4*>(Xs)[i] = make_uint4(0, 0, 0, 0);
@@ -286,9 +303,10 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
 
 template <int LOG2NB, int KS>
 cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
-                      float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+                      float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms, cudaStream_t st) {
   const int n = 1 << pl.log2n, NB = 1 << LOG2NB, NC = n / NB, MT = (pl.p + 15) / 16;
   size_t smem = (size_t)KS * 16 * (n + 8) * 2 + (size_t)pl.Kp / 2 + 128 + (size_t)(3 * pl.q + 1) + 32;
+  if (Hsigns) smem += (size_t)MT * 16 * (MT * 16 + 8) * 2;
   if (NC == 2) smem += (size_t)MT * 16 * n * 4;
   auto kern = rotate_quant_tc_kernel<LOG2NB, KS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -305,17 +323,18 @@ cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_p
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt);
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt,
+                            (const __nv_bfloat16*)Hsigns);
 }
 
 template <int LOG2NB>
 cudaError_t launch_tc_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                         float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+                         float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms, cudaStream_t st) {
   switch (ks) {
-    case 1: return launch_tc<LOG2NB, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 2: return launch_tc<LOG2NB, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 3: return launch_tc<LOG2NB, 3>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    default: return launch_tc<LOG2NB, 4>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 1: return launch_tc<LOG2NB, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
+    case 2: return launch_tc<LOG2NB, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
+    case 3: return launch_tc<LOG2NB, 3>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
+    default: return launch_tc<LOG2NB, 4>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
   }
 }
 
@@ -374,7 +393,7 @@ inline int grid_for(long long work, int threads) {
 }  // namespace
 
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq,
-                                   float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+                                   float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms, cudaStream_t st) {
   // many rows, or an order that only the multi-row-group kernel and the general kernel take
   if ((M >= XQ_ROTATE_ROWS_MIN_M || pl.log2n > 8 || pl.p == 1) && xq_rotate_rows_supported(pl))
     return xq_launch_rotate_rows(X, M, ldx, pl, Xq, sx, Yopt, A8opt, sms, st);
@@ -387,9 +406,9 @@ cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const 
   if (tc) {
     const int ks = (rows_a + 15) / 16;
     switch (pl.log2n) {
-      case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-      case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-      default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+      case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
+      case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
+      default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
     }
   }
   const size_t smem = sizeof(float) * (2 * (size_t)pl.Kp + 32) + (size_t)(3 * pl.q + 1) + 16;
