@@ -312,11 +312,23 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   }
 
   // ---------------- meet the other K slices and finish ------------------------------------------
+  // this CTA finishes blocks j = rank, rank + C, ...: one thread per (block, token, half of the channels);
+  // the scales of a thread's first output are fetched while the cluster barrier completes
+  const int mine = (n_blk - rank + C - 1) / C;
   cluster_arrive_release();
+  float e_sx = 0.f;
+  float4 e_s0 = make_float4(0.f, 0.f, 0.f, 0.f), e_s1 = e_s0;
+  if (warp < kConsumerWarps && tid < mine * p.M * 2) {
+    const int h = tid & 1, bm = tid >> 1, jj = bm / p.M, m = bm - jj * p.M;
+    const int n0 = (b0 + rank + jj * C) * 16 + 8 * h;
+    e_sx = p.sx[m];
+    if (n0 + 8 <= p.N && (p.N & 7) == 0) {
+      e_s0 = *reinterpret_cast<const float4*>(p.sw + n0);
+      e_s1 = *reinterpret_cast<const float4*>(p.sw + n0 + 4);
+    }
+  }
   cluster_wait_acquire();
   if (warp < kConsumerWarps && !*failed) {
-    // this CTA finishes blocks j = rank, rank + C, ...: one thread per (block, token, half of the channels)
-    const int mine = (n_blk - rank + C - 1) / C;
     for (int idx = tid; idx < mine * p.M * 2; idx += kConsumerThreads) {
       const int h = idx & 1, bm = idx >> 1;
       const int jj = bm / p.M, m = bm - jj * p.M;
@@ -332,10 +344,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] >>= 8;  // every product carries 16 x 16
       const int n0 = (b0 + j) * 16 + 8 * h;
-      const float sxm = p.sx[m];
+      const bool pre = idx == tid;  // scales already in registers
+      const float sxm = pre ? e_sx : p.sx[m];
       const size_t o = (size_t)m * p.N + n0;
       if (n0 + 8 <= p.N && (p.N & 7) == 0) {
-        const float4 s0 = *reinterpret_cast<const float4*>(p.sw + n0), s1 = *reinterpret_cast<const float4*>(p.sw + n0 + 4);
+        const float4 s0 = pre ? e_s0 : *reinterpret_cast<const float4*>(p.sw + n0);
+        const float4 s1 = pre ? e_s1 : *reinterpret_cast<const float4*>(p.sw + n0 + 4);
         const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
         uint32_t hw[4];
 #pragma unroll
