@@ -41,6 +41,9 @@ WORKLOADS = {
 }
 METRIC = "expanded W4A4 linear tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture summarised in
+# profiles/gemm_decode_1b_decode_m32.txt (mean over the five linears of a layer); other workloads: not captured per launch.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {("1b-decode", 32): 6.57e6}
 
 
 def measured_peaks():
@@ -333,8 +336,10 @@ def main():
         else:
             dom, dbytes, dt = "xq_rotate_quant (rotate_quant_tc_kernel)", rbytes, t_rot
         achieved = dbytes / dt / 1e9
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.workload, M)) if dom.startswith("xq_w4a4_gemm") else None
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                    "peak_source": peak_kind, "traffic": None, "per_kernel": per_kernel}
+                    "peak_source": peak_kind, "traffic": traffic, "traffic_unit": "bytes per launch (ncu)",
+                    "algorithmic_bytes_per_launch": dbytes / (layers * len(names)), "per_kernel": per_kernel}
 
     # ---- end to end through the host-buffer entry point -----------------------------------------
     Xh = {n: torch.from_numpy(xs_h[n].view(np.int16)).pin_memory() for n in names}
