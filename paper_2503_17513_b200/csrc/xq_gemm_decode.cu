@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int MT = 8 * NT;  // padded token count
-  const int rank = (int)cluster_ctarank();
+  const int rank = C == 1 ? 0 : (int)cluster_ctarank();
   const int cid = blockIdx.x / C, n_clusters = gridDim.x / C;
 
   unsigned char* ring = smem;
@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   if (tid == 64) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.sx));
   if (tid == 65) *failed = 0;
   __syncthreads();
-  cluster_arrive_relaxed();  // "this CTA runs": awaited before the first remote store
+  if (C > 1) cluster_arrive_relaxed();  // "this CTA runs": awaited before the first remote store
   pdl_launch_dependents();
 
   if (warp == kConsumerWarps) {
@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       }
     }
     __syncwarp();
-    cluster_wait_acquire();
+    if (C > 1) cluster_wait_acquire();
   } else {
     // ---------------- consumers ----------------------------------------------------------------
     // the epilogue's channel scales: bring them into L2 now, they are constants
@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
     // c * 128 + t * 32 + i * 8.
     {
       const int total = p.M * L;
-      constexpr int kBatch = 4;
+      constexpr int kBatch = 6;
       for (int base = tid; base < total; base += kBatch * kConsumerThreads) {
         uint4 v[kBatch];
 #pragma unroll
@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       }
     }
     bar_sync(1, kConsumerThreads);
-    cluster_wait_acquire();  // every CTA of the cluster has started: remote stores are legal
+    if (C > 1) cluster_wait_acquire();  // every CTA of the cluster has started: remote stores are legal
 
     const int ag = lane >> 2, at = lane & 3;  // MMA fragment coordinates: channel row / token column, word
     bool ok = true;
@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   // this CTA finishes blocks j = rank, rank + C, ...: one thread per (block, token, half of the channels);
   // the scales of a thread's first output are fetched while the cluster barrier completes
   const int mine = (n_blk - rank + C - 1) / C;
-  cluster_arrive_release();
+  if (C > 1) cluster_arrive_release();
   float e_sx = 0.f;
   float4 e_s0 = make_float4(0.f, 0.f, 0.f, 0.f), e_s1 = e_s0;
   if (warp < kConsumerWarps && tid < mine * p.M * 2) {
@@ -327,7 +327,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       e_s1 = *reinterpret_cast<const float4*>(p.sw + n0 + 4);
     }
   }
-  cluster_wait_acquire();
+  if (C > 1) cluster_wait_acquire();
+  else __syncthreads();
   if (warp < kConsumerWarps && !*failed) {
     for (int idx = tid; idx < mine * p.M * 2; idx += kConsumerThreads) {
       const int h = idx & 1, bm = idx >> 1;
@@ -418,6 +419,11 @@ cudaError_t launch_variant(const DecodeParams& p, int grid, size_t smem, cudaStr
 }
 
 cudaError_t dispatch(int nt, int C, const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
+  if (C == 1) {
+    if (nt == 1) return launch_variant<1, 1>(p, grid, smem, st, max_clusters);
+    if (nt == 2) return launch_variant<2, 1>(p, grid, smem, st, max_clusters);
+    return launch_variant<4, 1>(p, grid, smem, st, max_clusters);
+  }
   if (C == 2) {
     if (nt == 1) return launch_variant<1, 2>(p, grid, smem, st, max_clusters);
     if (nt == 2) return launch_variant<2, 2>(p, grid, smem, st, max_clusters);
@@ -449,7 +455,11 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
   d.nt = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
   const int MT = 8 * d.nt, groups = w->Kp / XQ_K_GROUP, n_blocks = (w->N + 15) / 16;
   const size_t cap = 227 * 1024;
-  for (int C = 2; C <= 4; C *= 2) {
+  // Small layers are latency-bound: when a CTA would stream less than 64 KiB anyway, skip the K cut
+  // between CTAs (no cluster barrier, no remote stores) if the whole token slice fits.
+  const size_t weight_bytes = (size_t)n_blocks * 16 * (w->Kp / 2);
+  const int c_first = (weight_bytes / (size_t)w->sms < 64 * 1024 && M * groups <= 1200) ? 1 : 2;  // and few tokens to expand
+  for (int C = c_first; C <= 4; C *= 2) {
     if (groups < 4 * C) break;
     const int Lmax = (groups + C - 1) / C, Lmin = groups / C;
     const int chunks = (Lmax + 3) / 4, chunks_min = (Lmin + 3) / 4;
