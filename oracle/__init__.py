@@ -16,6 +16,11 @@ from .xq_oracle import (  # noqa: F401
     rotate_dense,
     rotate_factored,
     quantize,
+    quantize_asym,
+    gemm_u_i64,
+    epilogue_asym,
+    rotate_quant_asym,
+    expanded_linear_asym,
     pack_int4,
     unpack_int4,
     gemm_i64,

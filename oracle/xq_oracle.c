@@ -15,7 +15,9 @@
  * case against a library Walsh-Hadamard matrix, truncated-column norms sqrt(K/Kp) (Remark 2),
  * energy and rank preservation (Remarks 1-2), the rotation invariance X W = X_hat W_hat
  * (Sec. 3), quantizer bounds and ties, brute-force / closed-form integer products, bf16
- * rounding against a library conversion.
+ * rounding against a library conversion; for the asymmetric activation quantizer: code range and
+ * end points, |y - s (u - z)| <= s / 2, exactness on an integer grid, and the identity
+ * s_x s_w (acc - z wsum) = sum_c [s_x (u - z)] [s_w qw] against a floating-point product.
  * Parity unpinned: xqo_ref_product's use as a quality axis (the paper prints no error figure
  * for round-to-nearest weights on synthetic data); the function itself is a plain product.
  */
@@ -261,6 +263,71 @@ void xqo_quantize(const double *y, int64_t rows, int64_t cols, int8_t *codes, fl
       codes[r * cols + c] = (int8_t)q;
     }
   }
+}
+
+/* Asymmetric variant of the activation quantizer (Sec. 4, "Quantization Details": the paper's
+ * activations are per-token asymmetric 4-bit).  The paper gives no formula; the reading used here
+ * is the usual min/max affine quantizer with the range forced to contain zero:
+ *   lo = min(0, min_c y_c), hi = max(0, max_c y_c), s = (hi - lo) / 15 (s = 1 for an all-zero row),
+ *   z = round_half_even(-lo / s) clamped to [0, 15], u_c = clamp(round_half_even(y_c / s) + z, 0, 15),
+ * and the value a code stands for is s * (u - z).  As in the symmetric case the scale is rounded
+ * to binary32 first (it crosses the library boundary as binary32) and the rounded value divides. */
+void xqo_quantize_asym(const double *y, int64_t rows, int64_t cols, uint8_t *codes, float *scales,
+                       int32_t *zero_points) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    const double *yr = y + r * cols;
+    double lo = 0.0, hi = 0.0;
+    for (int64_t c = 0; c < cols; ++c) {
+      if (yr[c] < lo) lo = yr[c];
+      if (yr[c] > hi) hi = yr[c];
+    }
+    float s32 = hi > lo ? (float)((hi - lo) / 15.0) : 1.0f;
+    if (!(s32 > 0.0f)) s32 = 1.0f;
+    double s = (double)s32;
+    double z = nearbyint(-lo / s);
+    if (z < 0.0) z = 0.0;
+    if (z > 15.0) z = 15.0;
+    scales[r] = s32;
+    zero_points[r] = (int32_t)z;
+    for (int64_t c = 0; c < cols; ++c) {
+      double q = nearbyint(yr[c] / s) + z;
+      if (q > 15.0) q = 15.0;
+      if (q < 0.0) q = 0.0;
+      codes[r * cols + c] = (uint8_t)q;
+    }
+  }
+}
+
+/* Quantized product with unsigned activation codes and signed weight codes, exact. */
+void xqo_gemm_u_i64(const uint8_t *ux, const int8_t *qw, int64_t M, int64_t N, int64_t Kp,
+                    int64_t *acc) {
+#pragma omp parallel for schedule(static) collapse(2)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n) {
+      int64_t s = 0;
+      for (int64_t c = 0; c < Kp; ++c) s += (int64_t)ux[m * Kp + c] * (int64_t)qw[n * Kp + c];
+      acc[m * N + n] = s;
+    }
+}
+
+/* Dequantizing epilogue of the asymmetric variant:
+ *   sum_c s_x (u - z) * s_w qw = s_x s_w (acc - z * sum_c qw[n][c]),
+ * the row sums of the weight codes computed here; one rounding to bf16. */
+void xqo_epilogue_asym(const int64_t *acc, const float *s_x, const int32_t *zp, const float *s_w,
+                       const int8_t *qw, int64_t M, int64_t N, int64_t Kp, uint16_t *out_bf16) {
+  int64_t *wsum = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+  for (int64_t n = 0; n < N; ++n) {
+    int64_t t = 0;
+    for (int64_t c = 0; c < Kp; ++c) t += qw[n * Kp + c];
+    wsum[n] = t;
+  }
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n)
+      out_bf16[m * N + n] = double_to_bf16((double)(acc[m * N + n] - (int64_t)zp[m] * wsum[n]) *
+                                           (double)s_x[m] * (double)s_w[n]);
+  free(wsum);
 }
 
 /* Two's-complement nibbles, two per byte: byte j of a row holds code 2j in bits 0-3 and code

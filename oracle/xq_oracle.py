@@ -144,6 +144,44 @@ def quantize(y: np.ndarray):
     return codes, scales
 
 
+def quantize_asym(y: np.ndarray):
+    """Per-row asymmetric INT4 (range forced to contain zero): returns (codes uint8 [rows, cols] in 0..15,
+    scales float32 [rows], zero points int32 [rows]); a code u stands for scale * (u - zero point)."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    rows, cols = y.shape
+    codes = np.empty((rows, cols), dtype=np.uint8)
+    scales = np.empty((rows,), dtype=np.float32)
+    zps = np.empty((rows,), dtype=np.int32)
+    _load().xqo_quantize_asym(_p(y), _i64(rows), _i64(cols), _p(codes), _p(scales), _p(zps))
+    return codes, scales, zps
+
+
+def gemm_u_i64(ux: np.ndarray, qw: np.ndarray) -> np.ndarray:
+    """acc[m, n] = sum_c ux[m, c] * qw[n, c] in int64 (unsigned activation codes)."""
+    ux = np.ascontiguousarray(ux, dtype=np.uint8)
+    qw = np.ascontiguousarray(qw, dtype=np.int8)
+    M, Kp = ux.shape
+    N, Kp2 = qw.shape
+    assert Kp == Kp2
+    acc = np.empty((M, N), dtype=np.int64)
+    _load().xqo_gemm_u_i64(_p(ux), _p(qw), _i64(M), _i64(N), _i64(Kp), _p(acc))
+    return acc
+
+
+def epilogue_asym(acc: np.ndarray, s_x: np.ndarray, zp: np.ndarray, s_w: np.ndarray, qw: np.ndarray) -> np.ndarray:
+    """bf16 bits of s_x[m] * s_w[n] * (acc - zp[m] * sum_c qw[n, c])."""
+    acc = np.ascontiguousarray(acc, dtype=np.int64)
+    s_x = np.ascontiguousarray(s_x, dtype=np.float32)
+    zp = np.ascontiguousarray(zp, dtype=np.int32)
+    s_w = np.ascontiguousarray(s_w, dtype=np.float32)
+    qw = np.ascontiguousarray(qw, dtype=np.int8)
+    M, N = acc.shape
+    Kp = qw.shape[1]
+    out = np.empty((M, N), dtype=np.uint16)
+    _load().xqo_epilogue_asym(_p(acc), _p(s_x), _p(zp), _p(s_w), _p(qw), _i64(M), _i64(N), _i64(Kp), _p(out))
+    return out
+
+
 def pack_int4(codes: np.ndarray) -> np.ndarray:
     codes = np.ascontiguousarray(codes, dtype=np.int8)
     rows, cols = codes.shape
@@ -211,6 +249,21 @@ def prepare_weights(pl: Plan, w_bits: np.ndarray):
     per output channel.  Returns (codes int8 [N, Kp], s_w float32 [N])."""
     _, codes, s = rotate_quant(pl, w_bits)
     return codes, s
+
+
+def rotate_quant_asym(pl: Plan, x_bits: np.ndarray):
+    """Online step with the asymmetric activation quantizer: (y fp64, codes uint8, s_x float32, zero points int32)."""
+    y = rotate(pl, x_bits)
+    codes, s, z = quantize_asym(y)
+    return y, codes, s, z
+
+
+def expanded_linear_asym(pl: Plan, x_bits: np.ndarray, w_bits: np.ndarray):
+    """Whole layer with asymmetric activations (weights unchanged: symmetric per channel)."""
+    _, ux, s_x, z = rotate_quant_asym(pl, x_bits)
+    qw, s_w = prepare_weights(pl, w_bits)
+    acc = gemm_u_i64(ux, qw)
+    return epilogue_asym(acc, s_x, z, s_w, qw), acc
 
 
 def expanded_linear(pl: Plan, x_bits: np.ndarray, w_bits: np.ndarray):

@@ -128,3 +128,93 @@ def test_whole_layer_close_to_unquantized_product(oracle):
     qw, sw = oracle.prepare_weights(pl, w)
     manual = (qx.astype(np.float64) * sx[:, None]) @ (qw.astype(np.float64) * sw[:, None]).T
     assert np.allclose(synth.bf16_bits_to_f32(out), manual, rtol=2.0**-8, atol=1e-30)
+
+
+# ---- asymmetric activation quantizer (the paper's setting, Sec. 4 "Quantization Details") --------
+
+def test_asym_quantizer_range_endpoints_and_error_bound(oracle):
+    g = np.random.default_rng(5)
+    y = g.standard_normal((40, 333)) * g.uniform(0.01, 30.0, size=(40, 1)) + g.uniform(-5, 5, size=(40, 1))
+    y[3] = 0.0                      # all-zero row
+    y[4] = np.abs(y[4])             # no negative values: the range still starts at zero
+    y[5] = -np.abs(y[5])            # no positive values
+    u, s, z = oracle.quantize_asym(y)
+    assert u.dtype == np.uint8 and u.min() >= 0 and u.max() <= 15
+    assert s[3] == 1.0 and z[3] == 0 and not u[3].any()
+    assert z[4] == 0 and z[5] == 15
+    lo = np.minimum(y.min(axis=1), 0.0)
+    hi = np.maximum(y.max(axis=1), 0.0)
+    for r in range(y.shape[0]):
+        if r == 3:
+            continue
+        assert np.isclose(s[r], (hi[r] - lo[r]) / 15.0, rtol=1e-6)
+        # the extremes map to the ends of the code range
+        if lo[r] < 0:
+            assert u[r, np.argmin(y[r])] == 0
+        if hi[r] > 0:
+            assert u[r, np.argmax(y[r])] in (14, 15)  # 14 when rounding the zero point shifted the grid down
+        # a code stands for s * (u - z); inside the range the error is at most half a step
+        # (plus the half step by which rounding the zero point can shift the grid)
+        err = np.abs(y[r] - s[r].astype(np.float64) * (u[r].astype(np.float64) - z[r]))
+        assert err.max() <= s[r] * (1.0 + 1e-6)
+        assert np.median(err) <= 0.5 * s[r]
+    assert np.all((z >= 0) & (z <= 15))
+
+
+def test_asym_quantizer_is_exact_on_an_integer_grid(oracle):
+    """Values k * step with k in [-z, 15 - z] and both end points present come back exactly."""
+    step = 0.375
+    for z0 in (0, 3, 8, 15):
+        k = np.arange(-z0, 16 - z0, dtype=np.float64)
+        y = np.tile(k * step, (2, 3))
+        u, s, z = oracle.quantize_asym(y)
+        assert np.allclose(s, step, rtol=1e-7) and np.all(z == z0)
+        assert np.array_equal(u[0, :16].astype(np.int64) - z0, k.astype(np.int64))
+
+
+def test_asym_ties_round_to_even(oracle):
+    # range [-2, 13] -> s = 1, z = 2; y = 0.5, 1.5, 2.5 are exact ties
+    y = np.array([[-2.0, 13.0, 0.5, 1.5, 2.5, -0.5, -1.5]])
+    u, s, z = oracle.quantize_asym(y)
+    assert s[0] == 1.0 and z[0] == 2
+    assert list(u[0].astype(int) - 2) == [-2, 13, 0, 2, 2, 0, -2]
+
+
+def test_asym_epilogue_identity_against_float_product(oracle):
+    """s_x s_w (acc - z wsum) equals the product of the dequantized operands (library matmul, fp64)."""
+    g = np.random.default_rng(9)
+    M, N, Kp = 7, 11, 96
+    ux = g.integers(0, 16, size=(M, Kp), dtype=np.uint8)
+    qw = g.integers(-8, 8, size=(N, Kp), dtype=np.int8)
+    z = g.integers(0, 16, size=M, dtype=np.int32)
+    s_x = synth.scales(M, seed=3, tag="ax")
+    s_w = synth.scales(N, seed=3, tag="aw")
+    acc = oracle.gemm_u_i64(ux, qw)
+    assert np.array_equal(acc, ux.astype(np.int64) @ qw.astype(np.int64).T)
+    out = synth.bf16_bits_to_f32(oracle.epilogue_asym(acc, s_x, z, s_w, qw)).astype(np.float64)
+    xdq = s_x[:, None].astype(np.float64) * (ux.astype(np.float64) - z[:, None])
+    wdq = s_w[:, None].astype(np.float64) * qw.astype(np.float64)
+    want = xdq @ wdq.T
+    assert np.all(np.abs(out - want) <= np.abs(want) * 2.0**-8 + 1e-30)
+    # closed form: all codes 15, zero point 5, weights all -8: acc = -120 Kp, wsum = -8 Kp -> (acc - z wsum) = -80 Kp
+    ux[:] = 15
+    qw[:] = -8
+    z[:] = 5
+    out = synth.bf16_bits_to_f32(oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), np.ones(M, np.float32), z, np.ones(N, np.float32), qw))
+    assert np.all(out == -80.0 * Kp)
+
+
+def test_asym_layer_is_closer_to_the_unquantized_product_than_chance(oracle):
+    """End to end on one-sided activations (where an asymmetric grid has twice the resolution): the
+    asymmetric layer reproduces the fp64 product of the bf16 inputs at least as well as the symmetric one."""
+    K, Kp, M, N = 200, 240, 12, 40
+    pl = oracle.plan(K, Kp)
+    x = synth.activations(M, K, seed=4, tag="asym")
+    w = synth.weights(N, K, seed=4, tag="asym")
+    ref = oracle.ref_product(x, w)
+    out_a = synth.bf16_bits_to_f32(oracle.expanded_linear_asym(pl, x, w)[0]).astype(np.float64)
+    out_s = synth.bf16_bits_to_f32(oracle.expanded_linear(pl, x, w)[0]).astype(np.float64)
+    ea = np.linalg.norm(out_a - ref) / np.linalg.norm(ref)
+    es = np.linalg.norm(out_s - ref) / np.linalg.norm(ref)
+    assert ea < 0.5 and es < 0.5  # both are 4-bit approximations of the same product
+    assert ea <= es * 1.25
