@@ -124,6 +124,28 @@ xq_status xq_w4a4_gemm(const uint8_t* Xq_dev, const float* s_x_dev, int32_t M, c
 xq_status xq_expanded_linear(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w,
                              void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
 
+/* The same three calls with per-token ASYMMETRIC activation codes (Sec. 4: the setting of the
+ * paper's experiments; weights stay symmetric per channel).  For each row, with y as above,
+ * lo = min(0, min y), hi = max(0, max y):
+ *   s_x = (hi - lo) / 15 (1 if hi = lo);  z = clamp(round_half_even(-lo / s_x), 0, 15);
+ *   u = clamp(round_half_even(y / s_x) + z, 0, 15), which stands for s_x * (u - z).
+ * Storage: codes and zero point are kept shifted by -8, so Xq holds the nibble c = u - 8
+ * (two's complement, same packing as xq_rotate_quant) and zp_dev, dev int32 [M], receives
+ * z - 8, in -8..7; a stored code stands for s_x * (c - zp).  The product is
+ *   acc[m][n] = sum_c (qx[m][c] - zp[m]) * qw[n][c]      (exact, int32; this is what acc_opt gets)
+ *   out[m][n] = bf16( acc * s_x[m] * s_w[n] ),
+ * computed as the signed product minus zp[m] times the channel's code sum, which the weights
+ * object holds.  xq_w4a4_gemm_asym accepts any nibbles and any zp in -8..7.  All other arguments,
+ * layouts, workspace and error behaviour as in the symmetric calls. */
+xq_status xq_rotate_quant_asym(const void* X_bf16_dev, int32_t M, int64_t ldx,
+                               const xq_hadamard_plan_t* plan, uint8_t* Xq_dev, float* s_x_dev,
+                               int32_t* zp_dev, float* Y_f32_opt_dev, void* stream);
+xq_status xq_w4a4_gemm_asym(const uint8_t* Xq_dev, const float* s_x_dev, const int32_t* zp_dev, int32_t M,
+                            const xq_weights* w, void* out_bf16_dev, int32_t* acc_opt_dev, void* ws_dev,
+                            size_t ws_bytes, void* stream);
+xq_status xq_expanded_linear_asym(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w,
+                                  void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
 /* The whole layer on HOST buffers: copies X (host, [M, K] contiguous; pinned memory makes the
  * copies asynchronous) into the workspace, runs the layer, copies out (host, bf16 [M, N]) back
  * and synchronizes `stream` before returning. */

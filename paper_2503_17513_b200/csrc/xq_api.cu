@@ -69,6 +69,7 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
   w->plan = pl;
   w->packed = nullptr;
   w->s_w = nullptr;
+  w->w_sum = nullptr;
   w->hp_signs = nullptr;
   if (cudaGetDevice(&w->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&w->sms, cudaDevAttrMultiProcessorCount, w->device) != cudaSuccess) {
@@ -77,7 +78,8 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
   }
   const size_t bytes = (size_t)w->Np * w->Kpp / 2;
   if (cudaMalloc((void**)&w->packed, bytes) != cudaSuccess ||
-      cudaMalloc((void**)&w->s_w, sizeof(float) * (size_t)w->Np) != cudaSuccess) {
+      cudaMalloc((void**)&w->s_w, sizeof(float) * (size_t)w->Np) != cudaSuccess ||
+      cudaMalloc((void**)&w->w_sum, sizeof(int32_t) * (size_t)w->Np) != cudaSuccess) {
     cudaGetLastError();
     xq_weights_free(w);
     return XQ_ERR_ALLOC;
@@ -117,6 +119,8 @@ xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w) {
   off += align_up((size_t)M_max * (size_t)(w->Kpp / 2), 256);
   L.sx = off;
   off += align_up(sizeof(float) * (size_t)M_max, 256);
+  L.zp = off;
+  off += align_up(sizeof(int32_t) * (size_t)M_max, 256);
   L.xstage = off;
   off += align_up((size_t)M_max * (size_t)w->K * 2, 256);
   L.ostage = off;
@@ -179,6 +183,7 @@ void xq_weights_free(xq_weights* w) {
   if (!w) return;
   if (w->packed) cudaFree(w->packed);
   if (w->s_w) cudaFree(w->s_w);
+  if (w->w_sum) cudaFree(w->w_sum);
   if (w->hp_signs) cudaFree(w->hp_signs);
   delete w;
 }
@@ -212,9 +217,10 @@ xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t K
                                     cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(w->s_w, 0, sizeof(float) * (size_t)w->Np, st);
   if (e == cudaSuccess)
-    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, nullptr, w->hp_signs, w->sms, st);
+    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, nullptr, w->hp_signs, nullptr, w->sms, st);
   if (e == cudaSuccess)
     e = xq_launch_relayout_to_blocks((const uint8_t*)dCanon.p, N, Kp, w->packed, w->Np, w->Kpp, st);
+  if (e == cudaSuccess) e = xq_launch_weight_sums(w->packed, w->Np, w->Kpp, w->w_sum, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -247,6 +253,7 @@ xq_status xq_weights_import(const int8_t* codes, const float* s_w, int32_t N, in
   if (e == cudaSuccess) e = xq_launch_pack_codes((const int8_t*)dCodes.p, (int64_t)(count / 2), (uint8_t*)dCanon.p, st);
   if (e == cudaSuccess)
     e = xq_launch_relayout_to_blocks((const uint8_t*)dCanon.p, N, Kp, w->packed, w->Np, w->Kpp, st);
+  if (e == cudaSuccess) e = xq_launch_weight_sums(w->packed, w->Np, w->Kpp, w->w_sum, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -292,11 +299,17 @@ xq_status xq_workspace_init(void* ws, size_t ws_bytes, void* stream) {
   return XQ_OK;
 }
 
-xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq,
-                          float* s_x, float* Yopt, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// asym: zp is required and receives the zero points; otherwise zp must be null.
+xq_status rotate_quant_impl(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq, float* s_x,
+                            int32_t* zp, bool asym, float* Yopt, void* stream) {
   if (!plan || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!X || !Xq || !s_x) return XQ_ERR_INVALID_ARG;
+  if (!X || !Xq || !s_x || (asym && !zp)) return XQ_ERR_INVALID_ARG;
+  if (zp && (reinterpret_cast<uintptr_t>(zp) & 3u)) return XQ_ERR_INVALID_ARG;
   // the plan must be one xq_hadamard_plan would return
   xq_hadamard_plan_t chk;
   xq_status s = xq_hadamard_plan(plan->K, plan->Kp, &chk);
@@ -311,32 +324,33 @@ xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadama
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
-  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, nullptr, nullptr, sms, (cudaStream_t)stream) != cudaSuccess) {
+  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, nullptr, nullptr, zp, sms, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
   return XQ_OK;
 }
 
-xq_status xq_w4a4_gemm(const uint8_t* Xq, const float* s_x, int32_t M, const xq_weights* w, void* out,
-                       int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
+xq_status gemm_impl(const uint8_t* Xq, const float* s_x, const int32_t* zp, bool asym, int32_t M, const xq_weights* w, void* out,
+                    int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!Xq || !s_x || !out) return XQ_ERR_INVALID_ARG;
+  if (!Xq || !s_x || !out || (asym && !zp)) return XQ_ERR_INVALID_ARG;
+  if (zp && (reinterpret_cast<uintptr_t>(zp) & 3u)) return XQ_ERR_INVALID_ARG;
   if (!aligned16(Xq) || !aligned16(out) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
       (acc_opt && !aligned16(acc_opt)))
     return XQ_ERR_INVALID_ARG;
   const xq_ws_layout L = xq_ws_compute(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
-  if (xq_launch_gemm(Xq, s_x, M, w, out, acc_opt, ws, L, false, (cudaStream_t)stream) != cudaSuccess) {
+  if (xq_launch_gemm(Xq, s_x, zp, M, w, out, acc_opt, ws, L, false, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
   return XQ_OK;
 }
 
-xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out, void* ws,
-                             size_t ws_bytes, void* stream) {
+xq_status linear_impl(const void* X, int32_t M, int64_t ldx, const xq_weights* w, bool asym, void* out, void* ws,
+                      size_t ws_bytes, void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X || !out) return XQ_ERR_INVALID_ARG;
@@ -346,14 +360,49 @@ xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_wei
   uint8_t* base = (uint8_t*)ws;
   uint8_t* Xq = base + L.xq;
   float* sx = (float*)(base + L.sx);
+  int32_t* zp = asym ? (int32_t*)(base + L.zp) : nullptr;
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + L.a8 : nullptr;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->hp_signs, w->sms, st) != cudaSuccess ||
-      xq_launch_gemm(Xq, sx, M, w, out, nullptr, ws, L, A8 != nullptr, st) != cudaSuccess) {
+  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->hp_signs, zp, w->sms, st) != cudaSuccess ||
+      xq_launch_gemm(Xq, sx, zp, M, w, out, nullptr, ws, L, A8 != nullptr, st) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
   return XQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq,
+                          float* s_x, float* Yopt, void* stream) {
+  return rotate_quant_impl(X, M, ldx, plan, Xq, s_x, nullptr, false, Yopt, stream);
+}
+
+xq_status xq_rotate_quant_asym(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq,
+                               float* s_x, int32_t* zp, float* Yopt, void* stream) {
+  return rotate_quant_impl(X, M, ldx, plan, Xq, s_x, zp, true, Yopt, stream);
+}
+
+xq_status xq_w4a4_gemm(const uint8_t* Xq, const float* s_x, int32_t M, const xq_weights* w, void* out,
+                       int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
+  return gemm_impl(Xq, s_x, nullptr, false, M, w, out, acc_opt, ws, ws_bytes, stream);
+}
+
+xq_status xq_w4a4_gemm_asym(const uint8_t* Xq, const float* s_x, const int32_t* zp, int32_t M, const xq_weights* w,
+                            void* out, int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
+  return gemm_impl(Xq, s_x, zp, true, M, w, out, acc_opt, ws, ws_bytes, stream);
+}
+
+xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out, void* ws,
+                             size_t ws_bytes, void* stream) {
+  return linear_impl(X, M, ldx, w, false, out, ws, ws_bytes, stream);
+}
+
+xq_status xq_expanded_linear_asym(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  return linear_impl(X, M, ldx, w, true, out, ws, ws_bytes, stream);
 }
 
 xq_status xq_expanded_linear_host(const void* X_host, int32_t M, const xq_weights* w, void* out_host, void* ws,

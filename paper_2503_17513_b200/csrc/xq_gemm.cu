@@ -1,5 +1,6 @@
 // Quantized product of the expanded layer (paper Sec. 3: Q(XR) Q(W~), computed at inference)
-// with the dequantizing epilogue: acc = sum_c qx qw (int32, exact), out = bf16(acc s_x s_w).
+// with the dequantizing epilogue: acc = sum_c (qx - z) qw (int32, exact; z = 0 for symmetric
+// tokens, else sum_c qx qw - z sum_c qw), out = bf16(acc s_x s_w).
 #include <cuda_bf16.h>
 
 #include "xq_internal.h"
@@ -11,7 +12,8 @@ namespace {
 
 // General kernel: one thread per output, any M, N, K' (K' a multiple of 8).  Shape-agnostic
 // path for sizes the tiled kernels do not take.
-__global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __restrict__ Xq, const float* __restrict__ sx, int M,
+__global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __restrict__ Xq, const float* __restrict__ sx,
+                                                           const int32_t* __restrict__ zp, const int32_t* __restrict__ wsum, int M,
                                                            const uint8_t* __restrict__ Wb, const float* __restrict__ sw, int N,
                                                            int Kp, int k_groups, __nv_bfloat16* __restrict__ out,
                                                            int32_t* __restrict__ acc_opt) {
@@ -30,6 +32,7 @@ __global__ void __launch_bounds__(128) gemm_general_kernel(const uint32_t* __res
     acc = __dp4a((int)wo, (int)xo, acc);
   }
   acc >>= 8;
+  if (zp) acc -= zp[m] * wsum[n];
   if (acc_opt) acc_opt[(long long)m * N + n] = acc;
   out[(long long)m * N + n] = __float2bfloat16_rn((float)acc * sx[m] * sw[n]);
 }
@@ -57,12 +60,12 @@ cudaError_t xq_launch_selftest_wait_timeout(int32_t* status, cudaStream_t st) {
 
 bool xq_gemm_wants_a8(int32_t M, const xq_weights* w) { return M > XQ_DECODE_MAX_M && xq_prefill_supported(M, w); }
 
-cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w, void* out,
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, bool a8_ready, cudaStream_t st) {
   if (w->Kp % 8 != 0) return cudaErrorInvalidValue;
   int32_t* header = (int32_t*)ws;
   if (M <= XQ_DECODE_MAX_M) {
-    const cudaError_t e = xq_launch_gemm_decode(Xq, sx, M, w, out, acc_opt, header, st);
+    const cudaError_t e = xq_launch_gemm_decode(Xq, sx, zp, M, w, out, acc_opt, header, st);
     if (e != cudaErrorNotSupported) return e;
   }
   if (xq_prefill_supported(M, w) && L.a8 != 0) {
@@ -71,10 +74,10 @@ cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const 
       const cudaError_t e = xq_launch_expand_tokens(Xq, M, w->Kp, A8, st);
       if (e != cudaSuccess) return e;
     }
-    return xq_launch_gemm_prefill(A8, sx, M, w, out, acc_opt, header, w->sms, st);
+    return xq_launch_gemm_prefill(A8, sx, zp, M, w, out, acc_opt, header, w->sms, st);
   }
   dim3 grid((w->N + 127) / 128, M);
-  gemm_general_kernel<<<grid, 128, 0, st>>>((const uint32_t*)Xq, sx, M, w->packed, w->s_w, w->N, w->Kp,
+  gemm_general_kernel<<<grid, 128, 0, st>>>((const uint32_t*)Xq, sx, zp, w->w_sum, M, w->packed, w->s_w, w->N, w->Kp,
                                             w->Kpp / XQ_K_GROUP, (__nv_bfloat16*)out, acc_opt);
   return cudaGetLastError();
 }

@@ -48,6 +48,8 @@ struct DecodeParams {
   const float* sx;
   __nv_bfloat16* out;
   int32_t* acc_opt;
+  const int32_t* zp;    // per-token zero points of asymmetric activation codes, or null
+  const int32_t* wsum;  // per-channel sums of the weight codes
   int32_t* status;
   int M, N, Kp;
   int k_groups;     // groups of 32 codes per channel block in the weight layout (K'' / 32)
@@ -345,6 +347,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] >>= 8;  // every product carries 16 x 16
       const int n0 = (b0 + j) * 16 + 8 * h;
+      if (p.zp) {  // sum (c - z) qw = sum c qw - z sum qw (w_sum covers the padded rows)
+        const int z = p.zp[m];
+        const int4 w0 = *reinterpret_cast<const int4*>(p.wsum + n0), w1 = *reinterpret_cast<const int4*>(p.wsum + n0 + 4);
+        v[0] -= z * w0.x; v[1] -= z * w0.y; v[2] -= z * w0.z; v[3] -= z * w0.w;
+        v[4] -= z * w1.x; v[5] -= z * w1.y; v[6] -= z * w1.z; v[7] -= z * w1.w;
+      }
       const bool pre = idx == tid;  // scales already in registers
       const float sxm = pre ? e_sx : p.sx[m];
       const size_t o = (size_t)m * p.N + n0;
@@ -507,8 +515,8 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
 
 }  // namespace
 
-cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
-                                  int32_t* acc_opt, int32_t* status, cudaStream_t st) {
+cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
+                                  void* out, int32_t* acc_opt, int32_t* status, cudaStream_t st) {
   const DecodePlan d = decode_plan(M, w);
   if (d.stages < 16) return cudaErrorNotSupported;
   DecodeParams p;
@@ -518,6 +526,8 @@ cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M,
   p.sx = sx;
   p.out = (__nv_bfloat16*)out;
   p.acc_opt = acc_opt;
+  p.zp = zp;
+  p.wsum = w->w_sum;
   p.status = status;
   p.M = M;
   p.N = w->N;

@@ -52,13 +52,15 @@ struct Cfg {
   static constexpr int kThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;
   static constexpr int kAccBufs = MH == 1 ? 2 : 1;
   static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kI8Stages * kI8StageBytes + (size_t)kPkStages * kPkBBytes +
-                                       kEpiWarps * BN * sizeof(float) + 256 /*barriers, flags*/;
+                                       kEpiWarps * 2 * BN * sizeof(float) /*scales, code sums*/ + 256 /*barriers, flags*/;
 };
 
 struct PrefillParams {
   const uint8_t* W;    // block layout
   const float* sw;
   const float* sx;
+  const int32_t* zp;   // per-token zero points of asymmetric activation codes, or null
+  const int32_t* wsum; // per-channel sums of the weight codes
   __nv_bfloat16* out;
   int32_t* acc_opt;
   int32_t* status;
@@ -90,7 +92,7 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
   unsigned char* i8 = base;                                        // kI8Stages x [A (MH x 16 KiB) | B 32 KiB], 1024-aligned
   unsigned char* pk = i8 + (size_t)kI8Stages * kI8StageBytes;      // kPkStages x 16 KiB of packed weights
   float* sw_tile = reinterpret_cast<float*>(pk + (size_t)kPkStages * kPkBBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sw_tile + C::kEpiWarps * BN);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sw_tile + C::kEpiWarps * 2 * BN);
   uint64_t* pk_full = bars;
   uint64_t* pk_empty = pk_full + kPkStages;
   uint64_t* i8_full = pk_empty + kPkStages;
@@ -219,7 +221,8 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
     // ---------------- epilogue ------------------------------------------------------------------
     const int q = warp & 3;                        // tensor-memory lane quarter this warp may read
     const int eh = (warp - kFirstEpiWarp) >> 2;    // which 128-row half of the tile (MH = 2)
-    float* sw_mine = sw_tile + (warp - kFirstEpiWarp) * BN;  // a private copy per warp: no cross-warp barrier
+    float* sw_mine = sw_tile + (warp - kFirstEpiWarp) * 2 * BN;  // a private copy per warp: no cross-warp barrier
+    int* ws_mine = reinterpret_cast<int*>(sw_mine + BN);         // code sums of the tile's channels (asymmetric tokens)
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
@@ -228,10 +231,14 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
       const uint32_t use = kAccBufs == 2 ? (tcount >> 1) : tcount;
       const int n0 = tn * BN;
       __syncwarp();
-      for (int i = lane; i < BN; i += 32) sw_mine[i] = (n0 + i < p.N) ? p.sw[n0 + i] : 0.f;
+      for (int i = lane; i < BN; i += 32) {
+        sw_mine[i] = (n0 + i < p.N) ? p.sw[n0 + i] : 0.f;
+        ws_mine[i] = (p.zp && n0 + i < p.N) ? p.wsum[n0 + i] : 0;
+      }
       __syncwarp();
       const int m = (tm * MH + eh) * BMH + q * 32 + lane;
       const float sxm = m < p.M ? p.sx[m] : 0.f;
+      const int zpm = (p.zp && m < p.M) ? p.zp[m] : 0;
       ok = mbar_wait_bounded(&acc_full[buf], use & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
       if (!ok) break;
       tc_fence_after_sync();
@@ -249,7 +256,8 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
             if (nc + 8 * g8 < p.N) {  // N is a multiple of 8 on this path
               int a[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) a[e] = (int)v[8 * g8 + e] >> 8;  // every product carries 16 x 16
+              for (int e = 0; e < 8; ++e)  // every product carries 16 x 16; sum (c - z) qw = sum c qw - z sum qw
+                a[e] = ((int)v[8 * g8 + e] >> 8) - zpm * ws_mine[c * 32 + 8 * g8 + e];
               if (p.acc_opt) {
                 *reinterpret_cast<int4*>(p.acc_opt + o + 8 * g8) = make_int4(a[0], a[1], a[2], a[3]);
                 *reinterpret_cast<int4*>(p.acc_opt + o + 8 * g8 + 4) = make_int4(a[4], a[5], a[6], a[7]);
@@ -395,8 +403,8 @@ cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, ui
   return cudaLaunchKernelEx(&cfg, expand_tokens_kernel, (const uint4*)Xq, pieces, (uint4*)A8);
 }
 
-cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, int32_t M, const xq_weights* w, void* out,
-                                   int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st) {
+cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
+                                   void* out, int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st) {
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
   CUtensorMap mapA;
@@ -411,6 +419,8 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, int32_t M
   p.W = w->packed;
   p.sw = w->s_w;
   p.sx = sx;
+  p.zp = zp;
+  p.wsum = w->w_sum;
   p.out = (__nv_bfloat16*)out;
   p.acc_opt = acc_opt;
   p.status = status;

@@ -64,6 +64,36 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_p
                : "r"(addr));
 }
 
+// Quantizer constants of one row (paper Sec. 4: per-token activations, per-channel weights).
+// Either way a stored code is c = clamp(rne(y / s) + z, -8, 7) and stands for s * (c - z).
+// Symmetric: s = absmax / 7 (1 for a zero row), z = 0.
+// Asymmetric (the range is forced to contain zero): s = (hi - lo) / 15 and the unsigned zero point
+// clamp(rne(-lo / s), 0, 15); codes and zero point are kept shifted by -8, so that they are the same
+// signed nibbles the symmetric path stores and the signed integer product serves both.
+struct RowQuant {
+  float s, inv;
+  int z;
+};
+__device__ __forceinline__ RowQuant row_quant_sym(float amax) {
+  RowQuant r;
+  r.s = amax > 0.f ? __fdiv_rn(amax, 7.f) : 1.f;
+  if (!(r.s > 0.f)) r.s = 1.f;
+  r.inv = __frcp_rn(r.s);
+  r.z = 0;
+  return r;
+}
+__device__ __forceinline__ RowQuant row_quant_asym(float lo, float hi) {  // lo <= 0 <= hi
+  RowQuant r;
+  r.s = hi > lo ? __fdiv_rn(hi - lo, 15.f) : 1.f;
+  if (!(r.s > 0.f)) r.s = 1.f;
+  r.inv = __frcp_rn(r.s);
+  r.z = max(0, min(15, __float2int_rn(__fdiv_rn(-lo, r.s)))) - 8;
+  return r;
+}
+__device__ __forceinline__ int row_code(const RowQuant& r, float y) {
+  return max(-8, min(7, __float2int_rn(y * r.inv) + r.z));
+}
+
 __device__ __forceinline__ uint32_t sign_bf16(int s) { return s > 0 ? 0x3F80u : (s < 0 ? 0xBF80u : 0u); }
 
 }  // namespace xqhad

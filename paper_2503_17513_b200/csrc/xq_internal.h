@@ -35,6 +35,7 @@ struct xq_weights {
   xq_hadamard_plan_t plan;
   uint8_t* packed;     // device, Np * Kpp / 2 bytes, block layout above
   float* s_w;          // device, Np floats (padding rows hold 0)
+  int32_t* w_sum;      // device, Np ints: sum of the row's codes (the zero-point term of asymmetric tokens)
   uint16_t* hp_signs;  // device, bf16 image of H_p^T for the rotate kernel ([P16][P16 + 8]); NULL when p == 1
   int device;
   int sms;             // multiprocessors of that device
@@ -53,6 +54,7 @@ struct xq_ws_layout {
   size_t header;   // XQ_WS_HEADER_BYTES
   size_t xq;       // M_max * Kp/2 bytes of packed activations
   size_t sx;       // M_max floats
+  size_t zp;       // M_max ints: zero points of asymmetric activation codes
   size_t xstage;   // M_max * K bf16 (host entry point)
   size_t ostage;   // M_max * N bf16 (host entry point)
   size_t a8;       // M_max * K'' bytes: byte-per-code tokens for the tensor-core GEMM (only when M_max > 32)
@@ -70,13 +72,15 @@ constexpr int XQ_DECODE_MAX_M = 32;
 // A8opt (optional): byte-per-code copy of the codes in the operand format of the tcgen05 GEMM, [M, Kp].
 // Hsigns (optional): device image of H_p^T as bf16, [P16][P16 + 8] with P16 = p rounded up to 16
 // (xq_weights::hp_signs); without it the kernel derives the signs itself.
+// zp (optional): when given, the rows are quantized asymmetrically (unsigned codes 0..15) and zp[m]
+// receives the row's zero point; when null, symmetrically (signed codes -8..7).
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl,
-                                   uint8_t* Xq, float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms,
-                                   cudaStream_t st);
+                                   uint8_t* Xq, float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp,
+                                   int sms, cudaStream_t st);
 // Throughput form for many rows (several independent row groups per CTA, double-buffered loads).
 bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl);
 cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
-                                  float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st);
+                                  float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st);
 constexpr int XQ_ROTATE_ROWS_MIN_M = 48;  // below this the one-CTA-per-row kernel has the shorter latency
 cudaError_t xq_launch_relayout_to_blocks(const uint8_t* canon, int32_t N, int32_t Kp, uint8_t* blocks,
                                          int32_t Np, int32_t Kpp, cudaStream_t st);
@@ -84,19 +88,22 @@ cudaError_t xq_launch_relayout_from_blocks(const uint8_t* blocks, int32_t Np, in
                                            int32_t N, int32_t Kp, cudaStream_t st);
 cudaError_t xq_launch_pack_codes(const int8_t* codes, int64_t count_pairs, uint8_t* packed, cudaStream_t st);
 cudaError_t xq_launch_unpack_codes(const uint8_t* packed, int64_t count_pairs, int8_t* codes, cudaStream_t st);
+// w_sum[n] = sum of the codes of row n of the block layout (0 for padding rows).
+cudaError_t xq_launch_weight_sums(const uint8_t* blocks, int32_t Np, int32_t Kpp, int32_t* w_sum, cudaStream_t st);
 // Decode path: returns cudaErrorNotSupported (nothing launched) when the shape does not fit it.
-cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
-                                  int32_t* acc_opt, int32_t* status, cudaStream_t st);
+// zp (optional, here and below): per-token zero points; the epilogue then removes zp[m] * w_sum[n].
+cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
+                                  void* out, int32_t* acc_opt, int32_t* status, cudaStream_t st);
 // Tensor-core path: takes the tokens one code per byte (16 x code, even codes of every word first),
 // as written by the rotate kernels' optional output or by xq_launch_expand_tokens.
 bool xq_prefill_supported(int32_t M, const xq_weights* w);
 cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, uint8_t* A8, cudaStream_t st);
-cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, int32_t M, const xq_weights* w, void* out,
-                                   int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st);
+cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
+                                   void* out, int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st);
 // True when M tokens against w go down the tensor-core path (so that the caller lets the rotate
 // kernel write the byte-per-code tokens).
 cudaError_t xq_launch_selftest_wait_timeout(int32_t* status, cudaStream_t st);
 bool xq_gemm_wants_a8(int32_t M, const xq_weights* w);
 // a8_ready: the a8 region of the workspace already holds the byte-per-code tokens.
-cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, int32_t M, const xq_weights* w, void* out,
+cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w, void* out,
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, bool a8_ready, cudaStream_t st);

@@ -24,7 +24,8 @@ __device__ __forceinline__ int quant_code(float y, float s) {
 __global__ void __launch_bounds__(256) rotate_quant_general_kernel(const __nv_bfloat16* __restrict__ X, int M,
                                                                    long long ldx, xq_hadamard_plan_t pl, float gamma,
                                                                    uint8_t* __restrict__ Xq, float* __restrict__ sx,
-                                                                   float* __restrict__ Yopt, uint8_t* __restrict__ A8opt) {
+                                                                   float* __restrict__ Yopt, uint8_t* __restrict__ A8opt,
+                                                                   int32_t* __restrict__ zp) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int K = pl.K, Kp = pl.Kp, p = pl.p, n = 1 << pl.log2n, q = pl.q;
   float* bufA = reinterpret_cast<float*>(smem_raw);
@@ -65,19 +66,27 @@ __global__ void __launch_bounds__(256) rotate_quant_general_kernel(const __nv_bf
       }
       __syncthreads();
     }
-    float amax = 0.f;
+    float vmax = 0.f, vmin = 0.f;
     for (int c = threadIdx.x; c < Kp; c += blockDim.x) {
       const float v = y[c] * gamma;
       y[c] = v;
-      amax = fmaxf(amax, fabsf(v));
+      vmax = fmaxf(vmax, v);
+      vmin = fminf(vmin, v);
     }
-    amax = block_max(amax, red);
-    float s = amax > 0.f ? __fdiv_rn(amax, 7.f) : 1.f;
-    if (!(s > 0.f)) s = 1.f;
-    if (threadIdx.x == 0) sx[row] = s;
+    RowQuant rq;
+    if (zp) {
+      vmax = block_max(vmax, red);
+      vmin = -block_max(-vmin, red);
+      rq = row_quant_asym(vmin, vmax);
+      if (threadIdx.x == 0) zp[row] = rq.z;
+    } else {
+      rq = row_quant_sym(block_max(fmaxf(vmax, -vmin), red));
+    }
+    if (threadIdx.x == 0) sx[row] = rq.s;
     uint8_t* out = Xq + (long long)row * (Kp / 2);
     for (int j = threadIdx.x; j < Kp / 2; j += blockDim.x) {
-      const int lo = quant_code(y[2 * j], s), hi = quant_code(y[2 * j + 1], s);
+      const int lo = zp ? row_code(rq, y[2 * j]) : quant_code(y[2 * j], rq.s);
+      const int hi = zp ? row_code(rq, y[2 * j + 1]) : quant_code(y[2 * j + 1], rq.s);
       out[j] = (uint8_t)((lo & 0xF) | ((hi & 0xF) << 4));
       if (A8opt) {
         // operand format of the tcgen05 GEMM: word kg of 8 codes -> 4 bytes of even codes x16, 4 of odd
@@ -110,7 +119,8 @@ template <int LOG2NB, int KS>
 __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx,
                                                               xq_hadamard_plan_t pl, float gamma, uint8_t* __restrict__ Xq,
                                                               float* __restrict__ sx, float* __restrict__ Yopt,
-                                                              uint8_t* __restrict__ A8opt, const __nv_bfloat16* __restrict__ Hsigns) {
+                                                              uint8_t* __restrict__ A8opt, const __nv_bfloat16* __restrict__ Hsigns,
+                                                              int32_t* __restrict__ zp) {
   constexpr int NB = 1 << LOG2NB;  // columns per warp
   constexpr int NT8 = NB / 8;      // n-tiles per warp
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -243,26 +253,33 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
       }
     }
     // scale by 1/sqrt(K'), per-token absmax
-    float amax = 0.f;
+    // (rows of the tile padding hold zeros: harmless, the asymmetric range contains zero anyway)
+    float vmax = 0.f, vmin = 0.f;
 #pragma unroll
     for (int j = 0; j < NT8; ++j)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         acc[j][e] *= gamma;
-        amax = fmaxf(amax, fabsf(acc[j][e]));
+        vmax = fmaxf(vmax, acc[j][e]);
+        vmin = fminf(vmin, acc[j][e]);
       }
-    amax = block_max(amax, red);
-    float s = amax > 0.f ? __fdiv_rn(amax, 7.f) : 1.f;
-    if (!(s > 0.f)) s = 1.f;
-    const float inv = __frcp_rn(s);
+    RowQuant rq;
+    if (zp) {
+      vmax = block_max(vmax, red);
+      vmin = -block_max(-vmin, red);
+      rq = row_quant_asym(vmin, vmax);
+    } else {
+      rq = row_quant_sym(block_max(fmaxf(vmax, -vmin), red));
+    }
+    const float s = rq.s;
     // quantize, pack: the quad's four bytes of one (row, j) form one word of 8 codes
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
       const int a2 = 16 * mt + g + 8 * r;
 #pragma unroll
       for (int j = 0; j < NT8; ++j) {
-        const int lo = max(-8, min(7, __float2int_rn(acc[j][2 * r] * inv)));
-        const int hi = max(-8, min(7, __float2int_rn(acc[j][2 * r + 1] * inv)));
+        const int lo = row_code(rq, acc[j][2 * r]);
+        const int hi = row_code(rq, acc[j][2 * r + 1]);
         uint32_t w = (uint32_t)((lo & 0xF) | ((hi & 0xF) << 4)) << (8 * t);
         w |= __shfl_xor_sync(0xffffffffu, w, 1);
         w |= __shfl_xor_sync(0xffffffffu, w, 2);
@@ -281,7 +298,10 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
       }
     }
     __syncthreads();
-    if (tid == 0) sx[row] = s;
+    if (tid == 0) {
+      sx[row] = s;
+      if (zp) zp[row] = rq.z;
+    }
     uint4* dst = reinterpret_cast<uint4*>(Xq + (long long)row * (Kp / 2));
     for (int i = tid; i < Kp / 32; i += nthreads) {
       const uint4 v = reinterpret_cast<const uint4*>(outp)[i];
@@ -303,7 +323,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
 
 template <int LOG2NB, int KS>
 cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
-                      float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms, cudaStream_t st) {
+                      float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st) {
   const int n = 1 << pl.log2n, NB = 1 << LOG2NB, NC = n / NB, MT = (pl.p + 15) / 16;
   size_t smem = (size_t)KS * 16 * (n + 8) * 2 + (size_t)pl.Kp / 2 + 128 + (size_t)(3 * pl.q + 1) + 32;
   if (Hsigns) smem += (size_t)MT * 16 * (MT * 16 + 8) * 2;
@@ -324,17 +344,17 @@ cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_p
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt,
-                            (const __nv_bfloat16*)Hsigns);
+                            (const __nv_bfloat16*)Hsigns, zp);
 }
 
 template <int LOG2NB>
 cudaError_t launch_tc_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                         float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms, cudaStream_t st) {
+                         float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st) {
   switch (ks) {
-    case 1: return launch_tc<LOG2NB, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
-    case 2: return launch_tc<LOG2NB, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
-    case 3: return launch_tc<LOG2NB, 3>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
-    default: return launch_tc<LOG2NB, 4>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
+    case 1: return launch_tc<LOG2NB, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
+    case 2: return launch_tc<LOG2NB, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
+    case 3: return launch_tc<LOG2NB, 3>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
+    default: return launch_tc<LOG2NB, 4>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
   }
 }
 
@@ -383,6 +403,20 @@ __global__ void unpack_codes_kernel(const uint8_t* __restrict__ packed, long lon
   }
 }
 
+// One thread per row of the block layout: the sum of its K'' signed nibbles (padding holds zeros).
+__global__ void weight_sums_kernel(const uint8_t* __restrict__ blocks, int Np, int Kpp, int32_t* __restrict__ w_sum) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= Np) return;
+  const int k_groups = Kpp / XQ_K_GROUP;
+  int acc = 0;
+  for (int kg = 0; kg < Kpp / 8; ++kg) {
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(blocks + xq_weight_word_offset(n, kg, k_groups));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc += (int)(w << (28 - 4 * i)) >> 28;
+  }
+  w_sum[n] = acc;
+}
+
 inline int grid_for(long long work, int threads) {
   long long g = (work + threads - 1) / threads;
   if (g < 1) g = 1;
@@ -393,10 +427,10 @@ inline int grid_for(long long work, int threads) {
 }  // namespace
 
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq,
-                                   float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int sms, cudaStream_t st) {
+                                   float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st) {
   // many rows, or an order that only the multi-row-group kernel and the general kernel take
   if ((M >= XQ_ROTATE_ROWS_MIN_M || pl.log2n > 8 || pl.p == 1) && xq_rotate_rows_supported(pl))
-    return xq_launch_rotate_rows(X, M, ldx, pl, Xq, sx, Yopt, A8opt, sms, st);
+    return xq_launch_rotate_rows(X, M, ldx, pl, Xq, sx, Yopt, A8opt, zp, sms, st);
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
   const int n = 1 << pl.log2n;
   const int rows_a = (pl.K + n - 1) / n;
@@ -406,16 +440,16 @@ cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const 
   if (tc) {
     const int ks = (rows_a + 15) / 16;
     switch (pl.log2n) {
-      case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
-      case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
-      default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, sms, st);
+      case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
+      case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
+      default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
     }
   }
   const size_t smem = sizeof(float) * (2 * (size_t)pl.Kp + 32) + (size_t)(3 * pl.q + 1) + 16;
   cudaError_t e = cudaFuncSetAttribute(rotate_quant_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int grid = M < sms * 8 ? M : sms * 8;
-  rotate_quant_general_kernel<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt);
+  rotate_quant_general_kernel<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp);
   return cudaGetLastError();
 }
 
@@ -430,6 +464,11 @@ cudaError_t xq_launch_relayout_from_blocks(const uint8_t* blocks, int32_t Np, in
                                            int32_t Kp, cudaStream_t st) {
   const long long work = (long long)N * (Kp / 2);
   relayout_from_blocks_kernel<<<grid_for(work, 256), 256, 0, st>>>((const uint32_t*)blocks, Np, Kpp, canon, N, Kp);
+  return cudaGetLastError();
+}
+
+cudaError_t xq_launch_weight_sums(const uint8_t* blocks, int32_t Np, int32_t Kpp, int32_t* w_sum, cudaStream_t st) {
+  weight_sums_kernel<<<(Np + 127) / 128, 128, 0, st>>>(blocks, Np, Kpp, w_sum);
   return cudaGetLastError();
 }
 

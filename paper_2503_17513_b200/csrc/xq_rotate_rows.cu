@@ -38,11 +38,11 @@ __device__ __forceinline__ void group_sync(int group, int Wr) {
   else xqptx::bar_sync(1 + group, 32 * Wr);
 }
 
-template <int LOG2N, int KS, int MTW>
+template <int LOG2N, int KS, int MTW, bool ASYM>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     rotate_quant_rows_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx, xq_hadamard_plan_t pl, float gamma,
                              uint8_t* __restrict__ Xq, float* __restrict__ sx, float* __restrict__ Yopt, uint8_t* __restrict__ A8opt,
-                             int Wr, int G, int fold) {
+                             int32_t* __restrict__ zp, int Wr, int G, int fold) {
   constexpr int n = 1 << LOG2N, NT8 = n / 8;
   constexpr int xpitch = n + 8;        // bf16 elements per staged row (conflict-free ldmatrix)
   constexpr int hpitch = KS * 16 + 8;  // bf16 elements per row of H_p^T
@@ -56,8 +56,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
   __nv_bfloat16* Xs_all = Hs + MT * 16 * hpitch;                                        // [G][2][KS * 16][xpitch]
   constexpr int tpitch = n + 8;        // floats per row of the transpose tile
   float* tr_all = reinterpret_cast<float*>(Xs_all + (size_t)G * 2 * KS * 16 * xpitch);  // [warps][8][tpitch]
-  float* red_all = tr_all + (size_t)G * Wr * 8 * tpitch;                                // [G][Wr] + 32 spare
-  int8_t* chi2 = reinterpret_cast<int8_t*>(red_all + G * Wr + 32);
+  float* red_all = tr_all + (size_t)G * Wr * 8 * tpitch;                                // [G][2 Wr] + 32 spare
+  int8_t* chi2 = reinterpret_cast<int8_t*>(red_all + 2 * G * Wr + 32);
   int8_t* sq = chi2 + 2 * q + 1;
 
   if (pl.p > 1) build_chi(q, chi2, sq);
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 
   __nv_bfloat16* Xs = Xs_all + (size_t)group * 2 * KS * 16 * xpitch;
   float* tr = tr_all + (size_t)warp * 8 * tpitch;
-  float* red = red_all + group * Wr;
+  float* red = red_all + group * 2 * Wr;
   constexpr int TPL = NT8 / 4;  // (row, j) tuples of eight columns per lane and pass of eight rows
   const int chunks = K / 8;  // 16-byte pieces of a row
   const int stride = gridDim.x * G;
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     // bits 1-2 (t): eight rows at a time through the warp's tile; afterwards fin[m][h][k][0..7] are
     // the columns 8 jj .. 8 jj + 7 of row a' = 16 (wg MTW + m) + 8 h + r, (r, jj) = tuple lane + 32 k
     float fin[MTW][2][TPL][8];
-    float amax = 0.f;
+    float amax = 0.f, amin = 0.f;  // symmetric: amax = max |y|; asymmetric: the row's extremes (both include 0)
 #pragma unroll
     for (int m = 0; m < MTW; ++m)
 #pragma unroll
@@ -179,23 +179,44 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
           f[0] = a0 + a4; f[1] = a1 + a5; f[2] = a2 + a6; f[3] = a3 + a7;
           f[4] = a0 - a4; f[5] = a1 - a5; f[6] = a2 - a6; f[7] = a3 - a7;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(f[i]));
+          for (int i = 0; i < 8; ++i) {
+            if (ASYM) {
+              amax = fmaxf(amax, f[i]);
+              amin = fminf(amin, f[i]);
+            } else {
+              amax = fmaxf(amax, fabsf(f[i]));
+            }
+          }
         }
         __syncwarp();
       }
-    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    if (Wr > 1) {
-      if (lane == 0) red[wg] = amax;
-      group_sync(group, Wr);
-      for (int i = 0; i < Wr; ++i) amax = fmaxf(amax, red[i]);
+    for (int o = 16; o > 0; o >>= 1) {
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      if (ASYM) amin = fminf(amin, __shfl_xor_sync(0xffffffffu, amin, o));
     }
-    amax *= gamma;  // the maximum of the scaled values: scaling is monotone
-    float s = amax > 0.f ? __fdiv_rn(amax, 7.f) : 1.f;
-    if (!(s > 0.f)) s = 1.f;
-    const float mult = gamma * __frcp_rn(s);
-    if (tg == 0) sx[row] = s;
+    if (Wr > 1) {
+      if (lane == 0) {
+        red[wg] = amax;
+        if (ASYM) red[Wr + wg] = amin;
+      }
+      group_sync(group, Wr);
+      for (int i = 0; i < Wr; ++i) {
+        amax = fmaxf(amax, red[i]);
+        if (ASYM) amin = fminf(amin, red[Wr + i]);
+      }
+    }
+    // the extremes of the scaled values: scaling is monotone
+    const xqhad::RowQuant rq = ASYM ? xqhad::row_quant_asym(amin * gamma, amax * gamma) : xqhad::row_quant_sym(amax * gamma);
+    const float mult = gamma * rq.inv;
+    if (tg == 0) {
+      sx[row] = rq.s;
+      if (ASYM) zp[row] = rq.z;
+    }
+    // the rounding constant 1.5 * 2^23 also carries the zero point and an offset of 8 (offset
+    // binary, undone below)
+    const float magic = 12582920.f + (float)rq.z;
     // quantize (round to nearest even through the 1.5 * 2^23 add: the low mantissa bits are the
-    // integer; |y / s| <= 7, so no clamp is needed), pack eight codes per word
+    // integer; symmetric |y / s| <= 7 needs no clamp), pack eight codes per word
     uint32_t* xq_row = reinterpret_cast<uint32_t*>(Xq + (long long)row * (Kp / 2));
 #pragma unroll
     for (int m = 0; m < MTW; ++m)
@@ -211,7 +232,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
           // nibbles become two's complement by flipping their top bits.
           uint32_t w = 0;
 #pragma unroll
-          for (int i = 7; i >= 0; --i) w = w * 16u + (uint32_t)__float_as_int(fmaf(f[i], mult, 12582920.f));
+          for (int i = 7; i >= 0; --i) {
+            float v = fmaf(f[i], mult, magic);
+            if (ASYM) v = fminf(fmaxf(v, 12582912.f), 12582927.f);  // rne(y / s) + z can leave the code range by one
+            w = w * 16u + (uint32_t)__float_as_int(v);
+          }
           w = (w - 0x4B400000u * 0x11111111u) ^ 0x88888888u;
           if (a2 < p) {
             xq_row[a2 * NT8 + jj] = w;
@@ -234,16 +259,16 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 
 template <int LOG2N, int KS, int MTW>
 cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
-                        float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+                        float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
   constexpr int n = 1 << LOG2N;
   const int fold = pl.log2n - LOG2N;  // Sylvester bits folded into the outer factor
   const int MT = ((pl.p << fold) + 15) / 16, Wr = (MT + MTW - 1) / MTW;
   int G = kMaxWarps / Wr;
   const size_t fixed = (size_t)MT * 16 * (KS * 16 + 8) * 2 + 32 * 4 + (size_t)(3 * pl.q + 1) + 64;
-  const size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 4;
+  const size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 8;
   while (G > 1 && fixed + G * per_group > 224 * 1024) --G;
   const size_t smem = fixed + G * per_group;
-  auto kern = rotate_quant_rows_kernel<LOG2N, KS, MTW>;
+  auto kern = zp ? rotate_quant_rows_kernel<LOG2N, KS, MTW, true> : rotate_quant_rows_kernel<LOG2N, KS, MTW, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int want = (M + G - 1) / G;
@@ -257,29 +282,29 @@ cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, Wr, G, fold);
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, Wr, G, fold);
 }
 
 template <int LOG2N, int MTW>
 cudaError_t launch_rows_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                           float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+                           float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
   switch (ks) {
-    case 1: return launch_rows<LOG2N, 1, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 2: return launch_rows<LOG2N, 2, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 3: return launch_rows<LOG2N, 3, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    default: return launch_rows<LOG2N, 4, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 1: return launch_rows<LOG2N, 1, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 2: return launch_rows<LOG2N, 2, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 3: return launch_rows<LOG2N, 3, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    default: return launch_rows<LOG2N, 4, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
   }
 }
 
 // n > 128 folded to 128: up to 128 staged rows
 cudaError_t launch_rows_folded(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                               float* sx, float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+                               float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
   switch (ks) {
-    case 5: return launch_rows<7, 5, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 6: return launch_rows<7, 6, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 7: return launch_rows<7, 7, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 8: return launch_rows<7, 8, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    default: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 5: return launch_rows<7, 5, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 6: return launch_rows<7, 6, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 7: return launch_rows<7, 7, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 8: return launch_rows<7, 8, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    default: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
   }
 }
 
@@ -300,15 +325,15 @@ bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
 }
 
 cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
-                                  float* Yopt, uint8_t* A8opt, int sms, cudaStream_t st) {
+                                  float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
   const int log2n = pl.log2n > 7 ? 7 : pl.log2n;
   const int n = 1 << log2n, rows_a = (pl.K + n - 1) / n, ks = (rows_a + 15) / 16;
   // tiles of 16 output rows per warp: 80 accumulator registers at n = 32, 64 at n = 64 and 128
   switch (pl.log2n) {
-    case 5: return launch_rows_ks<5, 5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 6: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    case 7: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
-    default: return launch_rows_folded(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, sms, st);
+    case 5: return launch_rows_ks<5, 5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 6: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 7: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    default: return launch_rows_folded(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
   }
 }

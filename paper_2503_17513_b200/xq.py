@@ -37,7 +37,7 @@ EXPORTS = [
     "xq_status_string", "xq_hadamard_plan", "xq_prepare_weights", "xq_weights_import", "xq_weights_export",
     "xq_weights_info", "xq_weights_free", "xq_workspace_bytes", "xq_workspace_init", "xq_rotate_quant",
     "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status", "xq_expanded_linear_static",
-    "xq_selftest_wait_timeout",
+    "xq_selftest_wait_timeout", "xq_rotate_quant_asym", "xq_w4a4_gemm_asym", "xq_expanded_linear_asym",
 ]
 
 
@@ -66,6 +66,9 @@ def lib() -> ctypes.CDLL:
         L.xq_rotate_quant.argtypes = [vp, i32, i64, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp]
         L.xq_w4a4_gemm.argtypes = [vp, vp, i32, vp, vp, vp, vp, sz, vp]
         L.xq_expanded_linear.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
+        L.xq_rotate_quant_asym.argtypes = [vp, i32, i64, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp, vp]
+        L.xq_w4a4_gemm_asym.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.xq_expanded_linear_asym.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
@@ -189,6 +192,25 @@ def xq_expanded_linear(X, w: Weights, out, ws, M=None, ldx=None, stream=None) ->
     ldx = X.stride(0) if ldx is None else ldx
     _check(lib().xq_expanded_linear(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _dp(ws),
                                     ws.numel() * ws.element_size(), _stream(stream)), "xq_expanded_linear")
+
+
+def xq_rotate_quant_asym(X, plan: HadamardPlan, Xq, s_x, zp, Y_f32=None, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_rotate_quant_asym(ctypes.c_void_p(X.data_ptr()), M, ldx, ctypes.byref(plan), _dp(Xq), _dp(s_x), _dp(zp),
+                                      _dp(Y_f32), _stream(stream)), "xq_rotate_quant_asym")
+
+
+def xq_w4a4_gemm_asym(Xq, s_x, zp, M: int, w: Weights, out, ws, acc=None, stream=None) -> None:
+    _check(lib().xq_w4a4_gemm_asym(_dp(Xq), _dp(s_x), _dp(zp), M, w.handle, _dp(out), _dp(acc), _dp(ws),
+                                   ws.numel() * ws.element_size(), _stream(stream)), "xq_w4a4_gemm_asym")
+
+
+def xq_expanded_linear_asym(X, w: Weights, out, ws, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_expanded_linear_asym(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _dp(ws),
+                                         ws.numel() * ws.element_size(), _stream(stream)), "xq_expanded_linear_asym")
 
 
 def xq_expanded_linear_host(X_host, w: Weights, out_host, ws, M=None, stream=None) -> None:
