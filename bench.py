@@ -172,10 +172,14 @@ def run_reference(args, table, layers, M, heavy):
         for name in table:
             pl, qw, sw, scale = prepared[name]
             t0 = time.perf_counter()
-            _, qx, sx = oracle.rotate_quant(pl, xs[name])
-            t1 = time.perf_counter()
-            acc = oracle.gemm_i64(qx, qw)
-            oracle.epilogue(acc, sx, sw)
+            if args.act == "asym":
+                _, ux, sx, z = oracle.rotate_quant_asym(pl, xs[name])
+                t1 = time.perf_counter()
+                oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), sx, z, sw, qw)
+            else:
+                _, qx, sx = oracle.rotate_quant(pl, xs[name])
+                t1 = time.perf_counter()
+                oracle.epilogue(oracle.gemm_i64(qx, qw), sx, sw)
             t2 = time.perf_counter()
             t_scaled += (t1 - t0) + (t2 - t1) * scale
         return t_scaled
@@ -199,7 +203,8 @@ def run_reference(args, table, layers, M, heavy):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": len(times),
         "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64/int64 (oracle)", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {','.join(table)} x {layers} layers, M={M}"},
+        "config": {"workload": f"{args.workload}: {','.join(table)} x {layers} layers, M={M}",
+                   "activations": "asymmetric per token" if args.act == "asym" else "symmetric per token"},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -216,6 +221,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--act", default="sym", choices=["sym", "asym"],
+                    help="per-token activation quantizer: symmetric (default) or asymmetric with a zero point")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -252,23 +259,34 @@ def main():
     wsp = {n: xq.new_workspace(M, Wt[n][0]) for n in names}
     Xq = {n: torch.empty((M, table[n][1] // 2), dtype=torch.uint8, device="cuda") for n in names}
     sx = {n: torch.empty((M,), dtype=torch.float32, device="cuda") for n in names}
+    zp = {n: torch.zeros((M,), dtype=torch.int32, device="cuda") for n in names}
+    asym = args.act == "asym"
     weight_bytes = sum(layers * (table[n][2] * table[n][1] // 2) for n in names)
     stream = torch.cuda.Stream()
 
     def step_linear():
         for l in range(layers):
             for n in names:
-                xq.xq_expanded_linear(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
+                if asym:
+                    xq.xq_expanded_linear_asym(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
+                else:
+                    xq.xq_expanded_linear(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
 
     def step_rotate_only():
         for l in range(layers):
             for n in names:
-                xq.xq_rotate_quant(X[n], Wt[n][l].plan, Xq[n], sx[n], stream=stream)
+                if asym:
+                    xq.xq_rotate_quant_asym(X[n], Wt[n][l].plan, Xq[n], sx[n], zp[n], stream=stream)
+                else:
+                    xq.xq_rotate_quant(X[n], Wt[n][l].plan, Xq[n], sx[n], stream=stream)
 
     def step_gemm_only():
         for l in range(layers):
             for n in names:
-                xq.xq_w4a4_gemm(Xq[n], sx[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
+                if asym:
+                    xq.xq_w4a4_gemm_asym(Xq[n], sx[n], zp[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
+                else:
+                    xq.xq_w4a4_gemm(Xq[n], sx[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
 
     def make_runner(fn):
         with torch.cuda.stream(stream):
@@ -348,7 +366,10 @@ def main():
     def step_host():
         for l in range(layers):
             for n in names:
-                xq.xq_expanded_linear_host(Xh[n], Wt[n][l], Oh[n], wsp[n], stream=stream)
+                if asym:
+                    xq.xq_expanded_linear_host_asym(Xh[n], Wt[n][l], Oh[n], wsp[n], stream=stream)
+                else:
+                    xq.xq_expanded_linear_host(Xh[n], Wt[n][l], Oh[n], wsp[n], stream=stream)
 
     e2e_steps = max(3, min(args.steps, 10))
     t_e2e = timed(step_host, e2e_steps, 3) / e2e_steps
@@ -367,13 +388,14 @@ def main():
 
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:
-        cpu_baseline = cpu_baseline_leg(table, layers, M, heavy)
+        cpu_baseline = cpu_baseline_leg(table, layers, M, heavy, asym)
 
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4 codes, int32 accumulate",
         "data": "synthetic",
         "config": {"workload": f"{args.workload}: {','.join(names)} x {layers} layers, M={M}", "tokens": M, "layers": layers,
+                   "activations": "asymmetric per token" if asym else "symmetric per token",
                    "weight_bytes": weight_bytes, "l2": "weights of one step exceed L2 (126 MB)" if weight_bytes > 126e6 else
                    "weights fit in L2", "cuda_graph": not args.no_graph, "parallelism": "replicas" if world > 1 else "single"},
         "TOPS": ops / t_step / 1e12, "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
@@ -384,7 +406,7 @@ def main():
         dist.destroy_process_group()
 
 
-def cpu_baseline_leg(table, layers, M, heavy):
+def cpu_baseline_leg(table, layers, M, heavy, asym=False):
     """The oracle, as it stands, on the host cores: online path of one layer's linears for a bounded
     token and channel sample, scaled linearly (the path is independent per token and per channel)."""
     import oracle
@@ -398,9 +420,14 @@ def cpu_baseline_leg(table, layers, M, heavy):
         x = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
         qw, sw = oracle.prepare_weights(pl, synth.weights(Ns, K, seed=0, tag=name))
         t0 = time.perf_counter()
-        _, qx, sx = oracle.rotate_quant(pl, x)
-        t1 = time.perf_counter()
-        oracle.epilogue(oracle.gemm_i64(qx, qw), sx, sw)
+        if asym:
+            _, ux, sx, z = oracle.rotate_quant_asym(pl, x)
+            t1 = time.perf_counter()
+            oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), sx, z, sw, qw)
+        else:
+            _, qx, sx = oracle.rotate_quant(pl, x)
+            t1 = time.perf_counter()
+            oracle.epilogue(oracle.gemm_i64(qx, qw), sx, sw)
         t2 = time.perf_counter()
         t_layer += (t1 - t0) + (t2 - t1) * (N / Ns)
     t_step = t_layer * layers * (M / Ms)

@@ -145,6 +145,9 @@ xq_status xq_w4a4_gemm_asym(const uint8_t* Xq_dev, const float* s_x_dev, const i
                             size_t ws_bytes, void* stream);
 xq_status xq_expanded_linear_asym(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w,
                                   void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+/* xq_expanded_linear_host (below) with asymmetric activation codes. */
+xq_status xq_expanded_linear_host_asym(const void* X_bf16_host, int32_t M, const xq_weights* w,
+                                       void* out_bf16_host, void* ws_dev, size_t ws_bytes, void* stream);
 
 /* The whole layer on HOST buffers: copies X (host, [M, K] contiguous; pinned memory makes the
  * copies asynchronous) into the workspace, runs the layer, copies out (host, bf16 [M, N]) back

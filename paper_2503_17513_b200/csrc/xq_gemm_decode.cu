@@ -319,11 +319,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   const int mine = (n_blk - rank + C - 1) / C;
   if (C > 1) cluster_arrive_release();
   float e_sx = 0.f;
+  int e_z = 0;
   float4 e_s0 = make_float4(0.f, 0.f, 0.f, 0.f), e_s1 = e_s0;
   if (warp < kConsumerWarps && tid < mine * p.M * 2) {
     const int h = tid & 1, bm = tid >> 1, jj = bm / p.M, m = bm - jj * p.M;
     const int n0 = (b0 + rank + jj * C) * 16 + 8 * h;
     e_sx = p.sx[m];
+    if (p.zp) e_z = p.zp[m];
     if (n0 + 8 <= p.N && (p.N & 7) == 0) {
       e_s0 = *reinterpret_cast<const float4*>(p.sw + n0);
       e_s1 = *reinterpret_cast<const float4*>(p.sw + n0 + 4);
@@ -336,6 +338,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       const int h = idx & 1, bm = idx >> 1;
       const int jj = bm / p.M, m = bm - jj * p.M;
       const int j = rank + jj * C;
+      const int n0 = (b0 + j) * 16 + 8 * h;
+      const bool pre = idx == tid;  // scales already in registers
+      int z = 0;
+      int4 w0 = make_int4(0, 0, 0, 0), w1 = w0;
+      if (p.zp) {  // issued ahead of the tile reads (w_sum covers the padded rows)
+        z = pre ? e_z : p.zp[m];
+        w0 = *reinterpret_cast<const int4*>(p.wsum + n0);
+        w1 = *reinterpret_cast<const int4*>(p.wsum + n0 + 4);
+      }
       const int* col = tiles + (size_t)jj * srcs * 16 * MT + (8 * h) * MT + m;
       int v[8];
 #pragma unroll
@@ -346,14 +357,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       }
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] >>= 8;  // every product carries 16 x 16
-      const int n0 = (b0 + j) * 16 + 8 * h;
-      if (p.zp) {  // sum (c - z) qw = sum c qw - z sum qw (w_sum covers the padded rows)
-        const int z = p.zp[m];
-        const int4 w0 = *reinterpret_cast<const int4*>(p.wsum + n0), w1 = *reinterpret_cast<const int4*>(p.wsum + n0 + 4);
+      if (p.zp) {  // sum (c - z) qw = sum c qw - z sum qw
         v[0] -= z * w0.x; v[1] -= z * w0.y; v[2] -= z * w0.z; v[3] -= z * w0.w;
         v[4] -= z * w1.x; v[5] -= z * w1.y; v[6] -= z * w1.z; v[7] -= z * w1.w;
       }
-      const bool pre = idx == tid;  // scales already in registers
       const float sxm = pre ? e_sx : p.sx[m];
       const size_t o = (size_t)m * p.N + n0;
       if (n0 + 8 <= p.N && (p.N & 7) == 0) {

@@ -38,6 +38,7 @@ EXPORTS = [
     "xq_weights_info", "xq_weights_free", "xq_workspace_bytes", "xq_workspace_init", "xq_rotate_quant",
     "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status", "xq_expanded_linear_static",
     "xq_selftest_wait_timeout", "xq_rotate_quant_asym", "xq_w4a4_gemm_asym", "xq_expanded_linear_asym",
+    "xq_expanded_linear_host_asym",
 ]
 
 
@@ -70,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.xq_w4a4_gemm_asym.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_asym.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
+        L.xq_expanded_linear_host_asym.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
@@ -219,6 +221,13 @@ def xq_expanded_linear_host(X_host, w: Weights, out_host, ws, M=None, stream=Non
     _check(lib().xq_expanded_linear_host(ctypes.c_void_p(X_host.data_ptr()), M, w.handle,
                                          ctypes.c_void_p(out_host.data_ptr()), _dp(ws), ws.numel() * ws.element_size(),
                                          _stream(stream)), "xq_expanded_linear_host")
+
+
+def xq_expanded_linear_host_asym(X_host, w: Weights, out_host, ws, M=None, stream=None) -> None:
+    M = X_host.shape[0] if M is None else M
+    _check(lib().xq_expanded_linear_host_asym(ctypes.c_void_p(X_host.data_ptr()), M, w.handle,
+                                              ctypes.c_void_p(out_host.data_ptr()), _dp(ws), ws.numel() * ws.element_size(),
+                                              _stream(stream)), "xq_expanded_linear_host_asym")
 
 
 def xq_expanded_linear_static(X, w: Weights, out, M=None, ldx=None, stream=None) -> None:

@@ -187,6 +187,12 @@ def test_expanded_linear_asym_end_to_end(xq, oracle, M, N, K, Kp, heavy):
     out2 = torch.empty_like(out)
     xq.xq_w4a4_gemm_asym(Xq, sx, zp, M, w, out2, ws)
     assert torch.equal(out, out2)
+    # and so does the host-buffer entry point
+    if K % 8 == 0:
+        xh = torch.from_numpy(x.view(np.int16)).pin_memory()
+        oh = torch.empty((M, N), dtype=torch.int16).pin_memory()
+        xq.xq_expanded_linear_host_asym(xh, w, oh, ws)
+        assert torch.equal(oh, out.cpu())
 
 
 def test_asym_is_closer_to_the_unquantized_product_on_shifted_rows(xq, oracle):

@@ -78,5 +78,6 @@ def test_null_arguments_rejected_before_any_cuda_call(xq):
     assert L.xq_rotate_quant_asym(null, 0, 8, ctypes.byref(pl), null, null, null, null, null) == xq.OK
     assert L.xq_w4a4_gemm_asym(null, null, null, 4, null, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_expanded_linear_asym(null, 4, 8, null, null, null, 0, null) == xq.ERR_INVALID_ARG
+    assert L.xq_expanded_linear_host_asym(null, 4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_poll_status(null, null) == xq.ERR_WORKSPACE
     L.xq_weights_free(null)  # allowed
