@@ -38,6 +38,8 @@ WORKLOADS = {
     "8b-decode": (synth.LLAMA_8B, 8, 16, False),
     "8b-prefill": (synth.LLAMA_8B, 4, 4096, True),
     "sweep": (synth.SWEEP_4096, 4, 8192, True),
+    "table1-1b-down": (synth.TABLE1_1B_DOWN, 8, 2048, True),
+    "table1-8b-down": (synth.TABLE1_8B_DOWN, 4, 4096, True),
 }
 METRIC = "expanded W4A4 linear tokens/s"
 FALLBACK_HBM_GBS = 6650.0

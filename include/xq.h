@@ -61,7 +61,8 @@ typedef struct xq_weights xq_weights;
 
 /* Factor Kp.  Host only, pure.  p is the smallest odd(Kp) * 2^j (j >= 2) that is a Paley order.
  * Errors: INVALID_ARG (out == NULL, K < 1, Kp < K, Kp odd and > 1), UNSUPPORTED_ORDER (no such
- * factor, or p above the kernels' limit of 256). */
+ * factor up to p = 8192; or p > 256, which only the general rotate kernel takes, with
+ * 8 Kp + 3 q + 256 bytes above the 227 KiB of shared memory that kernel may use). */
 xq_status xq_hadamard_plan(int32_t K, int32_t Kp, xq_hadamard_plan_t* out);
 
 /* Offline step (Sec. 3: expanded weights = truncated-Hadamard^T times W; Sec. 4: per-channel

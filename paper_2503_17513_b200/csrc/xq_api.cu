@@ -84,7 +84,7 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
     xq_weights_free(w);
     return XQ_ERR_ALLOC;
   }
-  if (pl.p > 1) {
+  if (pl.p > 1 && pl.p <= XQ_MAX_P_IMAGE) {
     // bf16 image of H_p^T (row a', column a) for the rotate kernel: a constant of the plan
     const int P16 = (pl.p + 15) / 16 * 16, pitch = P16 + 8;
     uint16_t* img = (uint16_t*)calloc((size_t)P16 * pitch, sizeof(uint16_t));
@@ -174,6 +174,8 @@ xq_status xq_hadamard_plan(int32_t K, int32_t Kp, xq_hadamard_plan_t* out) {
       }
     }
     if (!found) return XQ_ERR_UNSUPPORTED_ORDER;
+    // orders beyond the specialised kernels run in the general one: a row and its image in shared memory
+    if (pl.p > XQ_MAX_P_IMAGE && 8 * (size_t)Kp + 3 * (size_t)pl.q + 256 > 227 * 1024) return XQ_ERR_UNSUPPORTED_ORDER;
   }
   *out = pl;
   return XQ_OK;

@@ -65,7 +65,8 @@ xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
 // Size of the built-in scratch array of xq_expanded_linear_static.
 constexpr size_t XQ_STATIC_SCRATCH_BYTES = 4u << 20;
 
-constexpr int XQ_MAX_P = 256;
+constexpr int XQ_MAX_P = 8192;        // largest order-p factor (the general rotate kernel; its shared memory bounds K' too)
+constexpr int XQ_MAX_P_IMAGE = 256;   // largest p with a sign-matrix image (the kernels that read it stop there)
 constexpr int XQ_DECODE_MAX_M = 32;
 
 // Launchers (each returns the CUDA error of its launch).

@@ -428,15 +428,15 @@ inline int grid_for(long long work, int threads) {
 
 cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq,
                                    float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st) {
-  // many rows, or an order that only the multi-row-group kernel and the general kernel take
-  if ((M >= XQ_ROTATE_ROWS_MIN_M || pl.log2n > 8 || pl.p == 1) && xq_rotate_rows_supported(pl))
-    return xq_launch_rotate_rows(X, M, ldx, pl, Xq, sx, Yopt, A8opt, zp, sms, st);
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
   const int n = 1 << pl.log2n;
   const int rows_a = (pl.K + n - 1) / n;
   const int MT = (pl.p + 15) / 16;
   const bool tc = pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 8 && pl.K % 8 == 0 && rows_a <= 64 &&
                   MT * (n > 128 ? 2 : 1) <= 16;
+  // many rows, or an order that only the multi-row-group kernel and the general kernel take
+  if ((M >= XQ_ROTATE_ROWS_MIN_M || !tc) && xq_rotate_rows_supported(pl))
+    return xq_launch_rotate_rows(X, M, ldx, pl, Xq, sx, Yopt, A8opt, zp, sms, st);
   if (tc) {
     const int ks = (rows_a + 15) / 16;
     switch (pl.log2n) {

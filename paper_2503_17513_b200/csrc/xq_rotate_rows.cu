@@ -308,6 +308,18 @@ cudaError_t launch_rows_folded(int ks, const void* X, int32_t M, int64_t ldx, co
   }
 }
 
+// n = 64 with 65..128 staged rows (long inputs on a short Sylvester factor, e.g. 8192 -> 8960 = 140 x 64)
+cudaError_t launch_rows_64_long(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
+                                float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
+  switch (ks) {
+    case 5: return launch_rows<6, 5, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 6: return launch_rows<6, 6, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 7: return launch_rows<6, 7, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 8: return launch_rows<6, 8, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    default: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+  }
+}
+
 }  // namespace
 
 bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
@@ -315,8 +327,8 @@ bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
   if (pl.p == 1 && pl.log2n < 9) return false;  // small pure Sylvester orders: the general kernel
   const int log2n = pl.log2n > 7 ? 7 : pl.log2n, fold = pl.log2n - log2n;
   const int n = 1 << log2n, rows_a = (pl.K + n - 1) / n, MT = ((pl.p << fold) + 15) / 16;
-  if (rows_a > (fold ? 128 : 64) || MT > 15) return false;
-  if (fold) {  // the CTA must hold at least one row group
+  if (rows_a > ((fold || log2n == 6) ? 128 : 64) || MT > 15) return false;
+  if (rows_a > 64) {  // the CTA must hold at least one row group
     const int ks = (rows_a + 15) / 16;
     const size_t need = (size_t)MT * 16 * (ks * 16 + 8) * 2 + (size_t)2 * ks * 16 * (n + 8) * 2 + (size_t)MT * 8 * (n + 8) * 4 + 4096;
     if (need > 224 * 1024) return false;
@@ -332,7 +344,7 @@ cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const x
   // tiles of 16 output rows per warp: 80 accumulator registers at n = 32, 64 at n = 64 and 128
   switch (pl.log2n) {
     case 5: return launch_rows_ks<5, 5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 6: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 6: return launch_rows_64_long(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
     case 7: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
     default: return launch_rows_folded(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
   }

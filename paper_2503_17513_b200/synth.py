@@ -80,6 +80,19 @@ LLAMA_8B = {
     "up": (4096, 4352, 14336),
     "down": (14336, 15360, 4096),
 }
+# Down projections at the expansion sizes of the paper's Table 1 (8192 -> 2048 and 14336 -> 4096).  The two
+# largest 8B sizes (19968 = 312 x 64, 22016 = 5504 x 4) are left to the parity tests: their order-p factors
+# are beyond the tensor-core rotate kernels and would make a timing of the table a timing of the general kernel.
+TABLE1_1B_DOWN = {
+    "kp8960": (8192, 8960, 2048),
+    "kp9728": (8192, 9728, 2048),
+    "kp10240": (8192, 10240, 2048),
+    "kp12288": (8192, 12288, 2048),
+}
+TABLE1_8B_DOWN = {
+    "kp15360": (14336, 15360, 4096),
+    "kp18432": (14336, 18432, 4096),
+}
 SWEEP_4096 = {
     "kp4096": (4096, 4096, 4096),
     "kp4352": (4096, 4352, 4096),

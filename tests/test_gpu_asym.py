@@ -73,7 +73,7 @@ ROTATE_CASES = [
     (5, 100, 136), (3, 200, 240), (7, 70, 80), (2, 64, 64), (2, 8, 8), (16, 2048, 2176), (3, 8192, 8704),
     (2, 14336, 15360), (3, 4096, 4608), (3, 4096, 5120), (3, 4096, 4096), (33, 2048, 2176),
     (300, 2048, 2176), (333, 100, 160), (150, 4096, 4352), (100, 8192, 8704), (60, 14336, 15360),
-    (100, 4096, 5120), (50, 4096, 4096), (50, 8192, 12288), (64, 1000, 1024),
+    (100, 4096, 5120), (50, 4096, 4096), (50, 8192, 12288), (64, 1000, 1024), (60, 8192, 8960), (1, 14336, 19968),
 ]
 
 

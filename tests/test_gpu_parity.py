@@ -82,6 +82,10 @@ ROTATE_CASES = [
     (60, 14336, 15360), (100, 4096, 5120), (80, 5000, 5120),
     # n > 256 and pure Sylvester orders through the folded outer factor
     (50, 4096, 4096), (50, 8192, 12288), (64, 1000, 1024),
+    # the expansion sizes of Table 1: 140 x 64 (128 staged input rows), 76 x 128, 20 x 512, 36 x 512, and the two
+    # orders that only the general kernel takes (312 x 64, 5504 x 4)
+    (3, 8192, 8960), (60, 8192, 8960), (3, 8192, 9728), (60, 8192, 9728), (3, 8192, 10240), (2, 14336, 18432),
+    (60, 14336, 18432), (1, 14336, 19968), (1, 14336, 22016),
 ]
 
 
@@ -189,6 +193,8 @@ E2E_CASES = [
     (1, 512, 2048, 2176, False), (8, 512, 8192, 8704, False), (32, 256, 2048, 2176, False),
     (200, 384, 2048, 2176, True), (130, 256, 4096, 4608, True), (16, 256, 4096, 5120, False),
     (16, 256, 4096, 4096, False),
+    # Table 1 sizes
+    (8, 256, 8192, 8960, False), (64, 256, 14336, 18432, True), (4, 64, 14336, 19968, False), (2, 32, 14336, 22016, False),
 ]
 
 

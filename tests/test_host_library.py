@@ -39,14 +39,16 @@ def test_library_exports_every_declared_symbol(xq):
 
 def test_plan_matches_oracle_plan(xq, oracle):
     for K, Kp in [(2048, 2176), (8192, 8704), (4096, 4352), (14336, 15360), (4096, 4608), (4096, 5120),
-                  (4096, 4096), (8192, 8960), (8192, 9728), (8192, 12288), (100, 136), (50, 56), (1, 2)]:
+                  (4096, 4096), (8192, 8960), (8192, 9728), (8192, 10240), (8192, 12288), (14336, 18432), (14336, 19968),
+                  (14336, 22016), (100, 136), (50, 56), (1, 2)]:
         assert xq.xq_hadamard_plan(K, Kp).astuple() == tuple(oracle.plan(K, Kp).__dict__.values())
 
 
 def test_plan_errors(xq):
     for K, Kp, want in [(0, 8, xq.ERR_INVALID_ARG), (16, 8, xq.ERR_INVALID_ARG), (5, 7, xq.ERR_INVALID_ARG),
-                        (4, 6, xq.ERR_UNSUPPORTED_ORDER), (14336, 22016, xq.ERR_UNSUPPORTED_ORDER),
-                        (8192, 19968, xq.ERR_UNSUPPORTED_ORDER)]:
+                        (4, 6, xq.ERR_UNSUPPORTED_ORDER),
+                        # 39936 = 312 x 128: an order-312 factor goes to the general kernel, whose row buffers must fit shared memory
+                        (20000, 39936, xq.ERR_UNSUPPORTED_ORDER)]:
         with pytest.raises(xq.XqError) as e:
             xq.xq_hadamard_plan(K, Kp)
         assert e.value.status == want
