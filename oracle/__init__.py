@@ -29,5 +29,9 @@ from .xq_oracle import (  # noqa: F401
     prepare_weights,
     rotate_quant,
     expanded_linear,
+    rotate_heads,
+    rotate_quant_heads,
+    rotate_quant_heads_asym,
+    expanded_linear_heads,
     num_threads,
 )

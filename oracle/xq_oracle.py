@@ -272,3 +272,41 @@ def expanded_linear(pl: Plan, x_bits: np.ndarray, w_bits: np.ndarray):
     qw, s_w = prepare_weights(pl, w_bits)
     acc = gemm_i64(qx, qw)
     return epilogue(acc, s_x, s_w), acc
+
+
+# Head-wise expansion (Sec. 4 "Compute Graph Details" and Sec. 5 "Expanding R2 and R4": the rotation in
+# front of the attention output projection acts on every head separately, so expanding it grows each
+# head from head_dim to head_dim' channels).  The row is cut into `heads` blocks of pl.K channels,
+# each block goes through the rotation of the plan, the blocks are laid side by side again; the
+# quantizers then see the whole row, exactly as for a single long rotation.
+
+def rotate_heads(pl: Plan, heads: int, x_bits: np.ndarray) -> np.ndarray:
+    """x_bits: bf16 bits [rows, heads * pl.K]  ->  fp64 [rows, heads * pl.Kp]."""
+    x_bits = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    rows, cols = x_bits.shape
+    assert cols == heads * pl.K
+    y = np.empty((rows, heads * pl.Kp), dtype=np.float64)
+    for h in range(heads):
+        y[:, h * pl.Kp:(h + 1) * pl.Kp] = rotate_dense(pl, x_bits[:, h * pl.K:(h + 1) * pl.K])
+    return y
+
+
+def rotate_quant_heads(pl: Plan, heads: int, x_bits: np.ndarray):
+    """(y fp64, codes int8, scales float32): head-wise rotation, then the per-row symmetric quantizer."""
+    y = rotate_heads(pl, heads, x_bits)
+    codes, s = quantize(y)
+    return y, codes, s
+
+
+def rotate_quant_heads_asym(pl: Plan, heads: int, x_bits: np.ndarray):
+    y = rotate_heads(pl, heads, x_bits)
+    codes, s, z = quantize_asym(y)
+    return y, codes, s, z
+
+
+def expanded_linear_heads(pl: Plan, heads: int, x_bits: np.ndarray, w_bits: np.ndarray):
+    """Whole layer with the head-wise rotation on both operands: (out bf16 bits [M, N], acc int64)."""
+    _, qx, s_x = rotate_quant_heads(pl, heads, x_bits)
+    _, qw, s_w = rotate_quant_heads(pl, heads, w_bits)
+    acc = gemm_i64(qx, qw)
+    return epilogue(acc, s_x, s_w), acc

@@ -184,3 +184,46 @@ def test_factored_large_shape_energy_and_invariance(oracle):
     # one dense row of the definition as a spot check of the big index arithmetic
     yd = oracle.rotate_dense(pl, x[:1])
     assert np.linalg.norm(yd - yx[:1]) <= 1e-12 * np.linalg.norm(yd)
+
+
+# Head-wise expansion (Sec. 5 "Expanding R2 and R4"): 64 -> 72 = H_72 (Paley-I, q = 71), 64 -> 80 = H_20 (x) S_4,
+# 128 -> 144 = H_36 (x) S_4, 128 -> 160 = H_20 (x) S_8, and the unexpanded 64 -> 64.
+HEAD_PLANS = [(4, 64, 72), (3, 64, 80), (2, 128, 144), (2, 128, 160), (4, 64, 64), (5, 8, 12)]
+
+
+@pytest.mark.parametrize("heads,hd,hdp", HEAD_PLANS)
+def test_headwise_rotation_is_the_block_diagonal_matrix(oracle, heads, hd, hdp):
+    """The head-wise map is x @ kron(I_heads, H_hat): library Kronecker product and matmul."""
+    pl = oracle.plan(hd, hdp)
+    Hhat = oracle.hadamard_dense(pl, rows=hd).astype(np.float64) / np.sqrt(hdp)
+    B = np.kron(np.eye(heads), Hhat)
+    assert np.allclose(B @ B.T, np.eye(heads * hd), atol=1e-12)  # left inverse per block (Sec. 3)
+    x = synth.activations(3, heads * hd, seed=8, tag="heads")
+    xf = oracle.bf16_to_f64(x)
+    y = oracle.rotate_heads(pl, heads, x)
+    assert y.shape == (3, heads * hdp)
+    assert np.allclose(y, xf @ B, rtol=0, atol=1e-12 * np.abs(xf).max() * np.sqrt(hd))
+    # energy per head is preserved (Remark 2), so a head with a dominant channel stays inside its block
+    for h in range(heads):
+        assert np.allclose(np.linalg.norm(y[:, h * hdp:(h + 1) * hdp], axis=1),
+                           np.linalg.norm(xf[:, h * hd:(h + 1) * hd], axis=1), rtol=1e-12)
+
+
+@pytest.mark.parametrize("heads,hd,hdp", HEAD_PLANS)
+def test_headwise_rotation_invariance(oracle, heads, hd, hdp):
+    """Sec. 3 applied block by block: x W^T is unchanged when both operands get the head-wise map."""
+    pl = oracle.plan(hd, hdp)
+    x = synth.activations(4, heads * hd, seed=9, tag="hx")
+    w = synth.weights(6, heads * hd, seed=9, tag="hw")
+    ref = oracle.ref_product(x, w)
+    got = oracle.rotate_heads(pl, heads, x) @ oracle.rotate_heads(pl, heads, w).T
+    assert np.linalg.norm(got - ref) <= 1e-12 * np.linalg.norm(ref)
+
+
+def test_headwise_with_one_head_is_the_plain_rotation(oracle):
+    pl = oracle.plan(100, 136)
+    x = synth.activations(3, 100, seed=10)
+    assert np.array_equal(oracle.rotate_heads(pl, 1, x), oracle.rotate_dense(pl, x))
+    y, codes, s = oracle.rotate_quant_heads(pl, 1, x)
+    y2, codes2, s2 = oracle.rotate_quant(pl, x)
+    assert np.array_equal(codes, codes2) and np.array_equal(s, s2)
