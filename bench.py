@@ -40,6 +40,8 @@ WORKLOADS = {
     "sweep": (synth.SWEEP_4096, 4, 8192, True),
     "table1-1b-down": (synth.TABLE1_1B_DOWN, 8, 2048, True),
     "table1-8b-down": (synth.TABLE1_8B_DOWN, 4, 4096, True),
+    "heads-1b-o": (synth.HEADS_1B_O, 32, 32, False),
+    "heads-8b-o": (synth.HEADS_8B_O, 16, 16, False),
 }
 METRIC = "expanded W4A4 linear tokens/s"
 FALLBACK_HBM_GBS = 6650.0
@@ -135,7 +137,7 @@ def host_inputs(table, layers, M, heavy):
     Layers beyond the first reuse the first layer's draws rotated by whole rows (distinct memory, same
     distribution) to keep host-side generation short."""
     xs, ws = {}, {}
-    for name, (K, Kp, N) in table.items():
+    for name, (K, Kp, N, *hh) in table.items():
         xs[name] = synth.activations(M, K, seed=0, tag=name, heavy_tail=heavy)
         base = synth.weights(N, K, seed=0, tag=name)
         ws[name] = [np.roll(base, 7 * layer, axis=0) if layer else base for layer in range(layers)]
@@ -162,24 +164,25 @@ def run_reference(args, table, layers, M, heavy):
     Ms = min(M, 8)
     prepared = {}
     xs = {}
-    for name, (K, Kp, N) in table.items():
+    for name, (K, Kp, N, *hh) in table.items():
         Ns = min(N, 128)
-        pl = oracle.plan(K, Kp)
+        heads = hh[0] if hh else 1
+        pl = oracle.plan(K // heads, Kp // heads)
         xs[name] = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
-        qw, sw = oracle.prepare_weights(pl, synth.weights(Ns, K, seed=0, tag=name))
-        prepared[name] = (pl, qw, sw, N / Ns)
+        _, qw, sw = oracle.rotate_quant_heads(pl, heads, synth.weights(Ns, K, seed=0, tag=name))
+        prepared[name] = (pl, qw, sw, N / Ns, heads)
 
     def step():
         t_scaled = 0.0
         for name in table:
-            pl, qw, sw, scale = prepared[name]
+            pl, qw, sw, scale, heads = prepared[name]
             t0 = time.perf_counter()
             if args.act == "asym":
-                _, ux, sx, z = oracle.rotate_quant_asym(pl, xs[name])
+                _, ux, sx, z = oracle.rotate_quant_heads_asym(pl, heads, xs[name])
                 t1 = time.perf_counter()
                 oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), sx, z, sw, qw)
             else:
-                _, qx, sx = oracle.rotate_quant(pl, xs[name])
+                _, qx, sx = oracle.rotate_quant_heads(pl, heads, xs[name])
                 t1 = time.perf_counter()
                 oracle.epilogue(oracle.gemm_i64(qx, qw), sx, sw)
             t2 = time.perf_counter()
@@ -256,7 +259,14 @@ def main():
     xs_h, ws_h = host_inputs(table, layers, M, heavy)
     names = list(table)
     X = {n: torch.from_numpy(xs_h[n].view(np.int16)).cuda() for n in names}
-    Wt = {n: [xq.xq_prepare_weights(ws_h[n][l], table[n][1]) for l in range(layers)] for n in names}
+    heads_of = {n: (table[n][3] if len(table[n]) > 3 else 1) for n in names}
+
+    def prepare(n, l):
+        if heads_of[n] > 1:
+            return xq.xq_prepare_weights_heads(ws_h[n][l], heads_of[n], table[n][1] // heads_of[n])
+        return xq.xq_prepare_weights(ws_h[n][l], table[n][1])
+
+    Wt = {n: [prepare(n, l) for l in range(layers)] for n in names}
     out = {n: torch.empty((M, table[n][2]), dtype=torch.int16, device="cuda") for n in names}
     wsp = {n: xq.new_workspace(M, Wt[n][0]) for n in names}
     Xq = {n: torch.empty((M, table[n][1] // 2), dtype=torch.uint8, device="cuda") for n in names}
@@ -277,7 +287,9 @@ def main():
     def step_rotate_only():
         for l in range(layers):
             for n in names:
-                if asym:
+                if heads_of[n] > 1:
+                    xq.xq_rotate_quant_heads(X[n], heads_of[n], Wt[n][l].plan, Xq[n], sx[n], zp[n] if asym else None, stream=stream)
+                elif asym:
                     xq.xq_rotate_quant_asym(X[n], Wt[n][l].plan, Xq[n], sx[n], zp[n], stream=stream)
                 else:
                     xq.xq_rotate_quant(X[n], Wt[n][l].plan, Xq[n], sx[n], stream=stream)
@@ -337,7 +349,7 @@ def main():
     t_gemm = timed(make_runner(step_gemm_only), n_sub, 3) / n_sub
     launches_per_step = 2 * layers * len(names)
     hbm_peak, int8_peak, peak_kind = measured_peaks()
-    gbytes = sum(layers * gemm_bytes(M, *table[n]) for n in names)
+    gbytes = sum(layers * gemm_bytes(M, *table[n][:3]) for n in names)
     rbytes = sum(layers * rotate_bytes(M, table[n][0], table[n][1]) for n in names)
     ops = sum(layers * 2 * M * table[n][2] * table[n][1] for n in names)
     per_kernel = {"xq_w4a4_gemm": {"ms_per_step": t_gemm * 1e3, "GBps": gbytes / t_gemm / 1e9, "TOPS": ops / t_gemm / 1e12,
@@ -416,18 +428,19 @@ def cpu_baseline_leg(table, layers, M, heavy, asym=False):
     oracle.build()
     Ms = min(M, 32)
     t_layer = 0.0
-    for name, (K, Kp, N) in table.items():
+    for name, (K, Kp, N, *hh) in table.items():
         Ns = min(N, 512)
-        pl = oracle.plan(K, Kp)
+        heads = hh[0] if hh else 1
+        pl = oracle.plan(K // heads, Kp // heads)
         x = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
-        qw, sw = oracle.prepare_weights(pl, synth.weights(Ns, K, seed=0, tag=name))
+        _, qw, sw = oracle.rotate_quant_heads(pl, heads, synth.weights(Ns, K, seed=0, tag=name))
         t0 = time.perf_counter()
         if asym:
-            _, ux, sx, z = oracle.rotate_quant_asym(pl, x)
+            _, ux, sx, z = oracle.rotate_quant_heads_asym(pl, heads, x)
             t1 = time.perf_counter()
             oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), sx, z, sw, qw)
         else:
-            _, qx, sx = oracle.rotate_quant(pl, x)
+            _, qx, sx = oracle.rotate_quant_heads(pl, heads, x)
             t1 = time.perf_counter()
             oracle.epilogue(oracle.gemm_i64(qx, qw), sx, sw)
         t2 = time.perf_counter()

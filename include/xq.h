@@ -150,6 +150,27 @@ xq_status xq_expanded_linear_asym(const void* X_bf16_dev, int32_t M, int64_t ldx
 xq_status xq_expanded_linear_host_asym(const void* X_bf16_host, int32_t M, const xq_weights* w,
                                        void* out_bf16_host, void* ws_dev, size_t ws_bytes, void* stream);
 
+/* Head-wise form (Sec. 4 "Compute Graph Details", Sec. 5 "Expanding R2 and R4": the rotation in
+ * front of the attention output projection acts on every head separately, so expanding it grows
+ * every head from head_dim to head_dim_p channels).  A row is `heads` blocks of head_dim channels;
+ * every block is zero-padded to head_dim_p and multiplied by the Hadamard matrix of that order
+ * scaled 1 / sqrt(head_dim_p) (plan = xq_hadamard_plan(head_dim, head_dim_p)); the blocks stay side
+ * by side (row length heads * head_dim_p) and ONE quantizer runs over the whole row, symmetric, or
+ * asymmetric when zp_opt_dev != NULL (formats as in xq_rotate_quant / xq_rotate_quant_asym).
+ * Limits: 2 <= heads <= 128, head_dim <= 128 and a multiple of 8, head_dim_p <= 160 and a multiple
+ * of 8, heads * head_dim_p a multiple of 32; otherwise UNSUPPORTED_ORDER.  ldx >= heads * head_dim.
+ * xq_prepare_weights_heads is xq_prepare_weights with this map on the rows of W (host bf16
+ * [N, heads * head_dim]); the object then reports K = heads * head_dim, Kp = heads * head_dim_p and
+ * the plan of one head, and every xq_expanded_linear* call and xq_w4a4_gemm* call takes it as any
+ * other weights object (the layer calls run the head-wise online step).  xq_weights_heads returns
+ * the number of heads of an object (1 for xq_prepare_weights / xq_weights_import; 0 for NULL). */
+xq_status xq_rotate_quant_heads(const void* X_bf16_dev, int32_t M, int64_t ldx, int32_t heads,
+                                const xq_hadamard_plan_t* head_plan, uint8_t* Xq_dev, float* s_x_dev,
+                                int32_t* zp_opt_dev, float* Y_f32_opt_dev, void* stream);
+xq_status xq_prepare_weights_heads(const void* W_bf16_host, int32_t N, int32_t heads, int32_t head_dim,
+                                   int32_t head_dim_p, void* stream, xq_weights** out);
+int32_t xq_weights_heads(const xq_weights* w);
+
 /* The whole layer on HOST buffers: copies X (host, [M, K] contiguous; pinned memory makes the
  * copies asynchronous) into the workspace, runs the layer, copies out (host, bf16 [M, N]) back
  * and synchronizes `stream` before returning. */

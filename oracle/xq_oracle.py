@@ -287,7 +287,7 @@ def rotate_heads(pl: Plan, heads: int, x_bits: np.ndarray) -> np.ndarray:
     assert cols == heads * pl.K
     y = np.empty((rows, heads * pl.Kp), dtype=np.float64)
     for h in range(heads):
-        y[:, h * pl.Kp:(h + 1) * pl.Kp] = rotate_dense(pl, x_bits[:, h * pl.K:(h + 1) * pl.K])
+        y[:, h * pl.Kp:(h + 1) * pl.Kp] = rotate(pl, x_bits[:, h * pl.K:(h + 1) * pl.K])
     return y
 
 

@@ -54,10 +54,16 @@ struct DevBuf {  // scoped device allocation for the offline calls
   }
 };
 
-xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
+// heads == 1: one rotation K -> Kp.  heads > 1: K and Kp are the sizes of ONE head.
+xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out, int32_t heads = 1) {
   xq_hadamard_plan_t pl;
   xq_status st = xq_hadamard_plan(K, Kp, &pl);
   if (st != XQ_OK) return st;
+  if (heads > 1) {
+    if (!xq_rotate_heads_supported(pl, heads)) return XQ_ERR_UNSUPPORTED_ORDER;
+    K *= heads;
+    Kp *= heads;
+  }
   if (Kp % 8 != 0) return XQ_ERR_UNSUPPORTED_ORDER;  // the GEMM kernels read whole 8-code words
   xq_weights* w = new (std::nothrow) xq_weights();
   if (!w) return XQ_ERR_ALLOC;
@@ -67,6 +73,8 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
   w->Np = (int32_t)align_up((size_t)N, XQ_ROW_PAD);
   w->Kpp = (int32_t)align_up((size_t)Kp, XQ_K_BLOCK);
   w->plan = pl;
+  w->heads = heads;
+  w->head_signs = nullptr;
   w->packed = nullptr;
   w->s_w = nullptr;
   w->w_sum = nullptr;
@@ -84,7 +92,30 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out) {
     xq_weights_free(w);
     return XQ_ERR_ALLOC;
   }
-  if (pl.p > 1 && pl.p <= XQ_MAX_P_IMAGE) {
+  if (heads > 1) {
+    // bf16 image of the truncated head matrix, row c' = output channel, column c = input channel
+    const int d16 = (pl.K + 15) / 16 * 16, pitch = d16 + 8, n = 1 << pl.log2n;
+    const size_t elems = xq_head_image_elems(pl);
+    uint16_t* img = (uint16_t*)calloc(elems, sizeof(uint16_t));
+    if (!img) {
+      xq_weights_free(w);
+      return XQ_ERR_ALLOC;
+    }
+    for (int c2 = 0; c2 < pl.Kp; ++c2)
+      for (int c = 0; c < pl.K; ++c) {
+        int s = (__builtin_popcount((c & (n - 1)) & (c2 & (n - 1))) & 1) ? -1 : 1;
+        if (pl.p > 1) s *= host_paley_sign(pl, c >> pl.log2n, c2 >> pl.log2n);
+        img[(size_t)c2 * pitch + c] = s > 0 ? 0x3F80 : 0xBF80;
+      }
+    const bool ok = cudaMalloc((void**)&w->head_signs, elems * sizeof(uint16_t)) == cudaSuccess &&
+                    cudaMemcpy(w->head_signs, img, elems * sizeof(uint16_t), cudaMemcpyHostToDevice) == cudaSuccess;
+    free(img);
+    if (!ok) {
+      cudaGetLastError();
+      xq_weights_free(w);
+      return XQ_ERR_ALLOC;
+    }
+  } else if (pl.p > 1 && pl.p <= XQ_MAX_P_IMAGE) {
     // bf16 image of H_p^T (row a', column a) for the rotate kernel: a constant of the plan
     const int P16 = (pl.p + 15) / 16 * 16, pitch = P16 + 8;
     uint16_t* img = (uint16_t*)calloc((size_t)P16 * pitch, sizeof(uint16_t));
@@ -187,6 +218,7 @@ void xq_weights_free(xq_weights* w) {
   if (w->s_w) cudaFree(w->s_w);
   if (w->w_sum) cudaFree(w->w_sum);
   if (w->hp_signs) cudaFree(w->hp_signs);
+  if (w->head_signs) cudaFree(w->head_signs);
   delete w;
 }
 
@@ -199,13 +231,19 @@ xq_status xq_weights_info(const xq_weights* w, int32_t* N, int32_t* K, int32_t* 
   return XQ_OK;
 }
 
-xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t Kp, void* stream,
-                             xq_weights** out) {
-  if (!W_host || !out || N < 1 || K < 1 || Kp < K) return XQ_ERR_INVALID_ARG;
+}  // extern "C"
+
+namespace {
+
+// heads == 1: K -> Kp over the whole row; heads > 1: K, Kp are one head's sizes.
+xq_status prepare_impl(const void* W_host, int32_t N, int32_t heads, int32_t K, int32_t Kp, void* stream, xq_weights** out) {
+  if (!W_host || !out || N < 1 || K < 1 || Kp < K || heads < 1) return XQ_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   xq_weights* w = nullptr;
-  xq_status s = make_weights(N, K, Kp, &w);
+  xq_status s = make_weights(N, K, Kp, &w, heads);
   if (s != XQ_OK) return s;
+  K = w->K;
+  Kp = w->Kp;
   // Rows of W go through the same pad + rotate + quantize kernel as activation rows (both
   // operands receive the map v -> [v, 0] H / sqrt(K')), then into the block layout.
   const int64_t ldw = (int64_t)align_up((size_t)K, 8);
@@ -218,8 +256,7 @@ xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t K
   cudaError_t e = cudaMemcpy2DAsync(dW.p, (size_t)ldw * 2, W_host, (size_t)K * 2, (size_t)K * 2, (size_t)N,
                                     cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(w->s_w, 0, sizeof(float) * (size_t)w->Np, st);
-  if (e == cudaSuccess)
-    e = xq_launch_rotate_quant(dW.p, N, ldw, w->plan, (uint8_t*)dCanon.p, w->s_w, nullptr, nullptr, w->hp_signs, nullptr, w->sms, st);
+  if (e == cudaSuccess) e = xq_launch_rotate_for(w, dW.p, N, ldw, (uint8_t*)dCanon.p, w->s_w, nullptr, nullptr, st);
   if (e == cudaSuccess)
     e = xq_launch_relayout_to_blocks((const uint8_t*)dCanon.p, N, Kp, w->packed, w->Np, w->Kpp, st);
   if (e == cudaSuccess) e = xq_launch_weight_sums(w->packed, w->Np, w->Kpp, w->w_sum, st);
@@ -232,6 +269,22 @@ xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t K
   *out = w;
   return XQ_OK;
 }
+
+}  // namespace
+
+extern "C" {
+
+xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t Kp, void* stream, xq_weights** out) {
+  return prepare_impl(W_host, N, 1, K, Kp, stream, out);
+}
+
+xq_status xq_prepare_weights_heads(const void* W_host, int32_t N, int32_t heads, int32_t head_dim, int32_t head_dim_p,
+                                   void* stream, xq_weights** out) {
+  if (heads < 2) return XQ_ERR_INVALID_ARG;
+  return prepare_impl(W_host, N, heads, head_dim, head_dim_p, stream, out);
+}
+
+int32_t xq_weights_heads(const xq_weights* w) { return w ? w->heads : 0; }
 
 xq_status xq_weights_import(const int8_t* codes, const float* s_w, int32_t N, int32_t K, int32_t Kp,
                             void* stream, xq_weights** out) {
@@ -307,8 +360,8 @@ namespace {
 
 // asym: zp is required and receives the zero points; otherwise zp must be null.
 xq_status rotate_quant_impl(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq, float* s_x,
-                            int32_t* zp, bool asym, float* Yopt, void* stream) {
-  if (!plan || M < 0) return XQ_ERR_INVALID_ARG;
+                            int32_t* zp, bool asym, float* Yopt, void* stream, int32_t heads = 1) {
+  if (!plan || M < 0 || heads < 1) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X || !Xq || !s_x || (asym && !zp)) return XQ_ERR_INVALID_ARG;
   if (zp && (reinterpret_cast<uintptr_t>(zp) & 3u)) return XQ_ERR_INVALID_ARG;
@@ -317,16 +370,20 @@ xq_status rotate_quant_impl(const void* X, int32_t M, int64_t ldx, const xq_hada
   xq_status s = xq_hadamard_plan(plan->K, plan->Kp, &chk);
   if (s != XQ_OK) return s;
   if (memcmp(&chk, plan, sizeof(chk)) != 0) return XQ_ERR_INVALID_ARG;
-  if (ldx < plan->K || (ldx % 8) != 0) return XQ_ERR_INVALID_ARG;
+  if (ldx < (int64_t)heads * plan->K || (ldx % 8) != 0) return XQ_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(Xq) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
       (Yopt && !aligned16(Yopt)))
     return XQ_ERR_INVALID_ARG;
+  if (heads > 1 && !xq_rotate_heads_supported(*plan, heads)) return XQ_ERR_UNSUPPORTED_ORDER;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
-  if (xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, nullptr, nullptr, zp, sms, (cudaStream_t)stream) != cudaSuccess) {
+  const cudaError_t e =
+      heads > 1 ? xq_launch_rotate_heads(X, M, ldx, *plan, heads, Xq, s_x, Yopt, nullptr, nullptr, zp, sms, (cudaStream_t)stream)
+                : xq_launch_rotate_quant(X, M, ldx, *plan, Xq, s_x, Yopt, nullptr, nullptr, zp, sms, (cudaStream_t)stream);
+  if (e != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
@@ -365,7 +422,7 @@ xq_status linear_impl(const void* X, int32_t M, int64_t ldx, const xq_weights* w
   int32_t* zp = asym ? (int32_t*)(base + L.zp) : nullptr;
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + L.a8 : nullptr;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->hp_signs, zp, w->sms, st) != cudaSuccess ||
+  if (xq_launch_rotate_for(w, X, M, ldx, Xq, sx, A8, zp, st) != cudaSuccess ||
       xq_launch_gemm(Xq, sx, zp, M, w, out, nullptr, ws, L, A8 != nullptr, st) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
@@ -385,6 +442,12 @@ xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadama
 xq_status xq_rotate_quant_asym(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq,
                                float* s_x, int32_t* zp, float* Yopt, void* stream) {
   return rotate_quant_impl(X, M, ldx, plan, Xq, s_x, zp, true, Yopt, stream);
+}
+
+xq_status xq_rotate_quant_heads(const void* X, int32_t M, int64_t ldx, int32_t heads, const xq_hadamard_plan_t* head_plan,
+                                uint8_t* Xq, float* s_x, int32_t* zp_opt, float* Yopt, void* stream) {
+  if (heads < 2) return XQ_ERR_INVALID_ARG;
+  return rotate_quant_impl(X, M, ldx, head_plan, Xq, s_x, zp_opt, zp_opt != nullptr, Yopt, stream, heads);
 }
 
 xq_status xq_w4a4_gemm(const uint8_t* Xq, const float* s_x, int32_t M, const xq_weights* w, void* out,

@@ -30,12 +30,14 @@ constexpr int XQ_K_BLOCK = 128;
 constexpr int XQ_ROW_PAD = 256;
 
 struct xq_weights {
-  int32_t N, K, Kp;    // logical sizes
+  int32_t N, K, Kp;    // logical sizes (head-wise: K = heads * head_dim, Kp = heads * head_dim')
+  int32_t heads;       // 1: one rotation over the whole row (plan is K -> Kp); > 1: the plan is that of one head
   int32_t Np, Kpp;     // padded sizes (multiples of 256 and 128)
   xq_hadamard_plan_t plan;
   uint8_t* packed;     // device, Np * Kpp / 2 bytes, block layout above
   float* s_w;          // device, Np floats (padding rows hold 0)
   int32_t* w_sum;      // device, Np ints: sum of the row's codes (the zero-point term of asymmetric tokens)
+  uint16_t* head_signs;  // device, head-wise only: bf16 image of the truncated head matrix, [head_dim'][head_dim16 + 8]
   uint16_t* hp_signs;  // device, bf16 image of H_p^T for the rotate kernel ([P16][P16 + 8]); NULL when p == 1
   int device;
   int sms;             // multiprocessors of that device
@@ -82,6 +84,16 @@ cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const 
 bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl);
 cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
                                   float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st);
+// Head-wise form (the row is `heads` blocks of pl.K channels, each rotated by the plan's matrix; one
+// quantizer over the whole row).  Bimage (optional): xq_weights::head_signs.
+bool xq_rotate_heads_supported(const xq_hadamard_plan_t& pl, int32_t heads);
+size_t xq_head_image_elems(const xq_hadamard_plan_t& pl);
+cudaError_t xq_launch_rotate_heads(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, int32_t heads, uint8_t* Xq,
+                                   float* sx, float* Yopt, uint8_t* A8opt, const void* Bimage, int32_t* zp, int sms,
+                                   cudaStream_t st);
+// The online step of a layer, whichever form its weights were prepared with.
+inline cudaError_t xq_launch_rotate_for(const xq_weights* w, const void* X, int32_t M, int64_t ldx, uint8_t* Xq, float* sx,
+                                        uint8_t* A8opt, int32_t* zp, cudaStream_t st);
 constexpr int XQ_ROTATE_ROWS_MIN_M = 48;  // below this the one-CTA-per-row kernel has the shorter latency
 cudaError_t xq_launch_relayout_to_blocks(const uint8_t* canon, int32_t N, int32_t Kp, uint8_t* blocks,
                                          int32_t Np, int32_t Kpp, cudaStream_t st);
@@ -108,3 +120,10 @@ bool xq_gemm_wants_a8(int32_t M, const xq_weights* w);
 // a8_ready: the a8 region of the workspace already holds the byte-per-code tokens.
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w, void* out,
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, bool a8_ready, cudaStream_t st);
+
+inline cudaError_t xq_launch_rotate_for(const xq_weights* w, const void* X, int32_t M, int64_t ldx, uint8_t* Xq, float* sx,
+                                        uint8_t* A8opt, int32_t* zp, cudaStream_t st) {
+  if (w->heads > 1)
+    return xq_launch_rotate_heads(X, M, ldx, w->plan, w->heads, Xq, sx, nullptr, A8opt, w->head_signs, zp, w->sms, st);
+  return xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8opt, w->hp_signs, zp, w->sms, st);
+}

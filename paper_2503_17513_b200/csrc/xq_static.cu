@@ -72,7 +72,7 @@ extern "C" xq_status xq_expanded_linear_static(const void* X, int32_t M, int64_t
   L.a8 = M > XQ_DECODE_MAX_M ? off_a8 : 0;
   L.total = need;
   uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + off_a8 : nullptr;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, Xq, sx, nullptr, A8, w->hp_signs, nullptr, w->sms, st) != cudaSuccess ||
+  if (xq_launch_rotate_for(w, X, M, ldx, Xq, sx, A8, nullptr, st) != cudaSuccess ||
       xq_launch_gemm(Xq, sx, nullptr, M, w, out, nullptr, base, L, A8 != nullptr, st) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;

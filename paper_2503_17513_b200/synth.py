@@ -93,6 +93,16 @@ TABLE1_8B_DOWN = {
     "kp15360": (14336, 15360, 4096),
     "kp18432": (14336, 18432, 4096),
 }
+# Attention output projections with the head-wise rotation expanded (K, K', N, heads): 32 heads of 64 -> 72 / 80
+# channels (Llama-3.2-1B-like) and of 128 -> 144 / 160 channels (Llama-3-8B-like).
+HEADS_1B_O = {
+    "hd72": (2048, 2304, 2048, 32),
+    "hd80": (2048, 2560, 2048, 32),
+}
+HEADS_8B_O = {
+    "hd144": (4096, 4608, 4096, 32),
+    "hd160": (4096, 5120, 4096, 32),
+}
 SWEEP_4096 = {
     "kp4096": (4096, 4096, 4096),
     "kp4352": (4096, 4352, 4096),

@@ -38,7 +38,7 @@ EXPORTS = [
     "xq_weights_info", "xq_weights_free", "xq_workspace_bytes", "xq_workspace_init", "xq_rotate_quant",
     "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status", "xq_expanded_linear_static",
     "xq_selftest_wait_timeout", "xq_rotate_quant_asym", "xq_w4a4_gemm_asym", "xq_expanded_linear_asym",
-    "xq_expanded_linear_host_asym",
+    "xq_expanded_linear_host_asym", "xq_rotate_quant_heads", "xq_prepare_weights_heads", "xq_weights_heads",
 ]
 
 
@@ -72,11 +72,15 @@ def lib() -> ctypes.CDLL:
         L.xq_expanded_linear_asym.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host_asym.argtypes = [vp, i32, vp, vp, vp, sz, vp]
+        L.xq_rotate_quant_heads.argtypes = [vp, i32, i64, i32, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp, vp]
+        L.xq_prepare_weights_heads.argtypes = [vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.xq_weights_heads.argtypes = [vp]
+        L.xq_weights_heads.restype = i32
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
         for name in EXPORTS:
-            if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes"):
+            if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes", "xq_weights_heads"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -123,6 +127,7 @@ class Weights:
         _check(lib().xq_weights_info(self.handle, ctypes.byref(n), ctypes.byref(k), ctypes.byref(kp), ctypes.byref(pl)),
                "xq_weights_info")
         self.N, self.K, self.Kp, self.plan = n.value, k.value, kp.value, pl
+        self.heads = int(lib().xq_weights_heads(self.handle))
 
     def free(self):
         if self.handle:
@@ -143,6 +148,24 @@ def xq_prepare_weights(W_bf16_host: np.ndarray, Kp: int, stream=None) -> Weights
     h = ctypes.c_void_p()
     _check(lib().xq_prepare_weights(_hp(W), N, K, Kp, _stream(stream), ctypes.byref(h)), "xq_prepare_weights")
     return Weights(h.value)
+
+
+def xq_prepare_weights_heads(W_bf16_host: np.ndarray, heads: int, head_dim_p: int, stream=None) -> Weights:
+    """W: host uint16 bf16 bit patterns [N, heads * head_dim]; every head block is expanded to head_dim_p."""
+    W = np.ascontiguousarray(W_bf16_host, dtype=np.uint16)
+    N, K = W.shape
+    assert K % heads == 0
+    h = ctypes.c_void_p()
+    _check(lib().xq_prepare_weights_heads(_hp(W), N, heads, K // heads, head_dim_p, _stream(stream), ctypes.byref(h)),
+           "xq_prepare_weights_heads")
+    return Weights(h.value)
+
+
+def xq_rotate_quant_heads(X, heads: int, head_plan: HadamardPlan, Xq, s_x, zp=None, Y_f32=None, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_rotate_quant_heads(ctypes.c_void_p(X.data_ptr()), M, ldx, heads, ctypes.byref(head_plan), _dp(Xq), _dp(s_x),
+                                       _dp(zp), _dp(Y_f32), _stream(stream)), "xq_rotate_quant_heads")
 
 
 def xq_weights_import(codes_host: np.ndarray, s_w_host: np.ndarray, K: int, stream=None) -> Weights:

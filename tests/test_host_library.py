@@ -81,5 +81,11 @@ def test_null_arguments_rejected_before_any_cuda_call(xq):
     assert L.xq_w4a4_gemm_asym(null, null, null, 4, null, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_expanded_linear_asym(null, 4, 8, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_expanded_linear_host_asym(null, 4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
+    hp = xq.xq_hadamard_plan(64, 72)
+    assert L.xq_rotate_quant_heads(null, 4, 256, 4, ctypes.byref(hp), null, null, null, null, null) == xq.ERR_INVALID_ARG
+    assert L.xq_rotate_quant_heads(null, 0, 256, 4, ctypes.byref(hp), null, null, null, null, null) == xq.OK
+    assert L.xq_rotate_quant_heads(null, 0, 256, 1, ctypes.byref(hp), null, null, null, null, null) == xq.ERR_INVALID_ARG
+    assert L.xq_prepare_weights_heads(null, 4, 4, 64, 72, null, ctypes.byref(out)) == xq.ERR_INVALID_ARG
+    assert L.xq_weights_heads(null) == 0
     assert L.xq_poll_status(null, null) == xq.ERR_WORKSPACE
     L.xq_weights_free(null)  # allowed
