@@ -33,5 +33,11 @@ from .xq_oracle import (  # noqa: F401
     rotate_quant_heads,
     rotate_quant_heads_asym,
     expanded_linear_heads,
+    e2m1_value,
+    quantize_mx,
+    dequantize_mx,
+    gemm_mx,
+    rotate_quant_mx,
+    expanded_linear_mx,
     num_threads,
 )

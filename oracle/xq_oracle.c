@@ -394,3 +394,77 @@ int xqo_num_threads(void) {
   return 1;
 #endif
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * MXFP4 (Sec. 4 "Quantization Details": the OCP microscaling format, one E8M0 scale for each group
+ * of 32 elements, 4-bit E2M1 elements; the conversion rule is the OCP specification's).
+ *
+ * E2M1 code: bit 3 sign, bits 2-1 exponent, bit 0 mantissa; magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6.
+ * Group of 32 consecutive channels with largest magnitude a > 0:
+ *   shared exponent e = floor(log2(a)) - 2  (2 is the exponent of the largest E2M1 value, 6 = 1.5 * 2^2),
+ *   clamped to [-127, 127]; scale byte = e + 127; element = nearest E2M1 value to v / 2^e, ties to the
+ *   value with an even mantissa bit, magnitudes above 6 saturate to 6.
+ * A group of zeros takes e = 0 (the specification leaves it open) and all-zero codes.
+ * --------------------------------------------------------------------------------------------- */
+static const double kE2M1[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+
+static uint8_t e2m1_encode(double v) {
+  const uint8_t sign = (uint8_t)(v < 0.0 ? 8 : 0);
+  const double a = fabs(v);
+  int best = 7;
+  if (a < 6.0) {
+    /* between neighbours lo = kE2M1[i], hi = kE2M1[i + 1]: nearest, tie to the even code */
+    for (int i = 0; i < 7; ++i) {
+      if (a >= kE2M1[i] && a <= kE2M1[i + 1]) {
+        const double dl = a - kE2M1[i], dh = kE2M1[i + 1] - a;
+        best = dl < dh ? i : (dh < dl ? i + 1 : ((i & 1) ? i + 1 : i));
+        break;
+      }
+    }
+  }
+  return (uint8_t)(sign | best);
+}
+
+double xqo_e2m1_value(uint8_t code) { return (code & 8) ? -kE2M1[code & 7] : kE2M1[code & 7]; }
+
+void xqo_quantize_mx(const double *y, int64_t rows, int64_t cols, uint8_t *codes, uint8_t *scales) {
+  const int64_t groups = cols / 32;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t g = 0; g < groups; ++g) {
+      const double *v = y + r * cols + g * 32;
+      double a = 0.0;
+      for (int i = 0; i < 32; ++i)
+        if (fabs(v[i]) > a) a = fabs(v[i]);
+      int e = 0;
+      if (a > 0.0) {
+        int ex;
+        (void)frexp(a, &ex); /* a = f * 2^ex, f in [0.5, 1): floor(log2 a) = ex - 1 */
+        e = ex - 1 - 2;
+        if (e < -127) e = -127;
+        if (e > 127) e = 127;
+      }
+      scales[r * groups + g] = (uint8_t)(e + 127);
+      const double inv = ldexp(1.0, -e);
+      for (int i = 0; i < 32; ++i) codes[r * cols + g * 32 + i] = e2m1_encode(v[i] * inv);
+    }
+}
+
+/* Product of two MXFP4 matrices in fp64 (every term is exact in binary64; the sum is rounded only by
+ * fp64 addition): ref[m][n] = sum_g 2^(ex[m][g] + ew[n][g]) sum_{c in g} vx[m][c] vw[n][c]. */
+void xqo_gemm_mx(const uint8_t *cx, const uint8_t *sx, const uint8_t *cw, const uint8_t *sw, int64_t M,
+                 int64_t N, int64_t Kp, double *ref) {
+  const int64_t groups = Kp / 32;
+#pragma omp parallel for schedule(static) collapse(2)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n) {
+      double acc = 0.0;
+      for (int64_t g = 0; g < groups; ++g) {
+        double part = 0.0; /* sums of multiples of 0.25 below 32 * 36: exact */
+        for (int i = 0; i < 32; ++i)
+          part += xqo_e2m1_value(cx[m * Kp + g * 32 + i]) * xqo_e2m1_value(cw[n * Kp + g * 32 + i]);
+        acc += ldexp(part, (int)sx[m * groups + g] - 127 + (int)sw[n * groups + g] - 127);
+      }
+      ref[m * N + n] = acc;
+    }
+}

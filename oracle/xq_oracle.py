@@ -310,3 +310,60 @@ def expanded_linear_heads(pl: Plan, heads: int, x_bits: np.ndarray, w_bits: np.n
     _, qw, s_w = rotate_quant_heads(pl, heads, w_bits)
     acc = gemm_i64(qx, qw)
     return epilogue(acc, s_x, s_w), acc
+
+
+# MXFP4 (Sec. 4 "Quantization Details": OCP microscaling, an E8M0 scale per group of 32, E2M1 elements).
+
+def e2m1_value(codes: np.ndarray) -> np.ndarray:
+    """fp64 values of E2M1 codes (0..15)."""
+    lib = _load()
+    lib.xqo_e2m1_value.restype = ctypes.c_double
+    lib.xqo_e2m1_value.argtypes = [ctypes.c_uint8]
+    flat = np.asarray(codes, dtype=np.uint8).ravel()
+    return np.array([lib.xqo_e2m1_value(int(c)) for c in flat], dtype=np.float64).reshape(np.shape(codes))
+
+
+def quantize_mx(y: np.ndarray):
+    """Per group of 32 along the row: (codes uint8 [rows, cols] in 0..15, scale bytes uint8 [rows, cols / 32])."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    rows, cols = y.shape
+    assert cols % 32 == 0
+    codes = np.empty((rows, cols), dtype=np.uint8)
+    scales = np.empty((rows, cols // 32), dtype=np.uint8)
+    _load().xqo_quantize_mx(_p(y), _i64(rows), _i64(cols), _p(codes), _p(scales))
+    return codes, scales
+
+
+def dequantize_mx(codes: np.ndarray, scales: np.ndarray) -> np.ndarray:
+    lut = e2m1_value(np.arange(16, dtype=np.uint8))
+    v = lut[np.asarray(codes, dtype=np.uint8)]
+    return v * np.repeat(np.exp2(np.asarray(scales, dtype=np.float64) - 127.0), 32, axis=1)
+
+
+def gemm_mx(cx: np.ndarray, sx: np.ndarray, cw: np.ndarray, sw: np.ndarray) -> np.ndarray:
+    """fp64 product of two MXFP4 matrices (rows of cw are output channels)."""
+    cx = np.ascontiguousarray(cx, dtype=np.uint8)
+    cw = np.ascontiguousarray(cw, dtype=np.uint8)
+    sx = np.ascontiguousarray(sx, dtype=np.uint8)
+    sw = np.ascontiguousarray(sw, dtype=np.uint8)
+    M, Kp = cx.shape
+    N, Kp2 = cw.shape
+    assert Kp == Kp2 and Kp % 32 == 0 and sx.shape == (M, Kp // 32) and sw.shape == (N, Kp // 32)
+    ref = np.empty((M, N), dtype=np.float64)
+    _load().xqo_gemm_mx(_p(cx), _p(sx), _p(cw), _p(sw), _i64(M), _i64(N), _i64(Kp), _p(ref))
+    return ref
+
+
+def rotate_quant_mx(pl: Plan, x_bits: np.ndarray, heads: int = 1):
+    """(y fp64, codes, scale bytes): the online step with the MXFP4 quantizer (K' a multiple of 32)."""
+    y = rotate_heads(pl, heads, x_bits) if heads > 1 else rotate(pl, x_bits)
+    codes, s = quantize_mx(y)
+    return y, codes, s
+
+
+def expanded_linear_mx(pl: Plan, x_bits: np.ndarray, w_bits: np.ndarray, heads: int = 1):
+    """Whole layer with MXFP4 weights and activations: (out bf16 bits [M, N], fp64 product)."""
+    _, cx, sx = rotate_quant_mx(pl, x_bits, heads)
+    _, cw, sw = rotate_quant_mx(pl, w_bits, heads)
+    ref = gemm_mx(cx, sx, cw, sw)
+    return f64_to_bf16(ref), ref
