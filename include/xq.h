@@ -171,6 +171,38 @@ xq_status xq_prepare_weights_heads(const void* W_bf16_host, int32_t N, int32_t h
                                    int32_t head_dim_p, void* stream, xq_weights** out);
 int32_t xq_weights_heads(const xq_weights* w);
 
+/* MXFP4 form (Sec. 4 "Quantization Details": weights and activations in the OCP microscaling
+ * format -- an E8M0 scale for each group of 32 channels, 4-bit E2M1 elements; Sec. 5 "OCP MXFP4
+ * Results").  The rotation is the same; the quantizer works per group of 32 consecutive channels of
+ * the rotated row (K' a multiple of 32, at least 128):
+ *   e = floor(log2(max |y|)) - 2 clamped to [-127, 127] (0 for a group of zeros); scale byte e + 127;
+ *   element = the E2M1 value nearest to y / 2^e (0, 0.5, 1, 1.5, 2, 3, 4, 6 with a sign bit; ties to
+ *   the even mantissa bit; larger magnitudes saturate at 6); code = sign << 3 | exponent << 1 | mantissa.
+ * The product sums element products times 2^(e_x + e_w) per group in fp32 inside the tensor core
+ * (tcgen05.mma kind::mxf4 with block scaling) and is rounded once to bf16.
+ * Canonical formats at this boundary: codes dev [M, Kp/2] bytes (low nibble = even channel), scale
+ * bytes dev [M, Kp/32].  xq_mx_weights is opaque (device memory owned by the library);
+ * xq_mx_weights_import / _export take host arrays: import packed codes [N, Kp/2] and scales
+ * [N, Kp/32]; export one code per byte [N, Kp] and scales [N, Kp/32].  N must be a multiple of 8.
+ * xq_mx_rotate_quant needs Y_f32_dev, dev float [M, Kp]: it receives the rotated rows and is the
+ * kernel's only scratch.  Workspace: xq_mx_workspace_bytes, initialised once with xq_workspace_init;
+ * status through xq_poll_status.  Errors as for the INT4 calls. */
+typedef struct xq_mx_weights xq_mx_weights;
+xq_status xq_mx_prepare_weights(const void* W_bf16_host, int32_t N, int32_t K, int32_t Kp, void* stream,
+                                xq_mx_weights** out);
+xq_status xq_mx_weights_import(const uint8_t* codes_packed_host, const uint8_t* scales_host, int32_t N, int32_t K,
+                               int32_t Kp, void* stream, xq_mx_weights** out);
+xq_status xq_mx_weights_export(const xq_mx_weights* w, uint8_t* codes_host, uint8_t* scales_host);
+xq_status xq_mx_weights_info(const xq_mx_weights* w, int32_t* N, int32_t* K, int32_t* Kp, xq_hadamard_plan_t* plan);
+void xq_mx_weights_free(xq_mx_weights* w);
+size_t xq_mx_workspace_bytes(int32_t M_max, const xq_mx_weights* w);
+xq_status xq_mx_rotate_quant(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan,
+                             uint8_t* codes_dev, uint8_t* scales_dev, float* Y_f32_dev, void* stream);
+xq_status xq_mx_gemm(const uint8_t* codes_dev, const uint8_t* scales_dev, int32_t M, const xq_mx_weights* w,
+                     void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+xq_status xq_mx_expanded_linear(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_mx_weights* w,
+                                void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
 /* The whole layer on HOST buffers: copies X (host, [M, K] contiguous; pinned memory makes the
  * copies asynchronous) into the workspace, runs the layer, copies out (host, bf16 [M, N]) back
  * and synchronizes `stream` before returning. */

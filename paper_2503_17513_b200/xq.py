@@ -39,6 +39,8 @@ EXPORTS = [
     "xq_w4a4_gemm", "xq_expanded_linear", "xq_expanded_linear_host", "xq_poll_status", "xq_expanded_linear_static",
     "xq_selftest_wait_timeout", "xq_rotate_quant_asym", "xq_w4a4_gemm_asym", "xq_expanded_linear_asym",
     "xq_expanded_linear_host_asym", "xq_rotate_quant_heads", "xq_prepare_weights_heads", "xq_weights_heads",
+    "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
+    "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
 ]
 
 
@@ -76,11 +78,24 @@ def lib() -> ctypes.CDLL:
         L.xq_prepare_weights_heads.argtypes = [vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
         L.xq_weights_heads.argtypes = [vp]
         L.xq_weights_heads.restype = i32
+        L.xq_mx_prepare_weights.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.xq_mx_weights_import.argtypes = [vp, vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.xq_mx_weights_export.argtypes = [vp, vp, vp]
+        L.xq_mx_weights_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                         ctypes.POINTER(HadamardPlan)]
+        L.xq_mx_weights_free.argtypes = [vp]
+        L.xq_mx_weights_free.restype = None
+        L.xq_mx_workspace_bytes.argtypes = [i32, vp]
+        L.xq_mx_workspace_bytes.restype = sz
+        L.xq_mx_rotate_quant.argtypes = [vp, i32, i64, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp]
+        L.xq_mx_gemm.argtypes = [vp, vp, i32, vp, vp, vp, sz, vp]
+        L.xq_mx_expanded_linear.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
         for name in EXPORTS:
-            if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes", "xq_weights_heads"):
+            if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes", "xq_weights_heads", "xq_mx_weights_free",
+                            "xq_mx_workspace_bytes"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -269,3 +284,77 @@ def xq_selftest_wait_timeout(ws, stream=None) -> None:
 
 def xq_poll_status(ws, stream=None) -> int:
     return int(lib().xq_poll_status(_dp(ws), _stream(stream)))
+
+
+# ---- MXFP4 form ------------------------------------------------------------------------------------
+
+class MxWeights:
+    """Owner of one ``xq_mx_weights*`` (freed with the object)."""
+
+    def __init__(self, handle: int):
+        self.handle = ctypes.c_void_p(handle)
+        n, k, kp, pl = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32(), HadamardPlan()
+        _check(lib().xq_mx_weights_info(self.handle, ctypes.byref(n), ctypes.byref(k), ctypes.byref(kp), ctypes.byref(pl)),
+               "xq_mx_weights_info")
+        self.N, self.K, self.Kp, self.plan = n.value, k.value, kp.value, pl
+
+    def free(self):
+        if self.handle:
+            lib().xq_mx_weights_free(self.handle)
+            self.handle = ctypes.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def xq_mx_prepare_weights(W_bf16_host: np.ndarray, Kp: int, stream=None) -> MxWeights:
+    W = np.ascontiguousarray(W_bf16_host, dtype=np.uint16)
+    N, K = W.shape
+    h = ctypes.c_void_p()
+    _check(lib().xq_mx_prepare_weights(_hp(W), N, K, Kp, _stream(stream), ctypes.byref(h)), "xq_mx_prepare_weights")
+    return MxWeights(h.value)
+
+
+def xq_mx_weights_import(codes_packed_host: np.ndarray, scales_host: np.ndarray, K: int, stream=None) -> MxWeights:
+    codes = np.ascontiguousarray(codes_packed_host, dtype=np.uint8)
+    sc = np.ascontiguousarray(scales_host, dtype=np.uint8)
+    N, half = codes.shape
+    assert sc.shape == (N, half // 16)
+    h = ctypes.c_void_p()
+    _check(lib().xq_mx_weights_import(_hp(codes), _hp(sc), N, K, 2 * half, _stream(stream), ctypes.byref(h)), "xq_mx_weights_import")
+    return MxWeights(h.value)
+
+
+def xq_mx_weights_export(w: MxWeights):
+    codes = np.empty((w.N, w.Kp), dtype=np.uint8)
+    sc = np.empty((w.N, w.Kp // 32), dtype=np.uint8)
+    _check(lib().xq_mx_weights_export(w.handle, _hp(codes), _hp(sc)), "xq_mx_weights_export")
+    return codes, sc
+
+
+def new_mx_workspace(M_max: int, w: MxWeights, device="cuda") -> torch.Tensor:
+    ws = torch.empty(int(lib().xq_mx_workspace_bytes(M_max, w.handle)), dtype=torch.uint8, device=device)
+    xq_workspace_init(ws)
+    return ws
+
+
+def xq_mx_rotate_quant(X, plan: HadamardPlan, codes, scales, Y_f32, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_mx_rotate_quant(ctypes.c_void_p(X.data_ptr()), M, ldx, ctypes.byref(plan), _dp(codes), _dp(scales), _dp(Y_f32),
+                                    _stream(stream)), "xq_mx_rotate_quant")
+
+
+def xq_mx_gemm(codes, scales, M: int, w: MxWeights, out, ws, stream=None) -> None:
+    _check(lib().xq_mx_gemm(_dp(codes), _dp(scales), M, w.handle, _dp(out), _dp(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "xq_mx_gemm")
+
+
+def xq_mx_expanded_linear(X, w: MxWeights, out, ws, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_mx_expanded_linear(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _dp(ws),
+                                       ws.numel() * ws.element_size(), _stream(stream)), "xq_mx_expanded_linear")

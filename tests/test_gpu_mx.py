@@ -1,0 +1,172 @@
+"""GPU parity of the MXFP4 form (paper Sec. 4 "Quantization Details": OCP microscaling, an E8M0 scale
+per group of 32 channels, E2M1 elements) against the CPU oracle, through the C ABI.
+
+Bounds: rotated values rel-L2 <= 1e-5; scale bytes and codes equal to the oracle's except where the
+fp32 rotation puts a value across a rounding or power-of-two boundary (<= 0.01 % of codes, then the
+two dequantized values are neighbours on the group's grid); given identical codes and scales the
+product equals the exact one up to fp32 accumulation (rel-L2 <= 1e-5 before the bf16 rounding, i.e.
+bf16 outputs within one ulp); end to end rel-L2 <= 2e-2.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2503_17513_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+ROT_REL_L2 = 1e-5
+CODE_MISMATCH_FRAC = 1e-4
+E2E_REL_L2 = 2e-2
+
+
+@pytest.fixture(scope="module")
+def xq():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2503_17513_b200 import xq as binding
+
+    binding.lib()  # fails loudly if the CUDA library is missing
+    return binding
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda()
+    return torch.from_numpy(a).cuda()
+
+
+def host_u16(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().view(torch.int16).numpy().view(np.uint16)
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    d = np.linalg.norm(b)
+    return np.linalg.norm(a - b) / (d if d > 0 else 1.0)
+
+
+def unpack(packed):
+    out = np.empty((packed.shape[0], packed.shape[1] * 2), dtype=np.uint8)
+    out[:, 0::2] = packed & 0xF
+    out[:, 1::2] = packed >> 4
+    return out
+
+
+def pack(codes):
+    return (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)
+
+
+def check_quantized(oracle, codes, sc, codes_ref, sc_ref):
+    """Equal up to boundary effects: few differing entries, and those decode to neighbouring values."""
+    assert np.count_nonzero(sc != sc_ref) / sc.size <= CODE_MISMATCH_FRAC
+    same_scale = np.repeat(sc == sc_ref, 32, axis=1)
+    differ = (codes != codes_ref) & same_scale
+    assert np.count_nonzero(differ) / codes.size <= CODE_MISMATCH_FRAC
+    lut = oracle.e2m1_value(np.arange(16, dtype=np.uint8))
+    grid = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+    a, b = np.abs(lut[codes[differ]]), np.abs(lut[codes_ref[differ]])
+    ia, ib = np.searchsorted(grid, a), np.searchsorted(grid, b)
+    assert np.all(np.abs(ia - ib) <= 1)
+
+
+ROTATE_CASES = [(5, 100, 160), (3, 200, 256), (16, 2048, 2176), (3, 8192, 8704), (2, 14336, 15360), (3, 4096, 4096),
+                (300, 2048, 2176), (100, 8192, 8704), (60, 4096, 5120)]
+
+
+@pytest.mark.parametrize("M,K,Kp", ROTATE_CASES)
+def test_mx_rotate_quant_stage_parity(xq, oracle, M, K, Kp):
+    x = synth.activations(M, K, seed=15, tag=f"mx{K}", heavy_tail=(M > 8))
+    pl = xq.xq_hadamard_plan(K, Kp)
+    ldx = (K + 7) // 8 * 8
+    X = torch.zeros((M, ldx), dtype=torch.int16, device="cuda")
+    X[:, :K] = dev(x)
+    codes = torch.empty((M, Kp // 2), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((M, Kp // 32), dtype=torch.uint8, device="cuda")
+    Y = torch.empty((M, Kp), dtype=torch.float32, device="cuda")
+    xq.xq_mx_rotate_quant(X, pl, codes, sc, Y, M=M, ldx=ldx)
+    torch.cuda.synchronize()
+    y_ref, codes_ref, sc_ref = oracle.rotate_quant_mx(oracle.plan(K, Kp), x)
+    assert rel_l2(Y.cpu().numpy(), y_ref) <= ROT_REL_L2
+    check_quantized(oracle, unpack(codes.cpu().numpy()), sc.cpu().numpy(), codes_ref, sc_ref)
+
+
+GEMM_CASES = [
+    # (M, N, K, Kp): one tile with a K tail inside the 256-code block, ragged token and channel tails, several tiles per CTA
+    (5, 8, 100, 160), (33, 256, 64, 128), (1, 2048, 2048, 2176), (130, 264, 2048, 2176), (300, 512, 4096, 4608),
+    (129, 1000, 200, 256), (2048, 2048, 2048, 2176), (16, 512, 8192, 8704),
+]
+
+
+@pytest.mark.parametrize("M,N,K,Kp", GEMM_CASES)
+def test_mx_gemm_given_codes(xq, oracle, M, N, K, Kp):
+    """Random codes and a different random scale for every (row, group): any misplaced scale byte shows."""
+    g = np.random.default_rng(1000 * M + N)
+    cx = g.integers(0, 16, size=(M, Kp)).astype(np.uint8)
+    cw = g.integers(0, 16, size=(N, Kp)).astype(np.uint8)
+    sx = g.integers(115, 140, size=(M, Kp // 32)).astype(np.uint8)
+    sw = g.integers(115, 140, size=(N, Kp // 32)).astype(np.uint8)
+    w = xq.xq_mx_weights_import(pack(cw), sw, K)
+    codes_back, sc_back = xq.xq_mx_weights_export(w)
+    assert np.array_equal(codes_back, cw) and np.array_equal(sc_back, sw)
+    ws = xq.new_mx_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    xq.xq_mx_gemm(dev(pack(cx)), dev(sx), M, w, out, ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    ref = oracle.gemm_mx(cx, sx, cw, sw)
+    got = synth.bf16_bits_to_f32(host_u16(out)).astype(np.float64)
+    want = synth.bf16_bits_to_f32(oracle.f64_to_bf16(ref)).astype(np.float64)
+    assert rel_l2(got, ref) <= 3e-3            # bf16 rounding of the outputs
+    assert rel_l2(got, want) <= 1e-3           # against the one-rounding result: fp32 accumulation only
+    rms = np.sqrt(np.mean(ref**2))
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0**-7 + 1e-4 * rms)
+    # a second call on the same workspace gives the same bits
+    out2 = torch.empty_like(out)
+    xq.xq_mx_gemm(dev(pack(cx)), dev(sx), M, w, out2, ws)
+    assert torch.equal(out, out2)
+
+
+def test_mx_prepare_weights_parity(xq, oracle):
+    N, K, Kp = 264, 2048, 2176
+    wb = synth.weights(N, K, seed=16, tag="mxw")
+    w = xq.xq_mx_prepare_weights(wb, Kp)
+    assert (w.N, w.K, w.Kp) == (N, K, Kp)
+    codes, sc = xq.xq_mx_weights_export(w)
+    _, codes_ref, sc_ref = oracle.rotate_quant_mx(oracle.plan(K, Kp), wb)
+    check_quantized(oracle, codes, sc, codes_ref, sc_ref)
+
+
+E2E_CASES = [
+    # (M, N, K, Kp, heavy)
+    (4, 24, 100, 160, False), (16, 2048, 2048, 2176, False), (1, 512, 2048, 2176, False), (8, 512, 8192, 8704, False),
+    (200, 384, 2048, 2176, True), (130, 256, 4096, 4608, True), (300, 256, 14336, 15360, True),
+]
+
+
+@pytest.mark.parametrize("M,N,K,Kp,heavy", E2E_CASES)
+def test_mx_expanded_linear_end_to_end(xq, oracle, M, N, K, Kp, heavy):
+    x = synth.activations(M, K, seed=17, tag=f"me{M}", heavy_tail=heavy)
+    wb = synth.weights(N, K, seed=17, tag=f"me{N}")
+    w = xq.xq_mx_prepare_weights(wb, Kp)
+    ws = xq.new_mx_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    ldx = (K + 7) // 8 * 8
+    X = torch.zeros((M, ldx), dtype=torch.int16, device="cuda")
+    X[:, :K] = dev(x)
+    xq.xq_mx_expanded_linear(X, w, out, ws, M=M, ldx=ldx)
+    assert xq.xq_poll_status(ws) == xq.OK
+    out_ref, _ = oracle.expanded_linear_mx(oracle.plan(K, Kp), x, wb)
+    got = synth.bf16_bits_to_f32(host_u16(out))
+    want = synth.bf16_bits_to_f32(out_ref)
+    assert rel_l2(got, want) <= E2E_REL_L2
+    for m in range(M):
+        assert rel_l2(got[m], want[m]) <= E2E_REL_L2
+
+
+def test_mx_argument_errors(xq):
+    with pytest.raises(xq.XqError) as e:  # K' = 136 is not a whole number of 32-channel groups
+        xq.xq_mx_prepare_weights(np.zeros((8, 100), np.uint16), 136)
+    assert e.value.status == xq.ERR_UNSUPPORTED_ORDER
+    with pytest.raises(xq.XqError) as e:  # N must be a multiple of 8
+        xq.xq_mx_prepare_weights(np.zeros((5, 100), np.uint16), 160)
+    assert e.value.status == xq.ERR_UNSUPPORTED_ORDER

@@ -87,5 +87,14 @@ def test_null_arguments_rejected_before_any_cuda_call(xq):
     assert L.xq_rotate_quant_heads(null, 0, 256, 1, ctypes.byref(hp), null, null, null, null, null) == xq.ERR_INVALID_ARG
     assert L.xq_prepare_weights_heads(null, 4, 4, 64, 72, null, ctypes.byref(out)) == xq.ERR_INVALID_ARG
     assert L.xq_weights_heads(null) == 0
+    assert L.xq_mx_prepare_weights(null, 8, 100, 160, null, ctypes.byref(out)) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_weights_import(null, null, 8, 100, 160, null, ctypes.byref(out)) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_weights_export(null, null, null) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_weights_info(null, None, None, None, None) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_workspace_bytes(4, null) == 0
+    assert L.xq_mx_rotate_quant(null, 4, 104, ctypes.byref(pl), null, null, null, null) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_gemm(null, null, 4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_expanded_linear(null, 4, 104, null, null, null, 0, null) == xq.ERR_INVALID_ARG
+    L.xq_mx_weights_free(null)
     assert L.xq_poll_status(null, null) == xq.ERR_WORKSPACE
     L.xq_weights_free(null)  # allowed
