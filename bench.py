@@ -169,7 +169,11 @@ def run_reference(args, table, layers, M, heavy):
         heads = hh[0] if hh else 1
         pl = oracle.plan(K // heads, Kp // heads)
         xs[name] = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
-        _, qw, sw = oracle.rotate_quant_heads(pl, heads, synth.weights(Ns, K, seed=0, tag=name))
+        wsample = synth.weights(Ns, K, seed=0, tag=name)
+        if args.fmt == "mxfp4":
+            _, qw, sw = oracle.rotate_quant_mx(pl, wsample)
+        else:
+            _, qw, sw = oracle.rotate_quant_heads(pl, heads, wsample)
         prepared[name] = (pl, qw, sw, N / Ns, heads)
 
     def step():
@@ -177,7 +181,11 @@ def run_reference(args, table, layers, M, heavy):
         for name in table:
             pl, qw, sw, scale, heads = prepared[name]
             t0 = time.perf_counter()
-            if args.act == "asym":
+            if args.fmt == "mxfp4":
+                _, cx, sx = oracle.rotate_quant_mx(pl, xs[name])
+                t1 = time.perf_counter()
+                oracle.f64_to_bf16(oracle.gemm_mx(cx, sx, qw, sw))
+            elif args.act == "asym":
                 _, ux, sx, z = oracle.rotate_quant_heads_asym(pl, heads, xs[name])
                 t1 = time.perf_counter()
                 oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), sx, z, sw, qw)
@@ -209,7 +217,8 @@ def run_reference(args, table, layers, M, heavy):
         "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64/int64 (oracle)", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {','.join(table)} x {layers} layers, M={M}",
-                   "activations": "asymmetric per token" if args.act == "asym" else "symmetric per token"},
+                   "activations": "mxfp4 groups of 32" if args.fmt == "mxfp4" else
+                   ("asymmetric per token" if args.act == "asym" else "symmetric per token")},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -226,6 +235,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fmt", default="int4", choices=["int4", "mxfp4"],
+                    help="number format of weights and activations: INT4 with per-row scales (default) or MXFP4")
     ap.add_argument("--act", default="sym", choices=["sym", "asym"],
                     help="per-token activation quantizer: symmetric (default) or asymmetric with a zero point")
     args = ap.parse_args()
@@ -261,14 +272,23 @@ def main():
     X = {n: torch.from_numpy(xs_h[n].view(np.int16)).cuda() for n in names}
     heads_of = {n: (table[n][3] if len(table[n]) > 3 else 1) for n in names}
 
+    mx = args.fmt == "mxfp4"
+    if mx:
+        assert all(h == 1 for h in heads_of.values()) and args.act == "sym", "--fmt mxfp4 runs the single-rotation symmetric path"
+
     def prepare(n, l):
+        if mx:
+            return xq.xq_mx_prepare_weights(ws_h[n][l], table[n][1])
         if heads_of[n] > 1:
             return xq.xq_prepare_weights_heads(ws_h[n][l], heads_of[n], table[n][1] // heads_of[n])
         return xq.xq_prepare_weights(ws_h[n][l], table[n][1])
 
     Wt = {n: [prepare(n, l) for l in range(layers)] for n in names}
     out = {n: torch.empty((M, table[n][2]), dtype=torch.int16, device="cuda") for n in names}
-    wsp = {n: xq.new_workspace(M, Wt[n][0]) for n in names}
+    wsp = {n: (xq.new_mx_workspace(M, Wt[n][0]) if mx else xq.new_workspace(M, Wt[n][0])) for n in names}
+    if mx:
+        mx_sc = {n: torch.empty((M, table[n][1] // 32), dtype=torch.uint8, device="cuda") for n in names}
+        mx_y = {n: torch.empty((M, table[n][1]), dtype=torch.float32, device="cuda") for n in names}
     Xq = {n: torch.empty((M, table[n][1] // 2), dtype=torch.uint8, device="cuda") for n in names}
     sx = {n: torch.empty((M,), dtype=torch.float32, device="cuda") for n in names}
     zp = {n: torch.zeros((M,), dtype=torch.int32, device="cuda") for n in names}
@@ -279,7 +299,9 @@ def main():
     def step_linear():
         for l in range(layers):
             for n in names:
-                if asym:
+                if mx:
+                    xq.xq_mx_expanded_linear(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
+                elif asym:
                     xq.xq_expanded_linear_asym(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
                 else:
                     xq.xq_expanded_linear(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
@@ -287,7 +309,9 @@ def main():
     def step_rotate_only():
         for l in range(layers):
             for n in names:
-                if heads_of[n] > 1:
+                if mx:
+                    xq.xq_mx_rotate_quant(X[n], Wt[n][l].plan, Xq[n], mx_sc[n], mx_y[n], stream=stream)
+                elif heads_of[n] > 1:
                     xq.xq_rotate_quant_heads(X[n], heads_of[n], Wt[n][l].plan, Xq[n], sx[n], zp[n] if asym else None, stream=stream)
                 elif asym:
                     xq.xq_rotate_quant_asym(X[n], Wt[n][l].plan, Xq[n], sx[n], zp[n], stream=stream)
@@ -297,7 +321,9 @@ def main():
     def step_gemm_only():
         for l in range(layers):
             for n in names:
-                if asym:
+                if mx:
+                    xq.xq_mx_gemm(Xq[n], mx_sc[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
+                elif asym:
                     xq.xq_w4a4_gemm_asym(Xq[n], sx[n], zp[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
                 else:
                     xq.xq_w4a4_gemm(Xq[n], sx[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
@@ -347,8 +373,13 @@ def main():
     n_sub = max(3, min(args.steps, 20))
     t_rot = timed(make_runner(step_rotate_only), n_sub, 3) / n_sub
     t_gemm = timed(make_runner(step_gemm_only), n_sub, 3) / n_sub
-    launches_per_step = 2 * layers * len(names)
+    launches_per_step = (3 if mx else 2) * layers * len(names)  # MXFP4: rotate, group quantizer, GEMM
     hbm_peak, int8_peak, peak_kind = measured_peaks()
+    tensor_peak, tensor_note = int8_peak, ": 2 x sustained bf16 GEMM"
+    gemm_name = "xq_w4a4_gemm (gemm_prefill_kernel)"
+    if mx:
+        tensor_peak, tensor_note = 2.0 * int8_peak, ": 4 x sustained bf16 GEMM (FP4 : bf16 nominal ratio)"
+        gemm_name = "xq_mx_gemm (gemm_mx_kernel, tcgen05.mma kind::mxf4)"
     gbytes = sum(layers * gemm_bytes(M, *table[n][:3]) for n in names)
     rbytes = sum(layers * rotate_bytes(M, table[n][0], table[n][1]) for n in names)
     ops = sum(layers * 2 * M * table[n][2] * table[n][1] for n in names)
@@ -359,16 +390,16 @@ def main():
     if M > 32 and t_gemm >= t_rot:
         # dense contraction: the tensor roofline of its own dtype
         achieved = ops / t_gemm / 1e12
-        roofline = {"bound": "tensor", "kernel": "xq_w4a4_gemm (gemm_prefill_kernel)", "achieved": achieved, "peak": int8_peak,
-                    "unit": "TOP/s", "frac": achieved / int8_peak, "peak_source": peak_kind + ": 2 x sustained bf16 GEMM",
+        roofline = {"bound": "tensor", "kernel": gemm_name, "achieved": achieved, "peak": tensor_peak,
+                    "unit": "TOP/s", "frac": achieved / tensor_peak, "peak_source": peak_kind + tensor_note,
                     "traffic": None, "per_kernel": per_kernel}
     else:
         if t_gemm >= t_rot:
-            dom, dbytes, dt = "xq_w4a4_gemm (gemm_decode_kernel)", gbytes, t_gemm
+            dom, dbytes, dt = ("xq_mx_gemm (gemm_mx_kernel)" if mx else "xq_w4a4_gemm (gemm_decode_kernel)"), gbytes, t_gemm
         else:
             dom, dbytes, dt = "xq_rotate_quant (rotate_quant_tc_kernel)", rbytes, t_rot
         achieved = dbytes / dt / 1e9
-        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.workload, M)) if dom.startswith("xq_w4a4_gemm") else None
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.workload, M)) if dom.startswith("xq_w4a4_gemm") and not asym else None
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
                     "peak_source": peak_kind, "traffic": traffic, "traffic_unit": "bytes per launch (ncu)",
                     "algorithmic_bytes_per_launch": dbytes / (layers * len(names)), "per_kernel": per_kernel}
@@ -380,7 +411,9 @@ def main():
     def step_host():
         for l in range(layers):
             for n in names:
-                if asym:
+                if mx:
+                    xq.xq_mx_expanded_linear_host(Xh[n], Wt[n][l], Oh[n], wsp[n], stream=stream)
+                elif asym:
                     xq.xq_expanded_linear_host_asym(Xh[n], Wt[n][l], Oh[n], wsp[n], stream=stream)
                 else:
                     xq.xq_expanded_linear_host(Xh[n], Wt[n][l], Oh[n], wsp[n], stream=stream)
@@ -402,14 +435,15 @@ def main():
 
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:
-        cpu_baseline = cpu_baseline_leg(table, layers, M, heavy, asym)
+        cpu_baseline = cpu_baseline_leg(table, layers, M, heavy, asym, mx)
 
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4 codes, int32 accumulate",
+        "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "mxfp4 (e2m1 codes, e8m0 group scales), fp32 accumulate" if mx else "int4 codes, int32 accumulate",
         "data": "synthetic",
         "config": {"workload": f"{args.workload}: {','.join(names)} x {layers} layers, M={M}", "tokens": M, "layers": layers,
-                   "activations": "asymmetric per token" if asym else "symmetric per token",
+                   "activations": "mxfp4 groups of 32" if mx else ("asymmetric per token" if asym else "symmetric per token"),
                    "weight_bytes": weight_bytes, "l2": "weights of one step exceed L2 (126 MB)" if weight_bytes > 126e6 else
                    "weights fit in L2", "cuda_graph": not args.no_graph, "parallelism": "replicas" if world > 1 else "single"},
         "TOPS": ops / t_step / 1e12, "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
@@ -420,7 +454,7 @@ def main():
         dist.destroy_process_group()
 
 
-def cpu_baseline_leg(table, layers, M, heavy, asym=False):
+def cpu_baseline_leg(table, layers, M, heavy, asym=False, mx=False):
     """The oracle, as it stands, on the host cores: online path of one layer's linears for a bounded
     token and channel sample, scaled linearly (the path is independent per token and per channel)."""
     import oracle
@@ -433,9 +467,17 @@ def cpu_baseline_leg(table, layers, M, heavy, asym=False):
         heads = hh[0] if hh else 1
         pl = oracle.plan(K // heads, Kp // heads)
         x = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
-        _, qw, sw = oracle.rotate_quant_heads(pl, heads, synth.weights(Ns, K, seed=0, tag=name))
+        wsample = synth.weights(Ns, K, seed=0, tag=name)
+        if mx:
+            _, cw, sw = oracle.rotate_quant_mx(pl, wsample)
+        else:
+            _, qw, sw = oracle.rotate_quant_heads(pl, heads, wsample)
         t0 = time.perf_counter()
-        if asym:
+        if mx:
+            _, cx, sx = oracle.rotate_quant_mx(pl, x)
+            t1 = time.perf_counter()
+            oracle.f64_to_bf16(oracle.gemm_mx(cx, sx, cw, sw))
+        elif asym:
             _, ux, sx, z = oracle.rotate_quant_heads_asym(pl, heads, x)
             t1 = time.perf_counter()
             oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), sx, z, sw, qw)

@@ -202,6 +202,10 @@ xq_status xq_mx_gemm(const uint8_t* codes_dev, const uint8_t* scales_dev, int32_
                      void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
 xq_status xq_mx_expanded_linear(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_mx_weights* w,
                                 void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+/* Host buffers (X [M, K] contiguous, K a multiple of 8; out bf16 [M, N]): copies in, runs the layer, copies out,
+ * synchronizes `stream`. */
+xq_status xq_mx_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_mx_weights* w, void* out_bf16_host,
+                                     void* ws_dev, size_t ws_bytes, void* stream);
 
 /* The whole layer on HOST buffers: copies X (host, [M, K] contiguous; pinned memory makes the
  * copies asynchronous) into the workspace, runs the layer, copies out (host, bf16 [M, N]) back

@@ -94,6 +94,28 @@ __device__ __forceinline__ int row_code(const RowQuant& r, float y) {
   return max(-8, min(7, __float2int_rn(y * r.inv) + r.z));
 }
 
+// MXFP4 element (paper Sec. 4: OCP microscaling): the E2M1 code nearest to v, ties to the even mantissa
+// bit, magnitudes above 6 saturate; code = sign << 3 | magnitude index of {0, .5, 1, 1.5, 2, 3, 4, 6}.
+// Below 1 the grid is the subnormal one (step 0.5): index = rne(2 a).  From 1 on, a is rounded to one
+// mantissa bit in its bit pattern (round to nearest even on bit 22, carrying into the exponent) and
+// the index is 2 (exponent - 127) + mantissa bit + 2 = (bits >> 22) - 252.
+__device__ __forceinline__ uint32_t mx_e2m1_code(float v) {
+  const float a = fabsf(v);
+  uint32_t u = __float_as_uint(a);
+  u += 0x1FFFFFu + ((u >> 22) & 1u);
+  const uint32_t hi = min((u >> 22) - 252u, 7u);
+  const uint32_t c = a < 1.f ? (uint32_t)__float2int_rn(a + a) : hi;
+  return c | (v < 0.f ? 8u : 0u);  // a negative zero keeps the code of zero
+}
+// 2^-e as a float, e in [-127, 127] (2^-127 is a subnormal: it has no exponent field of its own).
+__device__ __forceinline__ float mx_inv_scale(int e) { return e < 127 ? __uint_as_float((uint32_t)(127 - e) << 23) : 5.877471754111438e-39f; }
+// Shared exponent of a group whose largest magnitude is a: floor(log2 a) - 2 in [-127, 127]; 0 for a = 0.
+__device__ __forceinline__ int mx_shared_exp(float a) {
+  if (!(a > 0.f)) return 0;
+  const int field = (int)((__float_as_uint(a) >> 23) & 0xFF);
+  return max(-127, min(127, (field == 0 ? -127 : field - 127) - 2));  // fp32 subnormals lie below 2^-126
+}
+
 __device__ __forceinline__ uint32_t sign_bf16(int s) { return s > 0 ? 0x3F80u : (s < 0 ? 0xBF80u : 0u); }
 
 }  // namespace xqhad

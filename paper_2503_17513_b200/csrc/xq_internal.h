@@ -71,6 +71,22 @@ constexpr int XQ_MAX_P = 8192;        // largest order-p factor (the general rot
 constexpr int XQ_MAX_P_IMAGE = 256;   // largest p with a sign-matrix image (the kernels that read it stop there)
 constexpr int XQ_DECODE_MAX_M = 32;
 
+// MXFP4 outputs of the online step in the layout the block-scaled GEMM reads: codes [rows][Kq / 2]
+// bytes (Kq = K' rounded up to 256, padding zero), scale bytes in 512-byte blocks of 128 rows x 4
+// groups: byte of (row m, group g) at xq_mx_sf_offset.
+struct xq_mx_out {
+  uint8_t* codes;
+  uint8_t* sf_blocks;
+  int32_t Kq;
+};
+__host__ __device__ inline size_t xq_mx_sf_offset(int m, int g, int Kq) {
+  return ((size_t)(m >> 7) * (Kq >> 7) + (g >> 2)) * 512 + (size_t)(m & 31) * 16 + (size_t)((m >> 5) & 3) * 4 + (g & 3);
+}
+// True when xq_launch_rotate_mx can emit them directly (otherwise the caller quantizes the fp32 rows).
+bool xq_rotate_mx_supported(const xq_hadamard_plan_t& pl);
+cudaError_t xq_launch_rotate_mx(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, const xq_mx_out& mx, int sms,
+                                cudaStream_t st);
+
 // Launchers (each returns the CUDA error of its launch).
 // A8opt (optional): byte-per-code copy of the codes in the operand format of the tcgen05 GEMM, [M, Kp].
 // Hsigns (optional): device image of H_p^T as bf16, [P16][P16 + 8] with P16 = p rounded up to 16

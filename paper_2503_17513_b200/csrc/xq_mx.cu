@@ -22,6 +22,7 @@
 
 #include <new>
 
+#include "xq_hadamard.cuh"
 #include "xq_internal.h"
 #include "xq_ptx.cuh"
 
@@ -42,9 +43,7 @@ namespace {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-__host__ __device__ inline size_t sf_offset(int m, int g, int Kq) {
-  return ((size_t)(m >> 7) * (Kq >> 7) + (g >> 2)) * 512 + (size_t)(m & 31) * 16 + (size_t)((m >> 5) & 3) * 4 + (g & 3);
-}
+__host__ __device__ inline size_t sf_offset(int m, int g, int Kq) { return xq_mx_sf_offset(m, g, Kq); }
 inline size_t sf_bytes(int rows, int Kq) { return (size_t)((rows + 127) / 128) * (Kq / 128) * 512; }
 
 // ---------------------------------------------------------------------------------------------
@@ -53,11 +52,6 @@ inline size_t sf_bytes(int rows, int Kq) { return (size_t)((rows + 127) / 128) *
 //   element = nearest E2M1 value to v / 2^e, ties to the even mantissa bit, saturating at 6.
 // Groups past K' (padding up to Kq) get zero codes.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t e2m1_code(float v) {
-  const float a = fabsf(v);
-  uint32_t c = a <= 0.25f ? 0u : a < 0.75f ? 1u : a <= 1.25f ? 2u : a < 1.75f ? 3u : a <= 2.5f ? 4u : a < 3.5f ? 5u : a <= 5.0f ? 6u : 7u;
-  return c | (v < 0.f ? 8u : 0u);
-}
 
 __global__ void __launch_bounds__(256) mx_quantize_kernel(const float* __restrict__ Y, int R, int Kp, int Kq, long long ldy,
                                                           uint8_t* __restrict__ codes, long long code_pitch,
@@ -73,13 +67,8 @@ __global__ void __launch_bounds__(256) mx_quantize_kernel(const float* __restric
     if (g < real) v = Y[(long long)m * ldy + 32 * g + lane];
     float a = fabsf(v);
     for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-    int e = 0;
-    if (a > 0.f) {
-      const int field = (int)((__float_as_uint(a) >> 23) & 0xFF);
-      e = (field == 0 ? -127 : field - 127) - 2;  // fp32 subnormals lie below 2^-126
-      e = max(-127, min(127, e));
-    }
-    const uint32_t code = e2m1_code(scalbnf(v, -e));  // exact scaling by a power of two
+    const int e = xqhad::mx_shared_exp(a);
+    const uint32_t code = xqhad::mx_e2m1_code(v * xqhad::mx_inv_scale(e));  // exact scaling by a power of two
     uint32_t w = code << (4 * (lane & 7));
     w |= __shfl_xor_sync(0xffffffffu, w, 1);
     w |= __shfl_xor_sync(0xffffffffu, w, 2);
@@ -407,7 +396,7 @@ cudaError_t launch_gemm(const uint8_t* codes, const uint8_t* sfa, int M, const x
 
 // Workspace: header (status word) | rotated rows fp32 | codes | scale blocks | scratch outputs of the rotate kernel.
 struct MxWs {
-  size_t y, codes, sf, xq, sx, total;
+  size_t y, codes, sf, xq, sx, xstage, ostage, total;
 };
 MxWs mx_ws(int M, const xq_mx_weights* w) {
   MxWs L;
@@ -422,6 +411,10 @@ MxWs mx_ws(int M, const xq_mx_weights* w) {
   off += align_up((size_t)M * (w->Kp / 2), 256);
   L.sx = off;
   off += align_up((size_t)M * 4, 256);
+  L.xstage = off;  // host entry point: staged inputs and outputs
+  off += align_up((size_t)M * w->K * 2, 256);
+  L.ostage = off;
+  off += align_up((size_t)M * w->N * 2, 256);
   L.total = off;
   return L;
 }
@@ -510,12 +503,16 @@ xq_status xq_mx_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_
     const int R = N - r0 < chunk ? N - r0 : chunk;
     e = cudaMemcpy2DAsync(dW.p, (size_t)ldw * 2, (const uint16_t*)W_host + (size_t)r0 * K, (size_t)K * 2, (size_t)K * 2, (size_t)R,
                           cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess)
-      e = xq_launch_rotate_quant(dW.p, R, ldw, w->plan, (uint8_t*)dXq.p, (float*)dS.p, (float*)dY.p, nullptr, nullptr, nullptr, w->sms, st);
     // chunk starts are multiples of 128 rows: scale blocks of different chunks do not interleave
-    if (e == cudaSuccess)
-      e = launch_quantize((const float*)dY.p, R, Kp, w->Kq, Kp, w->codes + (size_t)r0 * (w->Kq / 2), w->Kq / 2,
-                          w->sf + (size_t)(r0 / 128) * (w->Kq / 128) * 512, nullptr, st);
+    uint8_t* ccodes = w->codes + (size_t)r0 * (w->Kq / 2);
+    uint8_t* csf = w->sf + (size_t)(r0 / 128) * (w->Kq / 128) * 512;
+    if (e == cudaSuccess && xq_rotate_mx_supported(w->plan)) {
+      const xq_mx_out mx = {ccodes, csf, w->Kq};
+      e = xq_launch_rotate_mx(dW.p, R, ldw, w->plan, mx, w->sms, st);
+    } else if (e == cudaSuccess) {
+      e = xq_launch_rotate_quant(dW.p, R, ldw, w->plan, (uint8_t*)dXq.p, (float*)dS.p, (float*)dY.p, nullptr, nullptr, nullptr, w->sms, st);
+      if (e == cudaSuccess) e = launch_quantize((const float*)dY.p, R, Kp, w->Kq, Kp, ccodes, w->Kq / 2, csf, nullptr, st);
+    }
   }
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) {
@@ -642,11 +639,44 @@ xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
   uint8_t* base = (uint8_t*)ws;
   cudaStream_t st = (cudaStream_t)stream;
-  if (xq_launch_rotate_quant(X, M, ldx, w->plan, base + L.xq, (float*)(base + L.sx), (float*)(base + L.y), nullptr, w->hp_signs, nullptr,
-                             w->sms, st) != cudaSuccess ||
-      launch_quantize((const float*)(base + L.y), M, w->Kp, w->Kq, w->Kp, base + L.codes, w->Kq / 2, base + L.sf, nullptr, st) !=
-          cudaSuccess ||
+  cudaError_t e;
+  if (M >= XQ_ROTATE_ROWS_MIN_M && xq_rotate_mx_supported(w->plan)) {
+    // one kernel: pad, rotate, group exponents, codes and scale blocks straight in the GEMM's layout
+    const xq_mx_out mx = {base + L.codes, base + L.sf, w->Kq};
+    e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
+  } else {
+    e = xq_launch_rotate_quant(X, M, ldx, w->plan, base + L.xq, (float*)(base + L.sx), (float*)(base + L.y), nullptr, w->hp_signs, nullptr,
+                               w->sms, st);
+    if (e == cudaSuccess)
+      e = launch_quantize((const float*)(base + L.y), M, w->Kp, w->Kq, w->Kp, base + L.codes, w->Kq / 2, base + L.sf, nullptr, st);
+  }
+  if (e != cudaSuccess ||
       launch_gemm(base + L.codes, base + L.sf, M, w, out, (int32_t*)ws, st) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+xq_status xq_mx_expanded_linear_host(const void* X_host, int32_t M, const xq_mx_weights* w, void* out_host, void* ws, size_t ws_bytes,
+                                     void* stream) {
+  if (!w || M < 0) return XQ_ERR_INVALID_ARG;
+  if (M == 0) return XQ_OK;
+  if (!X_host || !out_host || w->K % 8 != 0) return XQ_ERR_INVALID_ARG;
+  const MxWs L = mx_ws(M, w);
+  if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
+  uint8_t* base = (uint8_t*)ws;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(base + L.xstage, X_host, (size_t)M * w->K * 2, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  xq_status s = xq_mx_expanded_linear(base + L.xstage, M, w->K, w, base + L.ostage, ws, ws_bytes, stream);
+  if (s != XQ_OK) return s;
+  e = cudaMemcpyAsync(out_host, base + L.ostage, (size_t)M * w->N * 2, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }

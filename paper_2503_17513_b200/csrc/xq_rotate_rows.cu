@@ -38,11 +38,14 @@ __device__ __forceinline__ void group_sync(int group, int Wr) {
   else xqptx::bar_sync(1 + group, 32 * Wr);
 }
 
-template <int LOG2N, int KS, int MTW, bool ASYM>
+// QM: 0 symmetric per-row INT4, 1 asymmetric per-row INT4, 2 MXFP4 (a shared exponent per 32 channels; Xq then has
+// the row pitch Kq / 2 and the scale bytes go to sfb in the block layout of the block-scaled GEMM).
+template <int LOG2N, int KS, int MTW, int QM>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     rotate_quant_rows_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx, xq_hadamard_plan_t pl, float gamma,
                              uint8_t* __restrict__ Xq, float* __restrict__ sx, float* __restrict__ Yopt, uint8_t* __restrict__ A8opt,
-                             int32_t* __restrict__ zp, int Wr, int G, int fold) {
+                             int32_t* __restrict__ zp, uint8_t* __restrict__ sfb, int Kq, int Wr, int G, int fold) {
+  constexpr bool ASYM = QM == 1;
   constexpr int n = 1 << LOG2N, NT8 = n / 8;
   constexpr int xpitch = n + 8;        // bf16 elements per staged row (conflict-free ldmatrix)
   constexpr int hpitch = KS * 16 + 8;  // bf16 elements per row of H_p^T
@@ -180,7 +183,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
           f[4] = a0 - a4; f[5] = a1 - a5; f[6] = a2 - a6; f[7] = a3 - a7;
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            if (ASYM) {
+            if (QM == 2) {
+              // the groups of 32 are reduced where they are quantized
+            } else if (ASYM) {
               amax = fmaxf(amax, f[i]);
               amin = fminf(amin, f[i]);
             } else {
@@ -190,6 +195,42 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
         }
         __syncwarp();
       }
+    if (QM == 2) {
+      // MXFP4: a thread holds 8 consecutive channels, four neighbouring lanes one group of 32
+      const long long cpitch = Kq / 2;
+#pragma unroll
+      for (int m = 0; m < MTW; ++m)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int k = 0; k < TPL; ++k) {
+            const int id = lane + 32 * k, r = id / NT8, jj = id % NT8;
+            const int a2 = 16 * (wg * MTW + m) + 8 * h + r;
+            float* f = fin[m][h][k];
+            float gmax = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              f[i] *= gamma;
+              gmax = fmaxf(gmax, fabsf(f[i]));
+            }
+            gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
+            gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
+            const int e = xqhad::mx_shared_exp(gmax);
+            const float inv = xqhad::mx_inv_scale(e);  // a power of two: the products are exact
+            uint32_t w = 0;
+#pragma unroll
+            for (int i = 7; i >= 0; --i) w = w * 16u + xqhad::mx_e2m1_code(f[i] * inv);
+            if (a2 < p) {
+              *reinterpret_cast<uint32_t*>(Xq + (long long)row * cpitch + 4ll * (a2 * NT8 + jj)) = w;
+              if ((jj & 3) == 0) sfb[xq_mx_sf_offset(row, (a2 * n + 8 * jj) >> 5, Kq)] = (uint8_t)(e + 127);
+            }
+          }
+      // padding up to Kq: zero codes, unit scales (never a NaN scale byte under the tensor core)
+      for (int i = tg; i < (Kq - Kp) / 8; i += gthreads) *reinterpret_cast<uint32_t*>(Xq + (long long)row * cpitch + Kp / 2 + 4 * i) = 0u;
+      for (int i = tg; i < (Kq - Kp) / 32; i += gthreads) sfb[xq_mx_sf_offset(row, Kp / 32 + i, Kq)] = (uint8_t)127;
+      group_sync(group, Wr);
+      continue;
+    }
     for (int o = 16; o > 0; o >>= 1) {
       amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
       if (ASYM) amin = fminf(amin, __shfl_xor_sync(0xffffffffu, amin, o));
@@ -259,7 +300,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 
 template <int LOG2N, int KS, int MTW>
 cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
-                        float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
+                        float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st, const xq_mx_out* mx = nullptr) {
   constexpr int n = 1 << LOG2N;
   const int fold = pl.log2n - LOG2N;  // Sylvester bits folded into the outer factor
   const int MT = ((pl.p << fold) + 15) / 16, Wr = (MT + MTW - 1) / MTW;
@@ -268,7 +309,11 @@ cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard
   const size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 8;
   while (G > 1 && fixed + G * per_group > 224 * 1024) --G;
   const size_t smem = fixed + G * per_group;
-  auto kern = zp ? rotate_quant_rows_kernel<LOG2N, KS, MTW, true> : rotate_quant_rows_kernel<LOG2N, KS, MTW, false>;
+  auto kern = mx ? rotate_quant_rows_kernel<LOG2N, KS, MTW, 2>
+                 : (zp ? rotate_quant_rows_kernel<LOG2N, KS, MTW, 1> : rotate_quant_rows_kernel<LOG2N, KS, MTW, 0>);
+  uint8_t* sfb = mx ? mx->sf_blocks : nullptr;
+  const int Kq = mx ? mx->Kq : 0;
+  if (mx) Xq = mx->codes;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int want = (M + G - 1) / G;
@@ -282,41 +327,41 @@ cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, Wr, G, fold);
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sfb, Kq, Wr, G, fold);
 }
 
 template <int LOG2N, int MTW>
 cudaError_t launch_rows_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                           float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
+                           float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st, const xq_mx_out* mx = nullptr) {
   switch (ks) {
-    case 1: return launch_rows<LOG2N, 1, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 2: return launch_rows<LOG2N, 2, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 3: return launch_rows<LOG2N, 3, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    default: return launch_rows<LOG2N, 4, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 1: return launch_rows<LOG2N, 1, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 2: return launch_rows<LOG2N, 2, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 3: return launch_rows<LOG2N, 3, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    default: return launch_rows<LOG2N, 4, MTW>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
   }
 }
 
 // n > 128 folded to 128: up to 128 staged rows
 cudaError_t launch_rows_folded(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                               float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
+                               float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st, const xq_mx_out* mx = nullptr) {
   switch (ks) {
-    case 5: return launch_rows<7, 5, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 6: return launch_rows<7, 6, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 7: return launch_rows<7, 7, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 8: return launch_rows<7, 8, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    default: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 5: return launch_rows<7, 5, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 6: return launch_rows<7, 6, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 7: return launch_rows<7, 7, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 8: return launch_rows<7, 8, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    default: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
   }
 }
 
 // n = 64 with 65..128 staged rows (long inputs on a short Sylvester factor, e.g. 8192 -> 8960 = 140 x 64)
 cudaError_t launch_rows_64_long(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                                float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
+                                float* sx, float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st, const xq_mx_out* mx = nullptr) {
   switch (ks) {
-    case 5: return launch_rows<6, 5, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 6: return launch_rows<6, 6, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 7: return launch_rows<6, 7, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 8: return launch_rows<6, 8, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    default: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 5: return launch_rows<6, 5, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 6: return launch_rows<6, 6, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 7: return launch_rows<6, 7, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 8: return launch_rows<6, 8, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    default: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
   }
 }
 
@@ -336,16 +381,31 @@ bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
   return true;
 }
 
-cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
-                                  float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
+namespace {
+cudaError_t rotate_rows_dispatch(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
+                                 float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st, const xq_mx_out* mx) {
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
   const int log2n = pl.log2n > 7 ? 7 : pl.log2n;
   const int n = 1 << log2n, rows_a = (pl.K + n - 1) / n, ks = (rows_a + 15) / 16;
   // tiles of 16 output rows per warp: 80 accumulator registers at n = 32, 64 at n = 64 and 128
   switch (pl.log2n) {
-    case 5: return launch_rows_ks<5, 5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 6: return launch_rows_64_long(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    case 7: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
-    default: return launch_rows_folded(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st);
+    case 5: return launch_rows_ks<5, 5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 6: return launch_rows_64_long(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 7: return launch_rows_ks<7, 1>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    default: return launch_rows_folded(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
   }
+}
+}  // namespace
+
+cudaError_t xq_launch_rotate_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, uint8_t* Xq, float* sx,
+                                  float* Yopt, uint8_t* A8opt, int32_t* zp, int sms, cudaStream_t st) {
+  return rotate_rows_dispatch(X, M, ldx, pl, Xq, sx, Yopt, A8opt, zp, sms, st, nullptr);
+}
+
+bool xq_rotate_mx_supported(const xq_hadamard_plan_t& pl) { return pl.Kp % 32 == 0 && xq_rotate_rows_supported(pl); }
+
+cudaError_t xq_launch_rotate_mx(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, const xq_mx_out& mx, int sms,
+                                cudaStream_t st) {
+  if (!xq_rotate_mx_supported(pl)) return cudaErrorNotSupported;
+  return rotate_rows_dispatch(X, M, ldx, pl, mx.codes, nullptr, nullptr, nullptr, nullptr, sms, st, &mx);
 }

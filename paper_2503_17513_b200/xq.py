@@ -41,6 +41,7 @@ EXPORTS = [
     "xq_expanded_linear_host_asym", "xq_rotate_quant_heads", "xq_prepare_weights_heads", "xq_weights_heads",
     "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
     "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
+    "xq_mx_expanded_linear_host",
 ]
 
 
@@ -90,6 +91,7 @@ def lib() -> ctypes.CDLL:
         L.xq_mx_rotate_quant.argtypes = [vp, i32, i64, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp]
         L.xq_mx_gemm.argtypes = [vp, vp, i32, vp, vp, vp, sz, vp]
         L.xq_mx_expanded_linear.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
+        L.xq_mx_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
@@ -358,3 +360,9 @@ def xq_mx_expanded_linear(X, w: MxWeights, out, ws, M=None, ldx=None, stream=Non
     ldx = X.stride(0) if ldx is None else ldx
     _check(lib().xq_mx_expanded_linear(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _dp(ws),
                                        ws.numel() * ws.element_size(), _stream(stream)), "xq_mx_expanded_linear")
+
+
+def xq_mx_expanded_linear_host(X_host, w: MxWeights, out_host, ws, M=None, stream=None) -> None:
+    M = X_host.shape[0] if M is None else M
+    _check(lib().xq_mx_expanded_linear_host(ctypes.c_void_p(X_host.data_ptr()), M, w.handle, ctypes.c_void_p(out_host.data_ptr()),
+                                            _dp(ws), ws.numel() * ws.element_size(), _stream(stream)), "xq_mx_expanded_linear_host")
