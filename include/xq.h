@@ -93,8 +93,8 @@ void xq_weights_free(xq_weights* w);
  * for up to M_max tokens against `w`.  0 on bad arguments. */
 size_t xq_workspace_bytes(int32_t M_max, const xq_weights* w);
 
-/* Must be called once on a fresh workspace (zeroes its status word and counters; enqueued on
- * `stream`). */
+/* Must be called once on a fresh workspace (zeroes its status word and counters -- the first
+ * 1 KiB, or 256 bytes of a smaller workspace; enqueued on `stream`). */
 xq_status xq_workspace_init(void* ws_dev, size_t ws_bytes, void* stream);
 
 /* Online step (Sec. 3: expanded activations = X times the truncated Hadamard matrix; Sec. 4:

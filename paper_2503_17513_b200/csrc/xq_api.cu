@@ -347,7 +347,9 @@ size_t xq_workspace_bytes(int32_t M_max, const xq_weights* w) {
 
 xq_status xq_workspace_init(void* ws, size_t ws_bytes, void* stream) {
   if (!ws || ws_bytes < XQ_WS_HEADER_BYTES || !aligned16(ws)) return XQ_ERR_WORKSPACE;
-  if (cudaMemsetAsync(ws, 0, XQ_WS_HEADER_BYTES, (cudaStream_t)stream) != cudaSuccess) {
+  // the status word, and the arrival counters that the MXFP4 workspaces keep behind it
+  const size_t clear = ws_bytes < XQ_WS_COUNTER_BYTES ? XQ_WS_HEADER_BYTES : XQ_WS_COUNTER_BYTES;
+  if (cudaMemsetAsync(ws, 0, clear, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }

@@ -52,6 +52,9 @@ __host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_gro
 // Workspace layout (all offsets multiples of 256 bytes).  The header is what xq_workspace_init
 // clears: word 0 is the sticky status.
 constexpr size_t XQ_WS_HEADER_BYTES = 256;
+// MXFP4 workspaces: status word, then (from byte 256) one arrival counter per 128-channel tile of the split-K
+// small-batch product; xq_workspace_init clears this much of a workspace that is at least this large.
+constexpr size_t XQ_WS_COUNTER_BYTES = 1024;
 struct xq_ws_layout {
   size_t header;   // XQ_WS_HEADER_BYTES
   size_t xq;       // M_max * Kp/2 bytes of packed activations

@@ -319,6 +319,202 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Product for few tokens (M <= 32): the roles of the operands are swapped -- 128 output channels
+// are the 128 rows of the MMA, the tokens its 32 columns -- so that a tile streams the weights of
+// 128 channels, and K is cut into S slices over S CTAs so that every multiprocessor streams.  Each
+// CTA leaves its 128 x 32 fp32 partial tile in the workspace and counts itself in; the CTA that
+// arrives last adds the S partial tiles in slice order (the result does not depend on arrival
+// order), writes bf16 and puts the counter back to zero.  Nobody waits for anybody.
+// ---------------------------------------------------------------------------------------------
+constexpr int DN = 32;                      // token columns of the MMA
+constexpr int kDStages = 8;
+constexpr int kDABytes = 128 * 128, kDBBytes = DN * 128, kDSfBytes = 1024;  // weights, tokens, scale blocks of each
+constexpr int kDStageBytes = kDABytes + kDBBytes + 2 * kDSfBytes;           // 22 KiB
+constexpr int kDTmemCols = 128;
+constexpr int kDSfaCol = 32, kDSfbCol = 48;  // per stage parity: + 32 columns
+constexpr size_t kDSmemBytes = 1024 + (size_t)kDStages * kDStageBytes + 256;
+
+struct MxDecodeParams {
+  const uint8_t* sfw;  // weight scale blocks
+  const uint8_t* sfx;  // token scale blocks
+  __nv_bfloat16* out;
+  float* partial;      // [tiles][S][128][32] fp32
+  int32_t* counters;   // [tiles]
+  int32_t* status;
+  int M, N, KB, Kq, S;
+};
+
+__device__ __forceinline__ uint32_t mx_idesc_n(uint32_t sf_id, int n) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(128 >> 4) << 24) | (sf_id << 4) | (sf_id << 29);
+}
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_mx_decode_kernel(const __grid_constant__ CUtensorMap mapW,
+                                                                     const __grid_constant__ CUtensorMap mapX, const MxDecodeParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  unsigned char* base = smem_raw + (((raw + 1023u) & ~1023u) - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)kDStages * kDStageBytes);
+  uint64_t* full = bars;
+  uint64_t* empty = full + kDStages;
+  uint64_t* acc_full = empty + kDStages;
+  uint64_t* drain = acc_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* last_flag = const_cast<int*>(reinterpret_cast<volatile int*>(tmem_slot + 2));
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile = blockIdx.x / p.S, split = blockIdx.x - tile * p.S;
+  const int kb_lo = (split * p.KB) / p.S, kb_hi = ((split + 1) * p.KB) / p.S;  // this CTA's 256-code blocks (at least one)
+
+  if (tid == 0) {
+    for (int s = 0; s < kDStages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(acc_full, 1);
+    mbar_init(drain, 1);
+    *failed = 0;
+    *last_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&mapW);
+    tma_prefetch_desc(&mapX);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kDTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    // ---------------- producer: weights first (they do not depend on the kernel before), then tokens ----------
+    const size_t kblocks = (size_t)(p.Kq >> 7);
+    bool ok = true;
+    const int nk = kb_hi - kb_lo, pre = nk < kDStages ? nk : kDStages;
+    if (lane == 0) {
+      for (int i = 0; i < pre; ++i) {
+        unsigned char* st = base + (size_t)i * kDStageBytes;
+        mbar_expect_tx(&full[i], kDStageBytes);
+        tma_load_2d(st, &mapW, (kb_lo + i) * 128, tile * 128, &full[i]);
+        bulk_g2s(st + kDABytes + kDBBytes, p.sfw + ((size_t)tile * kblocks + 2 * (kb_lo + i)) * 512, kDSfBytes, &full[i]);
+      }
+    }
+    __syncwarp();
+    pdl_wait();  // the tokens and their scales come from the kernel before this one
+    for (int i = 0; i < nk && ok; ++i) {
+      const int s = i % kDStages, kb = kb_lo + i;
+      if (i >= kDStages) {
+        ok = mbar_wait_bounded(&empty[s], ((i / kDStages) - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+        if (!ok) break;
+      }
+      if (lane == 0) {
+        unsigned char* st = base + (size_t)s * kDStageBytes;
+        if (i >= kDStages) {
+          mbar_expect_tx(&full[s], kDStageBytes);
+          tma_load_2d(st, &mapW, kb * 128, tile * 128, &full[s]);
+          bulk_g2s(st + kDABytes + kDBBytes, p.sfw + ((size_t)tile * kblocks + 2 * kb) * 512, kDSfBytes, &full[s]);
+        }
+        tma_load_2d(st + kDABytes, &mapX, kb * 128, 0, &full[s]);
+        bulk_g2s(st + kDABytes + kDBBytes + kDSfBytes, p.sfx + (size_t)(2 * kb) * 512, kDSfBytes, &full[s]);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issue -------------------------------------------------------------------
+    bool ok = true;
+    const int nk = kb_hi - kb_lo;
+    for (int i = 0; i < nk; ++i) {
+      const int s = i % kDStages;
+      ok = mbar_wait_bounded(&full[s], (i / kDStages) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+      if (!ok) break;
+      tc_fence_after_sync();
+      if (lane == 0) {
+        const uint32_t a_addr = smem_u32(base + (size_t)s * kDStageBytes);
+        const uint32_t sfa_smem = a_addr + kDABytes + kDBBytes, sfb_smem = sfa_smem + kDSfBytes;
+        const uint32_t sfa_t = tmem_base + kDSfaCol + 32 * (i & 1), sfb_t = tmem_base + kDSfbCol + 32 * (i & 1);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {  // K halves of 128 codes: 4 columns of channel scales, 4 of token scales (one used)
+          tmem_cp_32x128b_warpx4(sfa_t + 4 * j, sf_desc(sfa_smem + 512 * j));
+          tmem_cp_32x128b_warpx4(sfb_t + 4 * j, sf_desc(sfb_smem + 512 * j));
+        }
+        const uint64_t adesc = umma_desc_k128(a_addr), bdesc = umma_desc_k128(a_addr + kDABytes);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_mxf4_ss(tmem_base, adesc + 2 * k, bdesc + 2 * k, mx_idesc_n(2u * (k & 1), DN), (i | k) != 0 ? 1u : 0u, sfa_t + 4 * (k >> 1),
+                       sfb_t + 4 * (k >> 1));
+        umma_commit(&empty[s]);
+      }
+      __syncwarp();
+    }
+    if (ok && lane == 0) umma_commit(acc_full);
+    __syncwarp();
+    if (lane == 0) umma_commit(drain);
+    __syncwarp();
+    mbar_wait_bounded(drain, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);
+  } else {
+    // ---------------- epilogue: lane = one output channel, 32 token columns ---------------------------
+    const int q = warp & 3, et = (warp - 2) * 32 + lane;  // thread index among the 128 epilogue threads
+    const int c = q * 32 + lane, n = tile * 128 + c;
+    bool ok = mbar_wait_bounded(acc_full, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);
+    float v[32];
+    if (ok) {
+      tc_fence_after_sync();
+      uint32_t r[32];
+      tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16), r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int m = 0; m < 32; ++m) v[m] = __uint_as_float(r[m]);
+    }
+    bool reduce = ok && p.S == 1;
+    if (ok && p.S > 1) {
+      float4* dst = reinterpret_cast<float4*>(p.partial + (((size_t)tile * p.S + split) * 128 + c) * 32);
+#pragma unroll
+      for (int m4 = 0; m4 < 8; ++m4) __stcg(dst + m4, make_float4(v[4 * m4], v[4 * m4 + 1], v[4 * m4 + 2], v[4 * m4 + 3]));
+      __threadfence();
+    }
+    bar_sync(1, 128);
+    if (p.S > 1) {
+      if (et == 0) *last_flag = ok && atomicAdd(p.counters + tile, 1) == p.S - 1;
+      bar_sync(1, 128);
+      if (*last_flag) {
+        __threadfence();
+#pragma unroll
+        for (int m = 0; m < 32; ++m) v[m] = 0.f;
+        for (int s = 0; s < p.S; ++s) {  // slice order: the sum does not depend on who arrived when
+          const float4* src = reinterpret_cast<const float4*>(p.partial + (((size_t)tile * p.S + s) * 128 + c) * 32);
+#pragma unroll
+          for (int m4 = 0; m4 < 8; ++m4) {
+            const float4 t = __ldcg(src + m4);
+            v[4 * m4] += t.x; v[4 * m4 + 1] += t.y; v[4 * m4 + 2] += t.z; v[4 * m4 + 3] += t.w;
+          }
+        }
+        if (et == 0) p.counters[tile] = 0;  // ready for the next call on this workspace
+        reduce = true;
+      }
+    }
+    if (reduce && n < p.N) {
+#pragma unroll
+      for (int m = 0; m < 32; ++m)
+        if (m < p.M) p.out[(size_t)m * p.N + n] = __float2bfloat16_rn(v[m]);
+    }
+    tc_fence_before_sync();
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0 && *failed) {
+    for (int s = 0; s < kDStages; ++s) mbar_wait(&full[s], 0, 1u << 16), mbar_wait(&full[s], 1, 1u << 16);
+  }
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kDTmemCols);
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -370,6 +566,32 @@ cudaError_t launch_quantize(const float* Y, int R, int Kp, int Kq, int64_t ldy, 
   return cudaLaunchKernelEx(&cfg, mx_quantize_kernel, Y, R, Kp, Kq, (long long)ldy, codes, (long long)code_pitch, sf_blocks, sf_rows);
 }
 
+int mx_decode_splits(const xq_mx_weights* w);
+
+cudaError_t launch_gemm_decode(const uint8_t* codes, const uint8_t* sfx, int M, const xq_mx_weights* w, void* out, uint8_t* ws,
+                               size_t partial_off, cudaStream_t st) {
+  CUtensorMap mapW, mapX;
+  if (!make_map(&mapW, w->codes, w->Np, w->Kq, 128) || !make_map(&mapX, codes, M, w->Kq, DN)) return cudaErrorInvalidValue;
+  MxDecodeParams p;
+  p.sfw = w->sf;
+  p.sfx = sfx;
+  p.out = (__nv_bfloat16*)out;
+  p.partial = (float*)(ws + partial_off);
+  p.counters = (int32_t*)(ws + XQ_WS_HEADER_BYTES);
+  p.status = (int32_t*)ws;
+  p.M = M;
+  p.N = w->N;
+  p.Kq = w->Kq;
+  p.KB = w->Kq / 256;
+  p.S = mx_decode_splits(w);
+  cudaError_t e = cudaFuncSetAttribute(gemm_mx_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDSmemBytes);
+  if (e != cudaSuccess) return e;
+  const int tiles = (w->N + 127) / 128;
+  cudaLaunchAttribute attr[1];
+  cudaLaunchConfig_t cfg = pdl_config(dim3(tiles * p.S), dim3(kThreads), kDSmemBytes, st, attr);
+  return cudaLaunchKernelEx(&cfg, gemm_mx_decode_kernel, mapW, mapX, p);
+}
+
 // codes / scale blocks of the tokens in device form -> out
 cudaError_t launch_gemm(const uint8_t* codes, const uint8_t* sfa, int M, const xq_mx_weights* w, void* out, int32_t* status,
                         cudaStream_t st) {
@@ -396,11 +618,22 @@ cudaError_t launch_gemm(const uint8_t* codes, const uint8_t* sfa, int M, const x
 
 // Workspace: header (status word) | rotated rows fp32 | codes | scale blocks | scratch outputs of the rotate kernel.
 struct MxWs {
-  size_t y, codes, sf, xq, sx, xstage, ostage, total;
+  size_t y, codes, sf, xq, sx, xstage, ostage, partial, total;
 };
+constexpr int kMxDecodeMaxM = DN;
+// K slices of the small-batch product: every multiprocessor gets a CTA, a slice has at least one 256-code block.
+int mx_decode_splits(const xq_mx_weights* w) {
+  const int tiles = w->Np / 128, KB = w->Kq / 256;
+  int S = w->sms / tiles;
+  if (S < 1) S = 1;
+  if (S > KB) S = KB;
+  if (S > 3) S = 3;  // the last CTA of a tile adds S partial tiles one after the other: few, long slices
+  if (tiles > (int)((XQ_WS_COUNTER_BYTES - XQ_WS_HEADER_BYTES) / 4)) S = 1;  // one counter per tile
+  return S;
+}
 MxWs mx_ws(int M, const xq_mx_weights* w) {
   MxWs L;
-  size_t off = XQ_WS_HEADER_BYTES;
+  size_t off = XQ_WS_COUNTER_BYTES;
   L.y = off;
   off += align_up((size_t)M * w->Kp * 4, 256);
   L.codes = off;
@@ -415,6 +648,8 @@ MxWs mx_ws(int M, const xq_mx_weights* w) {
   off += align_up((size_t)M * w->K * 2, 256);
   L.ostage = off;
   off += align_up((size_t)M * w->N * 2, 256);
+  L.partial = off;  // partial tiles of the split-K small-batch product
+  off += (size_t)(w->Np / 128) * mx_decode_splits(w) * 128 * 32 * 4;
   L.total = off;
   return L;
 }
@@ -622,7 +857,8 @@ xq_status xq_mx_gemm(const uint8_t* codes, const uint8_t* scales, int32_t M, con
   cudaLaunchConfig_t cfg = pdl_config(dim3(148 * 4), dim3(256), 0, st, attr);
   if (cudaLaunchKernelEx(&cfg, mx_to_device_form_kernel, codes, scales, (int)M, (int)w->Kp, (int)w->Kq, base + L.codes, base + L.sf) !=
           cudaSuccess ||
-      launch_gemm(base + L.codes, base + L.sf, M, w, out, (int32_t*)ws, st) != cudaSuccess) {
+      (M <= kMxDecodeMaxM ? launch_gemm_decode(base + L.codes, base + L.sf, M, w, out, base, L.partial, st)
+                          : launch_gemm(base + L.codes, base + L.sf, M, w, out, (int32_t*)ws, st)) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
@@ -651,7 +887,8 @@ xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_
       e = launch_quantize((const float*)(base + L.y), M, w->Kp, w->Kq, w->Kp, base + L.codes, w->Kq / 2, base + L.sf, nullptr, st);
   }
   if (e != cudaSuccess ||
-      launch_gemm(base + L.codes, base + L.sf, M, w, out, (int32_t*)ws, st) != cudaSuccess) {
+      (M <= kMxDecodeMaxM ? launch_gemm_decode(base + L.codes, base + L.sf, M, w, out, base, L.partial, st)
+                          : launch_gemm(base + L.codes, base + L.sf, M, w, out, (int32_t*)ws, st)) != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }

@@ -94,7 +94,8 @@ def test_mx_rotate_quant_stage_parity(xq, oracle, M, K, Kp):
 GEMM_CASES = [
     # (M, N, K, Kp): one tile with a K tail inside the 256-code block, ragged token and channel tails, several tiles per CTA
     (5, 8, 100, 160), (33, 256, 64, 128), (1, 2048, 2048, 2176), (130, 264, 2048, 2176), (300, 512, 4096, 4608),
-    (129, 1000, 200, 256), (2048, 2048, 2048, 2176), (16, 512, 8192, 8704),
+    (129, 1000, 200, 256), (2048, 2048, 2048, 2176), (16, 512, 8192, 8704), (32, 8192, 2048, 2176), (8, 3072, 2048, 2176),
+    (32, 4096, 14336, 15360),
 ]
 
 
