@@ -115,31 +115,34 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out, int32
       xq_weights_free(w);
       return XQ_ERR_ALLOC;
     }
-  } else if (pl.p > 1 && pl.p <= XQ_MAX_P_IMAGE) {
-    // bf16 image of H_p^T (row a', column a) for the rotate kernel: a constant of the plan
-    const int P16 = (pl.p + 15) / 16 * 16, pitch = P16 + 8;
-    uint16_t* img = (uint16_t*)calloc((size_t)P16 * pitch, sizeof(uint16_t));
-    if (!img) {
-      xq_weights_free(w);
-      return XQ_ERR_ALLOC;
-    }
-    for (int a2 = 0; a2 < pl.p; ++a2)
-      for (int a = 0; a < pl.p; ++a) img[(size_t)a2 * pitch + a] = host_paley_sign(pl, a, a2) > 0 ? 0x3F80 : 0xBF80;
-    const size_t img_bytes = (size_t)P16 * pitch * sizeof(uint16_t);
-    const bool ok = cudaMalloc((void**)&w->hp_signs, img_bytes) == cudaSuccess &&
-                    cudaMemcpy(w->hp_signs, img, img_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
-    free(img);
-    if (!ok) {
-      cudaGetLastError();
-      xq_weights_free(w);
-      return XQ_ERR_ALLOC;
-    }
+  } else if (!xq_make_hp_signs(pl, &w->hp_signs)) {
+    cudaGetLastError();
+    xq_weights_free(w);
+    return XQ_ERR_ALLOC;
   }
   *out = w;
   return XQ_OK;
 }
 
 }  // namespace
+
+bool xq_make_hp_signs(const xq_hadamard_plan_t& pl, uint16_t** out) {
+  *out = nullptr;
+  if (pl.p <= 1 || pl.p > XQ_MAX_P_IMAGE) return true;  // no image: the kernels that read one do not take this plan
+  const int P16 = (pl.p + 15) / 16 * 16, pitch = P16 + 8;
+  uint16_t* img = (uint16_t*)calloc((size_t)P16 * pitch, sizeof(uint16_t));
+  if (!img) return false;
+  for (int a2 = 0; a2 < pl.p; ++a2)
+    for (int a = 0; a < pl.p; ++a) img[(size_t)a2 * pitch + a] = host_paley_sign(pl, a, a2) > 0 ? 0x3F80 : 0xBF80;
+  const size_t img_bytes = (size_t)P16 * pitch * sizeof(uint16_t);
+  const bool ok = cudaMalloc((void**)out, img_bytes) == cudaSuccess && cudaMemcpy(*out, img, img_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+  free(img);
+  if (!ok && *out) {
+    cudaFree(*out);
+    *out = nullptr;
+  }
+  return ok;
+}
 
 xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w) {
   xq_ws_layout L;

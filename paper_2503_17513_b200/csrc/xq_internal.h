@@ -66,6 +66,9 @@ struct xq_ws_layout {
   size_t total;
 };
 xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
+// bf16 image of H_p^T (row a', column a; [P16][P16 + 8]) in device memory: a constant of the plan that the one-row
+// rotate kernel reads.  *out stays null for plans without one.  False when the allocation or the copy fails.
+bool xq_make_hp_signs(const xq_hadamard_plan_t& pl, uint16_t** out);
 
 // Size of the built-in scratch array of xq_expanded_linear_static.
 constexpr size_t XQ_STATIC_SCRATCH_BYTES = 4u << 20;
@@ -89,6 +92,9 @@ __host__ __device__ inline size_t xq_mx_sf_offset(int m, int g, int Kq) {
 bool xq_rotate_mx_supported(const xq_hadamard_plan_t& pl);
 cudaError_t xq_launch_rotate_mx(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, const xq_mx_out& mx, int sms,
                                 cudaStream_t st);
+// The same from the one-row-per-CTA tensor-core kernel (few rows); cudaErrorNotSupported when the plan is not one of its.
+cudaError_t xq_launch_rotate_tc_mx(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, const xq_mx_out& mx,
+                                   const void* Hsigns, int sms, cudaStream_t st);
 
 // Launchers (each returns the CUDA error of its launch).
 // A8opt (optional): byte-per-code copy of the codes in the operand format of the tcgen05 GEMM, [M, Kp].

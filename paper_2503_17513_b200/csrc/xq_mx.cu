@@ -686,7 +686,7 @@ xq_status make_mx_weights(int32_t N, int32_t K, int32_t Kp, xq_mx_weights** out)
   }
   const size_t cb = (size_t)w->Np * (w->Kq / 2), sb = sf_bytes(w->Np, w->Kq);
   if (cudaMalloc((void**)&w->codes, cb) != cudaSuccess || cudaMalloc((void**)&w->sf, sb) != cudaSuccess ||
-      cudaMemset(w->codes, 0, cb) != cudaSuccess || cudaMemset(w->sf, 127, sb) != cudaSuccess) {
+      cudaMemset(w->codes, 0, cb) != cudaSuccess || cudaMemset(w->sf, 127, sb) != cudaSuccess || !xq_make_hp_signs(pl, &w->hp_signs)) {
     cudaGetLastError();
     xq_mx_weights_free(w);
     return XQ_ERR_ALLOC;
@@ -875,12 +875,13 @@ xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
   uint8_t* base = (uint8_t*)ws;
   cudaStream_t st = (cudaStream_t)stream;
-  cudaError_t e;
-  if (M >= XQ_ROTATE_ROWS_MIN_M && xq_rotate_mx_supported(w->plan)) {
-    // one kernel: pad, rotate, group exponents, codes and scale blocks straight in the GEMM's layout
-    const xq_mx_out mx = {base + L.codes, base + L.sf, w->Kq};
-    e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
-  } else {
+  cudaError_t e = cudaErrorNotSupported;
+  // one kernel: pad, rotate, group exponents, codes and scale blocks straight in the GEMM's layout
+  const xq_mx_out mx = {base + L.codes, base + L.sf, w->Kq};
+  if (M >= XQ_ROTATE_ROWS_MIN_M && xq_rotate_mx_supported(w->plan)) e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
+  else if (M < XQ_ROTATE_ROWS_MIN_M) e = xq_launch_rotate_tc_mx(X, M, ldx, w->plan, mx, w->hp_signs, w->sms, st);
+  if (e == cudaErrorNotSupported && xq_rotate_mx_supported(w->plan)) e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
+  if (e == cudaErrorNotSupported) {
     e = xq_launch_rotate_quant(X, M, ldx, w->plan, base + L.xq, (float*)(base + L.sx), (float*)(base + L.y), nullptr, w->hp_signs, nullptr,
                                w->sms, st);
     if (e == cudaSuccess)

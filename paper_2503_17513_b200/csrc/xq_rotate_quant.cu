@@ -120,7 +120,9 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
                                                               xq_hadamard_plan_t pl, float gamma, uint8_t* __restrict__ Xq,
                                                               float* __restrict__ sx, float* __restrict__ Yopt,
                                                               uint8_t* __restrict__ A8opt, const __nv_bfloat16* __restrict__ Hsigns,
-                                                              int32_t* __restrict__ zp) {
+                                                              int32_t* __restrict__ zp, uint8_t* __restrict__ sfb, int Kq) {
+  // sfb != null: MXFP4 instead of per-row INT4 -- a shared exponent per 32 channels, E2M1 codes; Xq then has the row
+  // pitch Kq / 2 and the scale bytes go to sfb in the block layout of the block-scaled GEMM (sx, zp, A8opt unused).
   constexpr int NB = 1 << LOG2NB;  // columns per warp
   constexpr int NT8 = NB / 8;      // n-tiles per warp
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -133,7 +135,8 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
 
   __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
   uint32_t* outp = reinterpret_cast<uint32_t*>(Xs + KS * 16 * pitch);  // Kp / 8 words
-  float* red = reinterpret_cast<float*>(outp + Kp / 8);               // 32 floats
+  uint8_t* sfs = reinterpret_cast<uint8_t*>(outp + Kp / 8);           // Kp / 32 scale bytes of the row (MXFP4)
+  float* red = reinterpret_cast<float*>(sfs + (Kp / 32 + 15) / 16 * 16);  // 32 floats
   int8_t* chi2 = reinterpret_cast<int8_t*>(red + 32);
   int8_t* sq = chi2 + 2 * q + 1;
   // shared image of H_p^T (only when the caller has one ready in global memory), then the exchange buffer
@@ -263,8 +266,32 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
         vmax = fmaxf(vmax, acc[j][e]);
         vmin = fminf(vmin, acc[j][e]);
       }
-    RowQuant rq;
-    if (zp) {
+    RowQuant rq = row_quant_sym(0.f);
+    if (sfb) {
+      // MXFP4: the group of 32 channels is four neighbouring column tiles of one row, spread over the quad
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int a2 = 16 * mt + g + 8 * r;
+#pragma unroll
+        for (int gq = 0; gq < NT8 / 4; ++gq) {
+          float gm = 0.f;
+#pragma unroll
+          for (int j = 4 * gq; j < 4 * gq + 4; ++j) gm = fmaxf(gm, fmaxf(fabsf(acc[j][2 * r]), fabsf(acc[j][2 * r + 1])));
+          gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, 1));
+          gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, 2));
+          const int e = mx_shared_exp(gm);
+          const float inv = mx_inv_scale(e);
+#pragma unroll
+          for (int j = 4 * gq; j < 4 * gq + 4; ++j) {
+            uint32_t w = (mx_e2m1_code(acc[j][2 * r] * inv) | (mx_e2m1_code(acc[j][2 * r + 1] * inv) << 4)) << (8 * t);
+            w |= __shfl_xor_sync(0xffffffffu, w, 1);
+            w |= __shfl_xor_sync(0xffffffffu, w, 2);
+            if (t == 0 && a2 < p) outp[(a2 * n + bc * NB) / 8 + j] = w;
+          }
+          if (t == 0 && a2 < p) sfs[(a2 * n + bc * NB) / 32 + gq] = (uint8_t)(e + 127);
+        }
+      }
+    } else if (zp) {
       vmax = block_max(vmax, red);
       vmin = -block_max(-vmin, red);
       rq = row_quant_asym(vmin, vmax);
@@ -274,7 +301,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
     const float s = rq.s;
     // quantize, pack: the quad's four bytes of one (row, j) form one word of 8 codes
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
+    for (int r = 0; r < 2 && !sfb; ++r) {
       const int a2 = 16 * mt + g + 8 * r;
 #pragma unroll
       for (int j = 0; j < NT8; ++j) {
@@ -298,11 +325,16 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
       }
     }
     __syncthreads();
-    if (tid == 0) {
+    if (tid == 0 && !sfb) {
       sx[row] = s;
       if (zp) zp[row] = rq.z;
     }
-    uint4* dst = reinterpret_cast<uint4*>(Xq + (long long)row * (Kp / 2));
+    if (sfb) {
+      // scale bytes into their blocks; padding up to Kq: unit scales and zero codes (never a NaN scale byte)
+      for (int i = tid; i < Kq / 32; i += nthreads) sfb[xq_mx_sf_offset(row, i, Kq)] = i < Kp / 32 ? sfs[i] : (uint8_t)127;
+      for (int i = tid; i < (Kq - Kp) / 8; i += nthreads) *reinterpret_cast<uint32_t*>(Xq + (long long)row * (Kq / 2) + Kp / 2 + 4 * i) = 0u;
+    }
+    uint4* dst = reinterpret_cast<uint4*>(Xq + (long long)row * ((sfb ? Kq : Kp) / 2));
     for (int i = tid; i < Kp / 32; i += nthreads) {
       const uint4 v = reinterpret_cast<const uint4*>(outp)[i];
       dst[i] = v;
@@ -323,9 +355,11 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
 
 template <int LOG2NB, int KS>
 cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
-                      float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st) {
+                      float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st,
+                      const xq_mx_out* mx = nullptr) {
   const int n = 1 << pl.log2n, NB = 1 << LOG2NB, NC = n / NB, MT = (pl.p + 15) / 16;
-  size_t smem = (size_t)KS * 16 * (n + 8) * 2 + (size_t)pl.Kp / 2 + 128 + (size_t)(3 * pl.q + 1) + 32;
+  size_t smem = (size_t)KS * 16 * (n + 8) * 2 + (size_t)pl.Kp / 2 + (size_t)pl.Kp / 32 + 16 + 128 + (size_t)(3 * pl.q + 1) + 32;
+  if (mx) Xq = mx->codes;
   if (Hsigns) smem += (size_t)MT * 16 * (MT * 16 + 8) * 2;
   if (NC == 2) smem += (size_t)MT * 16 * n * 4;
   auto kern = rotate_quant_tc_kernel<LOG2NB, KS>;
@@ -344,17 +378,19 @@ cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_p
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt,
-                            (const __nv_bfloat16*)Hsigns, zp);
+                            (const __nv_bfloat16*)Hsigns, zp,
+                            mx ? mx->sf_blocks : (uint8_t*)nullptr, mx ? (int)mx->Kq : 0);
 }
 
 template <int LOG2NB>
 cudaError_t launch_tc_ks(int ks, const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq,
-                         float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st) {
+                         float* sx, float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st,
+                         const xq_mx_out* mx = nullptr) {
   switch (ks) {
-    case 1: return launch_tc<LOG2NB, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
-    case 2: return launch_tc<LOG2NB, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
-    case 3: return launch_tc<LOG2NB, 3>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
-    default: return launch_tc<LOG2NB, 4>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
+    case 1: return launch_tc<LOG2NB, 1>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st, mx);
+    case 2: return launch_tc<LOG2NB, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st, mx);
+    case 3: return launch_tc<LOG2NB, 3>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st, mx);
+    default: return launch_tc<LOG2NB, 4>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st, mx);
   }
 }
 
@@ -451,6 +487,23 @@ cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const 
   const int grid = M < sms * 8 ? M : sms * 8;
   rotate_quant_general_kernel<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp);
   return cudaGetLastError();
+}
+
+cudaError_t xq_launch_rotate_tc_mx(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, const xq_mx_out& mx,
+                                   const void* Hsigns, int sms, cudaStream_t st) {
+  const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
+  const int n = 1 << pl.log2n;
+  const int rows_a = (pl.K + n - 1) / n;
+  const int MT = (pl.p + 15) / 16;
+  const bool tc = pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 8 && pl.K % 8 == 0 && rows_a <= 64 &&
+                  MT * (n > 128 ? 2 : 1) <= 16;
+  if (!tc || pl.Kp % 32 != 0) return cudaErrorNotSupported;
+  const int ks = (rows_a + 15) / 16;
+  switch (pl.log2n) {
+    case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, mx.codes, nullptr, nullptr, nullptr, Hsigns, nullptr, sms, st, &mx);
+    case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, mx.codes, nullptr, nullptr, nullptr, Hsigns, nullptr, sms, st, &mx);
+    default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, mx.codes, nullptr, nullptr, nullptr, Hsigns, nullptr, sms, st, &mx);
+  }
 }
 
 cudaError_t xq_launch_relayout_to_blocks(const uint8_t* canon, int32_t N, int32_t Kp, uint8_t* blocks, int32_t Np,
