@@ -286,9 +286,6 @@ def main():
     Wt = {n: [prepare(n, l) for l in range(layers)] for n in names}
     out = {n: torch.empty((M, table[n][2]), dtype=torch.int16, device="cuda") for n in names}
     wsp = {n: (xq.new_mx_workspace(M, Wt[n][0]) if mx else xq.new_workspace(M, Wt[n][0])) for n in names}
-    if mx:
-        mx_sc = {n: torch.empty((M, table[n][1] // 32), dtype=torch.uint8, device="cuda") for n in names}
-        mx_y = {n: torch.empty((M, table[n][1]), dtype=torch.float32, device="cuda") for n in names}
     Xq = {n: torch.empty((M, table[n][1] // 2), dtype=torch.uint8, device="cuda") for n in names}
     sx = {n: torch.empty((M,), dtype=torch.float32, device="cuda") for n in names}
     zp = {n: torch.zeros((M,), dtype=torch.int32, device="cuda") for n in names}
@@ -309,8 +306,8 @@ def main():
     def step_rotate_only():
         for l in range(layers):
             for n in names:
-                if mx:
-                    xq.xq_mx_rotate_quant(X[n], Wt[n][l].plan, Xq[n], mx_sc[n], mx_y[n], stream=stream)
+                if mx:  # the online step as the layer runs it: straight into the workspace, in the GEMM's input form
+                    xq.xq_mx_rotate_quant_staged(X[n], Wt[n][l], wsp[n], stream=stream)
                 elif heads_of[n] > 1:
                     xq.xq_rotate_quant_heads(X[n], heads_of[n], Wt[n][l].plan, Xq[n], sx[n], zp[n] if asym else None, stream=stream)
                 elif asym:
@@ -321,8 +318,8 @@ def main():
     def step_gemm_only():
         for l in range(layers):
             for n in names:
-                if mx:
-                    xq.xq_mx_gemm(Xq[n], mx_sc[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
+                if mx:  # the GEMM kernel alone, on the tokens the full step left quantized in the workspace
+                    xq.xq_mx_gemm_staged(M, Wt[n][l], out[n], wsp[n], stream=stream)
                 elif asym:
                     xq.xq_w4a4_gemm_asym(Xq[n], sx[n], zp[n], M, Wt[n][l], out[n], wsp[n], stream=stream)
                 else:
@@ -373,7 +370,7 @@ def main():
     n_sub = max(3, min(args.steps, 20))
     t_rot = timed(make_runner(step_rotate_only), n_sub, 3) / n_sub
     t_gemm = timed(make_runner(step_gemm_only), n_sub, 3) / n_sub
-    launches_per_step = (3 if mx else 2) * layers * len(names)  # MXFP4: rotate, group quantizer, GEMM
+    launches_per_step = 2 * layers * len(names)
     hbm_peak, int8_peak, peak_kind = measured_peaks()
     tensor_peak, tensor_note = int8_peak, ": 2 x sustained bf16 GEMM"
     gemm_name = "xq_w4a4_gemm (gemm_prefill_kernel)"

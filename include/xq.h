@@ -202,6 +202,16 @@ xq_status xq_mx_gemm(const uint8_t* codes_dev, const uint8_t* scales_dev, int32_
                      void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
 xq_status xq_mx_expanded_linear(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_mx_weights* w,
                                 void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+/* The two halves of xq_mx_expanded_linear, which is exactly these two calls in a row:
+ * xq_mx_rotate_quant_staged quantizes M token rows into the workspace, in the GEMM kernel's own
+ * input form (one kernel: pad, rotate, group exponents, codes); xq_mx_gemm_staged runs the product
+ * on the tokens that the last staging (or xq_mx_gemm) call with the same M and the same weights
+ * shape left there.  What a caller times separately, or re-runs against other weights of the same
+ * shape. */
+xq_status xq_mx_rotate_quant_staged(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_mx_weights* w, void* ws_dev,
+                                    size_t ws_bytes, void* stream);
+xq_status xq_mx_gemm_staged(int32_t M, const xq_mx_weights* w, void* out_bf16_dev, void* ws_dev, size_t ws_bytes,
+                            void* stream);
 /* Host buffers (X [M, K] contiguous, K a multiple of 8; out bf16 [M, N]): copies in, runs the layer, copies out,
  * synchronizes `stream`. */
 xq_status xq_mx_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_mx_weights* w, void* out_bf16_host,

@@ -865,12 +865,28 @@ xq_status xq_mx_gemm(const uint8_t* codes, const uint8_t* scales, int32_t M, con
   return XQ_OK;
 }
 
-xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_mx_weights* w, void* out, void* ws, size_t ws_bytes,
-                                void* stream) {
+xq_status xq_mx_gemm_staged(int32_t M, const xq_mx_weights* w, void* out, void* ws, size_t ws_bytes, void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!X || !out) return XQ_ERR_INVALID_ARG;
-  if (ldx < w->K || (ldx % 8) != 0 || !aligned16(X) || !aligned16(out)) return XQ_ERR_INVALID_ARG;
+  if (!out || !aligned16(out)) return XQ_ERR_INVALID_ARG;
+  const MxWs L = mx_ws(M, w);
+  if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
+  uint8_t* base = (uint8_t*)ws;
+  cudaStream_t st = (cudaStream_t)stream;
+  if ((M <= kMxDecodeMaxM ? launch_gemm_decode(base + L.codes, base + L.sf, M, w, out, base, L.partial, st)
+                          : launch_gemm(base + L.codes, base + L.sf, M, w, out, (int32_t*)ws, st)) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  return XQ_OK;
+}
+
+xq_status xq_mx_rotate_quant_staged(const void* X, int32_t M, int64_t ldx, const xq_mx_weights* w, void* ws, size_t ws_bytes,
+                                    void* stream) {
+  if (!w || M < 0) return XQ_ERR_INVALID_ARG;
+  if (M == 0) return XQ_OK;
+  if (!X) return XQ_ERR_INVALID_ARG;
+  if (ldx < w->K || (ldx % 8) != 0 || !aligned16(X)) return XQ_ERR_INVALID_ARG;
   const MxWs L = mx_ws(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
   uint8_t* base = (uint8_t*)ws;
@@ -887,13 +903,19 @@ xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_
     if (e == cudaSuccess)
       e = launch_quantize((const float*)(base + L.y), M, w->Kp, w->Kq, w->Kp, base + L.codes, w->Kq / 2, base + L.sf, nullptr, st);
   }
-  if (e != cudaSuccess ||
-      (M <= kMxDecodeMaxM ? launch_gemm_decode(base + L.codes, base + L.sf, M, w, out, base, L.partial, st)
-                          : launch_gemm(base + L.codes, base + L.sf, M, w, out, (int32_t*)ws, st)) != cudaSuccess) {
+  if (e != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
   return XQ_OK;
+}
+
+xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_mx_weights* w, void* out, void* ws, size_t ws_bytes,
+                                void* stream) {
+  if (M > 0 && (!out || !aligned16(out))) return XQ_ERR_INVALID_ARG;
+  const xq_status s = xq_mx_rotate_quant_staged(X, M, ldx, w, ws, ws_bytes, stream);
+  if (s != XQ_OK || M == 0) return s;
+  return xq_mx_gemm_staged(M, w, out, ws, ws_bytes, stream);
 }
 
 xq_status xq_mx_expanded_linear_host(const void* X_host, int32_t M, const xq_mx_weights* w, void* out_host, void* ws, size_t ws_bytes,

@@ -41,7 +41,7 @@ EXPORTS = [
     "xq_expanded_linear_host_asym", "xq_rotate_quant_heads", "xq_prepare_weights_heads", "xq_weights_heads",
     "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
     "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
-    "xq_mx_expanded_linear_host",
+    "xq_mx_expanded_linear_host", "xq_mx_gemm_staged", "xq_mx_rotate_quant_staged",
 ]
 
 
@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
         L.xq_mx_gemm.argtypes = [vp, vp, i32, vp, vp, vp, sz, vp]
         L.xq_mx_expanded_linear.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
         L.xq_mx_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
+        L.xq_mx_gemm_staged.argtypes = [i32, vp, vp, vp, sz, vp]
+        L.xq_mx_rotate_quant_staged.argtypes = [vp, i32, i64, vp, vp, sz, vp]
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
@@ -366,3 +368,14 @@ def xq_mx_expanded_linear_host(X_host, w: MxWeights, out_host, ws, M=None, strea
     M = X_host.shape[0] if M is None else M
     _check(lib().xq_mx_expanded_linear_host(ctypes.c_void_p(X_host.data_ptr()), M, w.handle, ctypes.c_void_p(out_host.data_ptr()),
                                             _dp(ws), ws.numel() * ws.element_size(), _stream(stream)), "xq_mx_expanded_linear_host")
+
+
+def xq_mx_gemm_staged(M: int, w: MxWeights, out, ws, stream=None) -> None:
+    _check(lib().xq_mx_gemm_staged(M, w.handle, _dp(out), _dp(ws), ws.numel() * ws.element_size(), _stream(stream)), "xq_mx_gemm_staged")
+
+
+def xq_mx_rotate_quant_staged(X, w: MxWeights, ws, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_mx_rotate_quant_staged(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(ws), ws.numel() * ws.element_size(),
+                                           _stream(stream)), "xq_mx_rotate_quant_staged")

@@ -162,6 +162,9 @@ def test_mx_expanded_linear_end_to_end(xq, oracle, M, N, K, Kp, heavy):
     assert rel_l2(got, want) <= E2E_REL_L2
     for m in range(M):
         assert rel_l2(got[m], want[m]) <= E2E_REL_L2
+    out3 = torch.empty_like(out)  # the product alone, on the tokens the call above left in the workspace
+    xq.xq_mx_gemm_staged(M, w, out3, ws)
+    assert torch.equal(out3, out)
     if K % 8 == 0:  # the host-buffer entry point gives the same bits
         xh = torch.from_numpy(x.view(np.int16)).pin_memory()
         oh = torch.empty((M, N), dtype=torch.int16).pin_memory()

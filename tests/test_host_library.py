@@ -96,6 +96,8 @@ def test_null_arguments_rejected_before_any_cuda_call(xq):
     assert L.xq_mx_gemm(null, null, 4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_mx_expanded_linear(null, 4, 104, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_mx_expanded_linear_host(null, 4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_gemm_staged(4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_rotate_quant_staged(null, 4, 104, null, null, 0, null) == xq.ERR_INVALID_ARG
     L.xq_mx_weights_free(null)
     assert L.xq_poll_status(null, null) == xq.ERR_WORKSPACE
     L.xq_weights_free(null)  # allowed
