@@ -235,3 +235,31 @@ def test_asym_argument_errors(xq):
         xq.xq_w4a4_gemm_asym(Xq, sx, None, M, w, out, ws)
     xq.xq_w4a4_gemm_asym(Xq, sx, zp, 0, w, out, ws)  # M = 0 is a no-op
     xq.xq_rotate_quant_asym(X, pl, Xq, sx, zp, M=0)
+
+
+FULL_CASES = [
+    # (tag, M, N, K, Kp, heavy, sampled rows): full workload sizes in the launch configuration the benchmark times
+    ("1b-qkv-m32", 32, 3072, 2048, 2176, False, 8), ("1b-down-m32", 32, 2048, 8192, 8704, False, 4),
+    ("1b-up-m2048", 2048, 8192, 2048, 2176, True, 6), ("8b-gate-m4096", 4096, 14336, 4096, 4352, True, 3),
+]
+
+
+@pytest.mark.parametrize("tag,M,N,K,Kp,heavy,nsample", FULL_CASES, ids=[c[0] for c in FULL_CASES])
+def test_asym_full_size_sampled_rows(xq, oracle, tag, M, N, K, Kp, heavy, nsample):
+    x = synth.activations(M, K, seed=0, tag=tag, heavy_tail=heavy)
+    wb = synth.weights(N, K, seed=0, tag=tag)
+    w = xq.xq_prepare_weights(wb, Kp)
+    ws = xq.new_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    xq.xq_expanded_linear_asym(dev(x), w, out, ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    rows = np.sort(np.random.default_rng(11).choice(M, size=min(nsample, M), replace=False))
+    if M > 1:
+        rows[-1] = M - 1
+    pl = oracle.plan(K, Kp)
+    qw, s_w = oracle.prepare_weights(pl, wb)
+    _, ux, s_x, z = oracle.rotate_quant_asym(pl, x[rows])
+    want = synth.bf16_bits_to_f32(oracle.epilogue_asym(oracle.gemm_u_i64(ux, qw), s_x, z, s_w, qw))
+    got = synth.bf16_bits_to_f32(host_u16(out[torch.from_numpy(rows).cuda()]))
+    for i in range(len(rows)):
+        assert rel_l2(got[i], want[i]) <= E2E_REL_L2, (tag, int(rows[i]))

@@ -179,3 +179,34 @@ def test_mx_argument_errors(xq):
     with pytest.raises(xq.XqError) as e:  # N must be a multiple of 8
         xq.xq_mx_prepare_weights(np.zeros((5, 100), np.uint16), 160)
     assert e.value.status == xq.ERR_UNSUPPORTED_ORDER
+
+
+FULL_CASES = [
+    # (tag, M, N, K, Kp, heavy, sampled rows): full workload sizes in the launch configuration the benchmark times
+    ("1b-qkv-m32", 32, 3072, 2048, 2176, False, 8), ("1b-down-m32", 32, 2048, 8192, 8704, False, 4),
+    ("1b-up-m2048", 2048, 8192, 2048, 2176, True, 6), ("8b-down-m16", 16, 4096, 14336, 15360, False, 2),
+    ("8b-gate-m4096", 4096, 14336, 4096, 4352, True, 3),
+]
+
+
+@pytest.mark.parametrize("tag,M,N,K,Kp,heavy,nsample", FULL_CASES, ids=[c[0] for c in FULL_CASES])
+def test_mx_full_size_sampled_rows(xq, oracle, tag, M, N, K, Kp, heavy, nsample):
+    x = synth.activations(M, K, seed=0, tag=tag, heavy_tail=heavy)
+    wb = synth.weights(N, K, seed=0, tag=tag)
+    w = xq.xq_mx_prepare_weights(wb, Kp)
+    ws = xq.new_mx_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    xq.xq_mx_expanded_linear(dev(x), w, out, ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    rows = np.sort(np.random.default_rng(11).choice(M, size=min(nsample, M), replace=False))
+    if M > 1:
+        rows[-1] = M - 1  # the last (possibly ragged-tile) row is always checked
+    pl = oracle.plan(K, Kp)
+    _, cw, sw = oracle.rotate_quant_mx(pl, wb)
+    _, cx, sx = oracle.rotate_quant_mx(pl, x[rows])
+    want = synth.bf16_bits_to_f32(oracle.f64_to_bf16(oracle.gemm_mx(cx, sx, cw, sw)))
+    got = synth.bf16_bits_to_f32(host_u16(out[torch.from_numpy(rows).cuda()]))
+    for i in range(len(rows)):
+        assert rel_l2(got[i], want[i]) <= E2E_REL_L2, (tag, int(rows[i]))
+    codes, sc = xq.xq_mx_weights_export(w)
+    check_quantized(oracle, codes, sc, cw, sw)
