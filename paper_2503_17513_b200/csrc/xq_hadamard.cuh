@@ -2,6 +2,7 @@
 // quadratic-character table of GF(q), block-wide maximum, transposing matrix loads.
 #pragma once
 
+#include <cuda_fp4.h>
 #include <stdint.h>
 
 namespace xqhad {
@@ -106,6 +107,11 @@ __device__ __forceinline__ uint32_t mx_e2m1_code(float v) {
   const uint32_t hi = min((u >> 22) - 252u, 7u);
   const uint32_t c = a < 1.f ? (uint32_t)__float2int_rn(a + a) : hi;
   return c | (v < 0.f ? 8u : 0u);  // a negative zero keeps the code of zero
+}
+// Two elements at once through the hardware conversion (round to nearest even, saturating): the byte holds the
+// code of lo in bits 0-3 and of hi in bits 4-7.
+__device__ __forceinline__ uint32_t mx_e2m1_pair(float lo, float hi) {
+  return (uint32_t)__nv_cvt_float2_to_fp4x2(make_float2(lo, hi), __NV_E2M1, cudaRoundNearest);
 }
 // 2^-e as a float, e in [-127, 127] (2^-127 is a subnormal: it has no exponent field of its own).
 __device__ __forceinline__ float mx_inv_scale(int e) { return e < 127 ? __uint_as_float((uint32_t)(127 - e) << 23) : 5.877471754111438e-39f; }

@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
           const float inv = mx_inv_scale(e);
 #pragma unroll
           for (int j = 4 * gq; j < 4 * gq + 4; ++j) {
-            uint32_t w = (mx_e2m1_code(acc[j][2 * r] * inv) | (mx_e2m1_code(acc[j][2 * r + 1] * inv) << 4)) << (8 * t);
+            uint32_t w = mx_e2m1_pair(acc[j][2 * r] * inv, acc[j][2 * r + 1] * inv) << (8 * t);
             w |= __shfl_xor_sync(0xffffffffu, w, 1);
             w |= __shfl_xor_sync(0xffffffffu, w, 2);
             if (t == 0 && a2 < p) outp[(a2 * n + bc * NB) / 8 + j] = w;

@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
         }
         __syncwarp();
       }
-    if (QM == 2) {
+    if constexpr (QM == 2) {
       // MXFP4: a thread holds 8 consecutive channels, four neighbouring lanes one group of 32
       const long long cpitch = Kq / 2;
 #pragma unroll
@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
             const float inv = xqhad::mx_inv_scale(e);  // a power of two: the products are exact
             uint32_t w = 0;
 #pragma unroll
-            for (int i = 7; i >= 0; --i) w = w * 16u + xqhad::mx_e2m1_code(f[i] * inv);
+            for (int i = 0; i < 4; ++i) w |= xqhad::mx_e2m1_pair(f[2 * i] * inv, f[2 * i + 1] * inv) << (8 * i);
             if (a2 < p) {
               *reinterpret_cast<uint32_t*>(Xq + (long long)row * cpitch + 4ll * (a2 * NT8 + jj)) = w;
               if ((jj & 3) == 0) sfb[xq_mx_sf_offset(row, (a2 * n + 8 * jj) >> 5, Kq)] = (uint8_t)(e + 127);
@@ -228,9 +228,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
       // padding up to Kq: zero codes, unit scales (never a NaN scale byte under the tensor core)
       for (int i = tg; i < (Kq - Kp) / 8; i += gthreads) *reinterpret_cast<uint32_t*>(Xq + (long long)row * cpitch + Kp / 2 + 4 * i) = 0u;
       for (int i = tg; i < (Kq - Kp) / 32; i += gthreads) sfb[xq_mx_sf_offset(row, Kp / 32 + i, Kq)] = (uint8_t)127;
-      group_sync(group, Wr);
-      continue;
-    }
+    } else {
     for (int o = 16; o > 0; o >>= 1) {
       amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
       if (ASYM) amin = fminf(amin, __shfl_xor_sync(0xffffffffu, amin, o));
@@ -293,6 +291,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
             }
           }
         }
+    }
     // every warp of the group is done with the stage before its reuse two loads from now
     group_sync(group, Wr);
   }
