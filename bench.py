@@ -171,7 +171,7 @@ def run_reference(args, table, layers, M, heavy):
         xs[name] = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
         wsample = synth.weights(Ns, K, seed=0, tag=name)
         if args.fmt == "mxfp4":
-            _, qw, sw = oracle.rotate_quant_mx(pl, wsample)
+            _, qw, sw = oracle.rotate_quant_mx(pl, wsample, heads)
         else:
             _, qw, sw = oracle.rotate_quant_heads(pl, heads, wsample)
         prepared[name] = (pl, qw, sw, N / Ns, heads)
@@ -182,7 +182,7 @@ def run_reference(args, table, layers, M, heavy):
             pl, qw, sw, scale, heads = prepared[name]
             t0 = time.perf_counter()
             if args.fmt == "mxfp4":
-                _, cx, sx = oracle.rotate_quant_mx(pl, xs[name])
+                _, cx, sx = oracle.rotate_quant_mx(pl, xs[name], heads)
                 t1 = time.perf_counter()
                 oracle.f64_to_bf16(oracle.gemm_mx(cx, sx, qw, sw))
             elif args.act == "asym":
@@ -274,9 +274,11 @@ def main():
 
     mx = args.fmt == "mxfp4"
     if mx:
-        assert all(h == 1 for h in heads_of.values()) and args.act == "sym", "--fmt mxfp4 runs the single-rotation symmetric path"
+        assert args.act == "sym", "--fmt mxfp4 has its own quantizer: --act does not apply"
 
     def prepare(n, l):
+        if mx and heads_of[n] > 1:
+            return xq.xq_mx_prepare_weights_heads(ws_h[n][l], heads_of[n], table[n][1] // heads_of[n])
         if mx:
             return xq.xq_mx_prepare_weights(ws_h[n][l], table[n][1])
         if heads_of[n] > 1:
@@ -466,12 +468,12 @@ def cpu_baseline_leg(table, layers, M, heavy, asym=False, mx=False):
         x = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
         wsample = synth.weights(Ns, K, seed=0, tag=name)
         if mx:
-            _, cw, sw = oracle.rotate_quant_mx(pl, wsample)
+            _, cw, sw = oracle.rotate_quant_mx(pl, wsample, heads)
         else:
             _, qw, sw = oracle.rotate_quant_heads(pl, heads, wsample)
         t0 = time.perf_counter()
         if mx:
-            _, cx, sx = oracle.rotate_quant_mx(pl, x)
+            _, cx, sx = oracle.rotate_quant_mx(pl, x, heads)
             t1 = time.perf_counter()
             oracle.f64_to_bf16(oracle.gemm_mx(cx, sx, cw, sw))
         elif asym:

@@ -190,6 +190,13 @@ int32_t xq_weights_heads(const xq_weights* w);
 typedef struct xq_mx_weights xq_mx_weights;
 xq_status xq_mx_prepare_weights(const void* W_bf16_host, int32_t N, int32_t K, int32_t Kp, void* stream,
                                 xq_mx_weights** out);
+/* MXFP4 weights behind the head-wise rotation (the paper's MXFP4 experiments expand the per-head rotation of the
+ * attention output projection, Sec. 5): rows of W are rotated per head as in xq_prepare_weights_heads (same limits, and
+ * heads * head_dim_p a multiple of 32, at least 128), then quantized in groups of 32 along the whole row; the layer calls
+ * on such an object run the head-wise online step.  xq_mx_weights_heads: number of heads (1 otherwise; 0 for NULL). */
+xq_status xq_mx_prepare_weights_heads(const void* W_bf16_host, int32_t N, int32_t heads, int32_t head_dim, int32_t head_dim_p,
+                                      void* stream, xq_mx_weights** out);
+int32_t xq_mx_weights_heads(const xq_mx_weights* w);
 xq_status xq_mx_weights_import(const uint8_t* codes_packed_host, const uint8_t* scales_host, int32_t N, int32_t K,
                                int32_t Kp, void* stream, xq_mx_weights** out);
 xq_status xq_mx_weights_export(const xq_mx_weights* w, uint8_t* codes_host, uint8_t* scales_host);

@@ -93,24 +93,7 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out, int32
     return XQ_ERR_ALLOC;
   }
   if (heads > 1) {
-    // bf16 image of the truncated head matrix, row c' = output channel, column c = input channel
-    const int d16 = (pl.K + 15) / 16 * 16, pitch = d16 + 8, n = 1 << pl.log2n;
-    const size_t elems = xq_head_image_elems(pl);
-    uint16_t* img = (uint16_t*)calloc(elems, sizeof(uint16_t));
-    if (!img) {
-      xq_weights_free(w);
-      return XQ_ERR_ALLOC;
-    }
-    for (int c2 = 0; c2 < pl.Kp; ++c2)
-      for (int c = 0; c < pl.K; ++c) {
-        int s = (__builtin_popcount((c & (n - 1)) & (c2 & (n - 1))) & 1) ? -1 : 1;
-        if (pl.p > 1) s *= host_paley_sign(pl, c >> pl.log2n, c2 >> pl.log2n);
-        img[(size_t)c2 * pitch + c] = s > 0 ? 0x3F80 : 0xBF80;
-      }
-    const bool ok = cudaMalloc((void**)&w->head_signs, elems * sizeof(uint16_t)) == cudaSuccess &&
-                    cudaMemcpy(w->head_signs, img, elems * sizeof(uint16_t), cudaMemcpyHostToDevice) == cudaSuccess;
-    free(img);
-    if (!ok) {
+    if (!xq_make_head_signs(pl, &w->head_signs)) {
       cudaGetLastError();
       xq_weights_free(w);
       return XQ_ERR_ALLOC;
@@ -125,6 +108,28 @@ xq_status make_weights(int32_t N, int32_t K, int32_t Kp, xq_weights** out, int32
 }
 
 }  // namespace
+
+bool xq_make_head_signs(const xq_hadamard_plan_t& pl, uint16_t** out) {
+  *out = nullptr;
+  const int d16 = (pl.K + 15) / 16 * 16, pitch = d16 + 8, n = 1 << pl.log2n;
+  const size_t elems = xq_head_image_elems(pl);
+  uint16_t* img = (uint16_t*)calloc(elems, sizeof(uint16_t));
+  if (!img) return false;
+  for (int c2 = 0; c2 < pl.Kp; ++c2)
+    for (int c = 0; c < pl.K; ++c) {
+      int s = (__builtin_popcount((c & (n - 1)) & (c2 & (n - 1))) & 1) ? -1 : 1;
+      if (pl.p > 1) s *= host_paley_sign(pl, c >> pl.log2n, c2 >> pl.log2n);
+      img[(size_t)c2 * pitch + c] = s > 0 ? 0x3F80 : 0xBF80;
+    }
+  const bool ok = cudaMalloc((void**)out, elems * sizeof(uint16_t)) == cudaSuccess &&
+                  cudaMemcpy(*out, img, elems * sizeof(uint16_t), cudaMemcpyHostToDevice) == cudaSuccess;
+  free(img);
+  if (!ok && *out) {
+    cudaFree(*out);
+    *out = nullptr;
+  }
+  return ok;
+}
 
 bool xq_make_hp_signs(const xq_hadamard_plan_t& pl, uint16_t** out) {
   *out = nullptr;

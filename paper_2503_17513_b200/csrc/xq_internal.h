@@ -69,6 +69,9 @@ xq_ws_layout xq_ws_compute(int32_t M_max, const xq_weights* w);
 // bf16 image of H_p^T (row a', column a; [P16][P16 + 8]) in device memory: a constant of the plan that the one-row
 // rotate kernel reads.  *out stays null for plans without one.  False when the allocation or the copy fails.
 bool xq_make_hp_signs(const xq_hadamard_plan_t& pl, uint16_t** out);
+// bf16 image of the truncated matrix of one head (row c' = output channel, column c = input channel;
+// [head_dim'][head_dim16 + 8]) for the head-wise rotate kernel.
+bool xq_make_head_signs(const xq_hadamard_plan_t& pl, uint16_t** out);
 
 // Size of the built-in scratch array of xq_expanded_linear_static.
 constexpr size_t XQ_STATIC_SCRATCH_BYTES = 4u << 20;

@@ -29,7 +29,9 @@
 using namespace xqptx;
 
 struct xq_mx_weights {
-  int32_t N, K, Kp;  // logical sizes
+  int32_t N, K, Kp;  // logical sizes (head-wise: heads * head_dim, heads * head_dim')
+  int32_t heads;     // 1: one rotation K -> Kp; > 1: the plan is that of one head
+  uint16_t* head_signs;
   int32_t Np, Kq;    // rows padded to 256, K' padded to 256
   xq_hadamard_plan_t plan;
   uint8_t* codes;    // device, Np * Kq / 2
@@ -662,11 +664,17 @@ struct DevBuf {
   }
 };
 
-xq_status make_mx_weights(int32_t N, int32_t K, int32_t Kp, xq_mx_weights** out) {
-  if (N < 1 || K < 1 || Kp < K) return XQ_ERR_INVALID_ARG;
+// heads > 1: K and Kp are the sizes of ONE head
+xq_status make_mx_weights(int32_t N, int32_t K, int32_t Kp, xq_mx_weights** out, int32_t heads = 1) {
+  if (N < 1 || K < 1 || Kp < K || heads < 1) return XQ_ERR_INVALID_ARG;
   xq_hadamard_plan_t pl;
   xq_status s = xq_hadamard_plan(K, Kp, &pl);
   if (s != XQ_OK) return s;
+  if (heads > 1) {
+    if (!xq_rotate_heads_supported(pl, heads)) return XQ_ERR_UNSUPPORTED_ORDER;
+    K *= heads;
+    Kp *= heads;
+  }
   if (Kp % 32 != 0 || Kp < 128 || N % 8 != 0) return XQ_ERR_UNSUPPORTED_ORDER;  // whole groups; 16-byte output pieces
   xq_mx_weights* w = new (std::nothrow) xq_mx_weights();
   if (!w) return XQ_ERR_ALLOC;
@@ -676,6 +684,8 @@ xq_status make_mx_weights(int32_t N, int32_t K, int32_t Kp, xq_mx_weights** out)
   w->Np = (int32_t)align_up((size_t)N, 256);
   w->Kq = (int32_t)align_up((size_t)Kp, 256);
   w->plan = pl;
+  w->heads = heads;
+  w->head_signs = nullptr;
   w->codes = nullptr;
   w->sf = nullptr;
   w->hp_signs = nullptr;
@@ -686,7 +696,8 @@ xq_status make_mx_weights(int32_t N, int32_t K, int32_t Kp, xq_mx_weights** out)
   }
   const size_t cb = (size_t)w->Np * (w->Kq / 2), sb = sf_bytes(w->Np, w->Kq);
   if (cudaMalloc((void**)&w->codes, cb) != cudaSuccess || cudaMalloc((void**)&w->sf, sb) != cudaSuccess ||
-      cudaMemset(w->codes, 0, cb) != cudaSuccess || cudaMemset(w->sf, 127, sb) != cudaSuccess || !xq_make_hp_signs(pl, &w->hp_signs)) {
+      cudaMemset(w->codes, 0, cb) != cudaSuccess || cudaMemset(w->sf, 127, sb) != cudaSuccess ||
+      !(heads > 1 ? xq_make_head_signs(pl, &w->head_signs) : xq_make_hp_signs(pl, &w->hp_signs))) {
     cudaGetLastError();
     xq_mx_weights_free(w);
     return XQ_ERR_ALLOC;
@@ -704,6 +715,7 @@ void xq_mx_weights_free(xq_mx_weights* w) {
   if (w->codes) cudaFree(w->codes);
   if (w->sf) cudaFree(w->sf);
   if (w->hp_signs) cudaFree(w->hp_signs);
+  if (w->head_signs) cudaFree(w->head_signs);
   delete w;
 }
 
@@ -716,12 +728,25 @@ xq_status xq_mx_weights_info(const xq_mx_weights* w, int32_t* N, int32_t* K, int
   return XQ_OK;
 }
 
-xq_status xq_mx_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t Kp, void* stream, xq_mx_weights** out) {
+}  // extern "C"
+
+namespace {
+// the fp32 rows of the online step, for the forms that have no fused quantizer
+cudaError_t rotate_to_fp32(const xq_mx_weights* w, const void* X, int32_t M, int64_t ldx, uint8_t* xq_scratch, float* sx_scratch, float* Y,
+                           cudaStream_t st) {
+  if (w->heads > 1)
+    return xq_launch_rotate_heads(X, M, ldx, w->plan, w->heads, xq_scratch, sx_scratch, Y, nullptr, w->head_signs, nullptr, w->sms, st);
+  return xq_launch_rotate_quant(X, M, ldx, w->plan, xq_scratch, sx_scratch, Y, nullptr, w->hp_signs, nullptr, w->sms, st);
+}
+
+xq_status mx_prepare_impl(const void* W_host, int32_t N, int32_t heads, int32_t K, int32_t Kp, void* stream, xq_mx_weights** out) {
   if (!W_host || !out) return XQ_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   xq_mx_weights* w = nullptr;
-  xq_status s = make_mx_weights(N, K, Kp, &w);
+  xq_status s = make_mx_weights(N, K, Kp, &w, heads);
   if (s != XQ_OK) return s;
+  K = w->K;
+  Kp = w->Kp;
   // rows of W go through the same pad + rotate kernels as token rows, in chunks of 2048 rows
   const int chunk = 2048;
   const int64_t ldw = (int64_t)align_up((size_t)K, 8);
@@ -741,11 +766,11 @@ xq_status xq_mx_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_
     // chunk starts are multiples of 128 rows: scale blocks of different chunks do not interleave
     uint8_t* ccodes = w->codes + (size_t)r0 * (w->Kq / 2);
     uint8_t* csf = w->sf + (size_t)(r0 / 128) * (w->Kq / 128) * 512;
-    if (e == cudaSuccess && xq_rotate_mx_supported(w->plan)) {
+    if (e == cudaSuccess && w->heads == 1 && xq_rotate_mx_supported(w->plan)) {
       const xq_mx_out mx = {ccodes, csf, w->Kq};
       e = xq_launch_rotate_mx(dW.p, R, ldw, w->plan, mx, w->sms, st);
     } else if (e == cudaSuccess) {
-      e = xq_launch_rotate_quant(dW.p, R, ldw, w->plan, (uint8_t*)dXq.p, (float*)dS.p, (float*)dY.p, nullptr, nullptr, nullptr, w->sms, st);
+      e = rotate_to_fp32(w, dW.p, R, ldw, (uint8_t*)dXq.p, (float*)dS.p, (float*)dY.p, st);
       if (e == cudaSuccess) e = launch_quantize((const float*)dY.p, R, Kp, w->Kq, Kp, ccodes, w->Kq / 2, csf, nullptr, st);
     }
   }
@@ -758,6 +783,22 @@ xq_status xq_mx_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_
   *out = w;
   return XQ_OK;
 }
+
+}  // namespace
+
+extern "C" {
+
+xq_status xq_mx_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t Kp, void* stream, xq_mx_weights** out) {
+  return mx_prepare_impl(W_host, N, 1, K, Kp, stream, out);
+}
+
+xq_status xq_mx_prepare_weights_heads(const void* W_host, int32_t N, int32_t heads, int32_t head_dim, int32_t head_dim_p, void* stream,
+                                      xq_mx_weights** out) {
+  if (heads < 2) return XQ_ERR_INVALID_ARG;
+  return mx_prepare_impl(W_host, N, heads, head_dim, head_dim_p, stream, out);
+}
+
+int32_t xq_mx_weights_heads(const xq_mx_weights* w) { return w ? w->heads : 0; }
 
 xq_status xq_mx_weights_import(const uint8_t* codes_packed, const uint8_t* scales, int32_t N, int32_t K, int32_t Kp, void* stream,
                                xq_mx_weights** out) {
@@ -894,12 +935,16 @@ xq_status xq_mx_rotate_quant_staged(const void* X, int32_t M, int64_t ldx, const
   cudaError_t e = cudaErrorNotSupported;
   // one kernel: pad, rotate, group exponents, codes and scale blocks straight in the GEMM's layout
   const xq_mx_out mx = {base + L.codes, base + L.sf, w->Kq};
-  if (M >= XQ_ROTATE_ROWS_MIN_M && xq_rotate_mx_supported(w->plan)) e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
-  else if (M < XQ_ROTATE_ROWS_MIN_M) e = xq_launch_rotate_tc_mx(X, M, ldx, w->plan, mx, w->hp_signs, w->sms, st);
-  if (e == cudaErrorNotSupported && xq_rotate_mx_supported(w->plan)) e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
+  if (w->heads > 1) {
+    // head-wise rotation: fp32 rows, then the group quantizer (groups of 32 run along the whole row, across head boundaries)
+  } else if (M >= XQ_ROTATE_ROWS_MIN_M && xq_rotate_mx_supported(w->plan)) {
+    e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
+  } else if (M < XQ_ROTATE_ROWS_MIN_M) {
+    e = xq_launch_rotate_tc_mx(X, M, ldx, w->plan, mx, w->hp_signs, w->sms, st);
+  }
+  if (e == cudaErrorNotSupported && w->heads == 1 && xq_rotate_mx_supported(w->plan)) e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
   if (e == cudaErrorNotSupported) {
-    e = xq_launch_rotate_quant(X, M, ldx, w->plan, base + L.xq, (float*)(base + L.sx), (float*)(base + L.y), nullptr, w->hp_signs, nullptr,
-                               w->sms, st);
+    e = rotate_to_fp32(w, X, M, ldx, base + L.xq, (float*)(base + L.sx), (float*)(base + L.y), st);
     if (e == cudaSuccess)
       e = launch_quantize((const float*)(base + L.y), M, w->Kp, w->Kq, w->Kp, base + L.codes, w->Kq / 2, base + L.sf, nullptr, st);
   }

@@ -42,6 +42,7 @@ EXPORTS = [
     "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
     "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
     "xq_mx_expanded_linear_host", "xq_mx_gemm_staged", "xq_mx_rotate_quant_staged",
+    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads",
 ]
 
 
@@ -94,12 +95,15 @@ def lib() -> ctypes.CDLL:
         L.xq_mx_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_mx_gemm_staged.argtypes = [i32, vp, vp, vp, sz, vp]
         L.xq_mx_rotate_quant_staged.argtypes = [vp, i32, i64, vp, vp, sz, vp]
+        L.xq_mx_prepare_weights_heads.argtypes = [vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.xq_mx_weights_heads.argtypes = [vp]
+        L.xq_mx_weights_heads.restype = i32
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
         for name in EXPORTS:
             if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes", "xq_weights_heads", "xq_mx_weights_free",
-                            "xq_mx_workspace_bytes"):
+                            "xq_mx_workspace_bytes", "xq_mx_weights_heads"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -301,6 +305,7 @@ class MxWeights:
         _check(lib().xq_mx_weights_info(self.handle, ctypes.byref(n), ctypes.byref(k), ctypes.byref(kp), ctypes.byref(pl)),
                "xq_mx_weights_info")
         self.N, self.K, self.Kp, self.plan = n.value, k.value, kp.value, pl
+        self.heads = int(lib().xq_mx_weights_heads(self.handle))
 
     def free(self):
         if self.handle:
@@ -379,3 +384,13 @@ def xq_mx_rotate_quant_staged(X, w: MxWeights, ws, M=None, ldx=None, stream=None
     ldx = X.stride(0) if ldx is None else ldx
     _check(lib().xq_mx_rotate_quant_staged(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(ws), ws.numel() * ws.element_size(),
                                            _stream(stream)), "xq_mx_rotate_quant_staged")
+
+
+def xq_mx_prepare_weights_heads(W_bf16_host: np.ndarray, heads: int, head_dim_p: int, stream=None) -> MxWeights:
+    W = np.ascontiguousarray(W_bf16_host, dtype=np.uint16)
+    N, K = W.shape
+    assert K % heads == 0
+    h = ctypes.c_void_p()
+    _check(lib().xq_mx_prepare_weights_heads(_hp(W), N, heads, K // heads, head_dim_p, _stream(stream), ctypes.byref(h)),
+           "xq_mx_prepare_weights_heads")
+    return MxWeights(h.value)

@@ -210,3 +210,33 @@ def test_mx_full_size_sampled_rows(xq, oracle, tag, M, N, K, Kp, heavy, nsample)
         assert rel_l2(got[i], want[i]) <= E2E_REL_L2, (tag, int(rows[i]))
     codes, sc = xq.xq_mx_weights_export(w)
     check_quantized(oracle, codes, sc, cw, sw)
+
+
+HEADS_CASES = [
+    # (M, N, heads, head_dim, head_dim'): the R2 + R4 setting of the paper's MXFP4 tables -- head-wise rotation, MXFP4 codes;
+    # 72-channel heads make the groups of 32 straddle head boundaries
+    (4, 64, 4, 64, 72), (16, 2048, 32, 64, 72), (200, 384, 32, 64, 80), (130, 256, 32, 128, 144),
+]
+
+
+@pytest.mark.parametrize("M,N,heads,hd,hdp", HEADS_CASES)
+def test_mx_heads_end_to_end(xq, oracle, M, N, heads, hd, hdp):
+    K = heads * hd
+    x = synth.activations(M, K, seed=18, tag=f"mh{M}", heavy_tail=(M > 32))
+    wb = synth.weights(N, K, seed=18, tag=f"mh{N}")
+    w = xq.xq_mx_prepare_weights_heads(wb, heads, hdp)
+    assert (w.N, w.K, w.Kp, w.heads) == (N, K, heads * hdp, heads)
+    opl = oracle.plan(hd, hdp)
+    codes, sc = xq.xq_mx_weights_export(w)
+    _, cw, sw = oracle.rotate_quant_mx(opl, wb, heads)
+    check_quantized(oracle, codes, sc, cw, sw)
+    ws = xq.new_mx_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    xq.xq_mx_expanded_linear(dev(x), w, out, ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    out_ref, _ = oracle.expanded_linear_mx(opl, x, wb, heads)
+    got = synth.bf16_bits_to_f32(host_u16(out))
+    want = synth.bf16_bits_to_f32(out_ref)
+    assert rel_l2(got, want) <= E2E_REL_L2
+    for m in range(M):
+        assert rel_l2(got[m], want[m]) <= E2E_REL_L2

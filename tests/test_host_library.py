@@ -98,6 +98,8 @@ def test_null_arguments_rejected_before_any_cuda_call(xq):
     assert L.xq_mx_expanded_linear_host(null, 4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_mx_gemm_staged(4, null, null, null, 0, null) == xq.ERR_INVALID_ARG
     assert L.xq_mx_rotate_quant_staged(null, 4, 104, null, null, 0, null) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_prepare_weights_heads(null, 8, 4, 64, 72, null, ctypes.byref(out)) == xq.ERR_INVALID_ARG
+    assert L.xq_mx_weights_heads(null) == 0
     L.xq_mx_weights_free(null)
     assert L.xq_poll_status(null, null) == xq.ERR_WORKSPACE
     L.xq_weights_free(null)  # allowed
