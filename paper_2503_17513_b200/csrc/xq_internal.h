@@ -118,7 +118,7 @@ bool xq_rotate_heads_supported(const xq_hadamard_plan_t& pl, int32_t heads);
 size_t xq_head_image_elems(const xq_hadamard_plan_t& pl);
 cudaError_t xq_launch_rotate_heads(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, int32_t heads, uint8_t* Xq,
                                    float* sx, float* Yopt, uint8_t* A8opt, const void* Bimage, int32_t* zp, int sms,
-                                   cudaStream_t st);
+                                   cudaStream_t st, const struct xq_mx_out* mx = nullptr);  // mx: MXFP4 outputs instead (Xq, sx, zp, A8opt unused)
 // The online step of a layer, whichever form its weights were prepared with.
 inline cudaError_t xq_launch_rotate_for(const xq_weights* w, const void* X, int32_t M, int64_t ldx, uint8_t* Xq, float* sx,
                                         uint8_t* A8opt, int32_t* zp, cudaStream_t st);

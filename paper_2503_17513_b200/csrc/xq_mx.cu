@@ -766,9 +766,11 @@ xq_status mx_prepare_impl(const void* W_host, int32_t N, int32_t heads, int32_t 
     // chunk starts are multiples of 128 rows: scale blocks of different chunks do not interleave
     uint8_t* ccodes = w->codes + (size_t)r0 * (w->Kq / 2);
     uint8_t* csf = w->sf + (size_t)(r0 / 128) * (w->Kq / 128) * 512;
-    if (e == cudaSuccess && w->heads == 1 && xq_rotate_mx_supported(w->plan)) {
-      const xq_mx_out mx = {ccodes, csf, w->Kq};
-      e = xq_launch_rotate_mx(dW.p, R, ldw, w->plan, mx, w->sms, st);
+    const xq_mx_out mxo = {ccodes, csf, w->Kq};
+    if (e == cudaSuccess && w->heads > 1) {
+      e = xq_launch_rotate_heads(dW.p, R, ldw, w->plan, w->heads, ccodes, nullptr, nullptr, nullptr, w->head_signs, nullptr, w->sms, st, &mxo);
+    } else if (e == cudaSuccess && xq_rotate_mx_supported(w->plan)) {
+      e = xq_launch_rotate_mx(dW.p, R, ldw, w->plan, mxo, w->sms, st);
     } else if (e == cudaSuccess) {
       e = rotate_to_fp32(w, dW.p, R, ldw, (uint8_t*)dXq.p, (float*)dS.p, (float*)dY.p, st);
       if (e == cudaSuccess) e = launch_quantize((const float*)dY.p, R, Kp, w->Kq, Kp, ccodes, w->Kq / 2, csf, nullptr, st);
@@ -936,7 +938,7 @@ xq_status xq_mx_rotate_quant_staged(const void* X, int32_t M, int64_t ldx, const
   // one kernel: pad, rotate, group exponents, codes and scale blocks straight in the GEMM's layout
   const xq_mx_out mx = {base + L.codes, base + L.sf, w->Kq};
   if (w->heads > 1) {
-    // head-wise rotation: fp32 rows, then the group quantizer (groups of 32 run along the whole row, across head boundaries)
+    e = xq_launch_rotate_heads(X, M, ldx, w->plan, w->heads, mx.codes, nullptr, nullptr, nullptr, w->head_signs, nullptr, w->sms, st, &mx);
   } else if (M >= XQ_ROTATE_ROWS_MIN_M && xq_rotate_mx_supported(w->plan)) {
     e = xq_launch_rotate_mx(X, M, ldx, w->plan, mx, w->sms, st);
   } else if (M < XQ_ROTATE_ROWS_MIN_M) {

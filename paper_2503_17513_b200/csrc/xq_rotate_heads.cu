@@ -34,12 +34,17 @@ __device__ __forceinline__ void group_sync(int group, int HT) {
   else xqptx::bar_sync(1 + group, 32 * HT);
 }
 
-__global__ void __launch_bounds__(kWarps * 32, 2) rotate_quant_heads_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx,
+template <bool MX>
+__global__ void __launch_bounds__(kWarps * 32, MX ? 1 : 2) rotate_quant_heads_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx,
                                                                          xq_hadamard_plan_t pl, int heads, float gamma,
                                                                          uint8_t* __restrict__ Xq, float* __restrict__ sx,
                                                                          float* __restrict__ Yopt, uint8_t* __restrict__ A8opt,
                                                                          const __nv_bfloat16* __restrict__ Bimage,
-                                                                         int32_t* __restrict__ zp, int G) {
+                                                                         int32_t* __restrict__ zp, uint8_t* __restrict__ sfb, int Kq,
+                                                                         int G) {
+  // MX: MXFP4 instead of per-row INT4 -- a shared exponent for every 32 consecutive channels of the whole row
+  // (groups may cross head boundaries), E2M1 codes; Xq then has the row pitch Kq / 2 and the scale bytes go to sfb in
+  // the block layout of the block-scaled GEMM (sx, zp, A8opt unused).
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int d = pl.K, dp = pl.Kp, q = pl.q, n = 1 << pl.log2n;
   const int d16 = (d + 15) / 16 * 16, pitch = d16 + 8;  // bf16 elements per row of both operands (conflict-free 32-bit reads)
@@ -52,7 +57,9 @@ __global__ void __launch_bounds__(kWarps * 32, 2) rotate_quant_heads_kernel(cons
   __nv_bfloat16* Xs_all = Bs + (size_t)dp * pitch;                           // [G][2][H16][pitch]
   uint32_t* outp_all = reinterpret_cast<uint32_t*>(Xs_all + (size_t)G * 2 * H16 * pitch);  // [G][Kp / 8] words
   float* red_all = reinterpret_cast<float*>(outp_all + (size_t)G * (Kp / 8));              // [G][2 HT] + 32 spare
-  int8_t* chi2 = reinterpret_cast<int8_t*>(red_all + 2 * kWarps + 32);
+  float* tmax_all = red_all + 2 * kWarps + 32;                                             // [G][Kp / 8]: largest magnitude per 8-column tile
+  uint8_t* sfs_all = reinterpret_cast<uint8_t*>(tmax_all + (size_t)G * (Kp / 8));            // [G][Kp / 32]: the row's scale bytes
+  int8_t* chi2 = reinterpret_cast<int8_t*>(sfs_all + (size_t)G * (Kp / 32));
   int8_t* sq = chi2 + 2 * q + 1;
 
   xqptx::pdl_launch_dependents();
@@ -132,11 +139,11 @@ __global__ void __launch_bounds__(kWarps * 32, 2) rotate_quant_heads_kernel(cons
         vmax = fmaxf(vmax, acc[j][e]);
         vmin = fminf(vmin, acc[j][e]);
       }
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int o = 16; o > 0 && !MX; o >>= 1) {
       vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, o));
       vmin = fminf(vmin, __shfl_xor_sync(0xffffffffu, vmin, o));
     }
-    if (HT > 1) {
+    if (HT > 1 && !MX) {
       if (lane == 0) {
         red[ht] = vmax;
         red[HT + ht] = vmin;
@@ -148,10 +155,50 @@ __global__ void __launch_bounds__(kWarps * 32, 2) rotate_quant_heads_kernel(cons
       }
     }
     const RowQuant rq = zp ? row_quant_asym(vmin, vmax) : row_quant_sym(fmaxf(vmax, -vmin));
+    if constexpr (MX) {
+      // MXFP4: tile (head h, columns 8 j ..) is tile h NT + j of the row; four consecutive tiles are one group
+      float* tmax = tmax_all + (size_t)group * (Kp / 8);
+      uint8_t* sfs = sfs_all + (size_t)group * (Kp / 32);
+#pragma unroll
+      for (int j = 0; j < kMaxNT; ++j) {
+        if (j < NT) {
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const int h = 16 * ht + g + 8 * r;
+            float m = fmaxf(fabsf(acc[j][2 * r]), fabsf(acc[j][2 * r + 1]));
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+            if (t == 0 && h < heads) tmax[h * NT + j] = m;
+          }
+        }
+      }
+      group_sync(group, HT);
+#pragma unroll
+      for (int j = 0; j < kMaxNT; ++j) {
+        if (j < NT) {
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const int h = 16 * ht + g + 8 * r;
+            const int idx = (h < heads ? h : 0) * NT + j;
+            const float4 q4 = *reinterpret_cast<const float4*>(tmax + (idx & ~3));
+            const int e = mx_shared_exp(fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w)));
+            const float inv = mx_inv_scale(e);
+            uint32_t w = mx_e2m1_pair(acc[j][2 * r] * inv, acc[j][2 * r + 1] * inv) << (8 * t);
+            w |= __shfl_xor_sync(0xffffffffu, w, 1);
+            w |= __shfl_xor_sync(0xffffffffu, w, 2);
+            if (t == 0 && h < heads) {
+              outp[idx] = w;
+              if ((idx & 3) == 0) sfs[idx >> 2] = (uint8_t)(e + 127);
+            }
+          }
+          asm volatile("" ::: "memory");  // keeps the tile-maximum loads of later column tiles from being hoisted (registers)
+        }
+      }
+    }
     // quantize, pack: the quad's four bytes of one (head, column tile) form one word of 8 codes
 #pragma unroll
     for (int j = 0; j < kMaxNT; ++j) {
-      if (j < NT) {
+      if (j < NT && !MX) {
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
           const int h = 16 * ht + g + 8 * r;
@@ -167,11 +214,16 @@ __global__ void __launch_bounds__(kWarps * 32, 2) rotate_quant_heads_kernel(cons
       }
     }
     group_sync(group, HT);
-    if (gtid == 0) {
+    if (gtid == 0 && !MX) {
       sx[row] = rq.s;
       if (zp) zp[row] = rq.z;
     }
-    uint4* dst = reinterpret_cast<uint4*>(Xq + (long long)row * (Kp / 2));
+    if (MX) {  // scale bytes into their blocks; padding up to Kq: unit scales and zero codes (never a NaN scale byte)
+      const uint8_t* sfs = sfs_all + (size_t)group * (Kp / 32);
+      for (int i = gtid; i < Kq / 32; i += gthreads) sfb[xq_mx_sf_offset(row, i, Kq)] = i < Kp / 32 ? sfs[i] : (uint8_t)127;
+      for (int i = gtid; i < (Kq - Kp) / 8; i += gthreads) *reinterpret_cast<uint32_t*>(Xq + (long long)row * (Kq / 2) + Kp / 2 + 4 * i) = 0u;
+    }
+    uint4* dst = reinterpret_cast<uint4*>(Xq + (long long)row * ((MX ? Kq : Kp) / 2));
     for (int i = gtid; i < Kp / 32; i += gthreads) {
       const uint4 v = reinterpret_cast<const uint4*>(outp)[i];
       dst[i] = v;
@@ -194,7 +246,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) rotate_quant_heads_kernel(cons
 
 size_t heads_smem(const xq_hadamard_plan_t& pl, int heads, int G) {
   const int d16 = (pl.K + 15) / 16 * 16, pitch = d16 + 8, H16 = (heads + 15) / 16 * 16;
-  return (size_t)pl.Kp * pitch * 2 + (size_t)G * 2 * H16 * pitch * 2 + (size_t)G * heads * pl.Kp / 2 + (2 * kWarps + 32) * 4 +
+  return (size_t)pl.Kp * pitch * 2 + (size_t)G * 2 * H16 * pitch * 2 + (size_t)G * heads * pl.Kp + (size_t)G * heads * pl.Kp / 32 + (2 * kWarps + 32) * 4 +
          (size_t)(3 * pl.q + 1) + 32;
 }
 
@@ -213,8 +265,12 @@ size_t xq_head_image_elems(const xq_hadamard_plan_t& pl) {
 
 cudaError_t xq_launch_rotate_heads(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, int32_t heads, uint8_t* Xq,
                                    float* sx, float* Yopt, uint8_t* A8opt, const void* Bimage, int32_t* zp, int sms,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, const xq_mx_out* mx) {
   if (!xq_rotate_heads_supported(pl, heads)) return cudaErrorNotSupported;
+  if (mx) {
+    if (((long long)heads * pl.Kp) % 32 != 0) return cudaErrorNotSupported;
+    Xq = mx->codes;
+  }
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
   const int HT = (heads + 15) / 16;
   // token groups per CTA: as many as the warps allow once there are more tokens than multiprocessors
@@ -223,9 +279,10 @@ cudaError_t xq_launch_rotate_heads(const void* X, int32_t M, int64_t ldx, const 
   if (G > want) G = want;
   while (G > 1 && heads_smem(pl, heads, G) > 200 * 1024) --G;
   const size_t smem = heads_smem(pl, heads, G);
-  cudaError_t e = cudaFuncSetAttribute(rotate_quant_heads_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  auto kern = mx ? rotate_quant_heads_kernel<true> : rotate_quant_heads_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int per_sm = smem > 100 * 1024 ? 1 : 2;  // two CTAs fit the register file
+  const int per_sm = (mx || smem > 100 * 1024) ? 1 : 2;  // two CTAs of the INT4 form fit the register file
   const int ctas = (M + G - 1) / G;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(ctas < sms * per_sm ? ctas : sms * per_sm);
@@ -237,6 +294,7 @@ cudaError_t xq_launch_rotate_heads(const void* X, int32_t M, int64_t ldx, const 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, rotate_quant_heads_kernel, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, (int)heads, gamma,
-                            Xq, sx, Yopt, A8opt, (const __nv_bfloat16*)Bimage, zp, G);
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, (int)heads, gamma,
+                            Xq, sx, Yopt, A8opt, (const __nv_bfloat16*)Bimage, zp, mx ? mx->sf_blocks : (uint8_t*)nullptr,
+                            mx ? (int)mx->Kq : 0, G);
 }
