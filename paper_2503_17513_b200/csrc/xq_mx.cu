@@ -36,6 +36,7 @@ struct xq_mx_weights {
   xq_hadamard_plan_t plan;
   uint8_t* codes;    // device, Np * Kq / 2
   uint8_t* sf;       // device, (Np / 128) * (Kq / 128) * 512
+  uint8_t* sf_wide;  // device, the same bytes in the order of 224-channel tiles: ceil(N / 224) * (Kq / 128) * 1024
   uint16_t* hp_signs;
   int device, sms;
 };
@@ -120,15 +121,24 @@ __global__ void mx_from_device_form_kernel(const uint8_t* __restrict__ codes, co
 //   warp 1   MMA issue: copies the scale blocks into tensor memory (tcgen05.cp), then four
 //            tcgen05.mma kind::mxf4 of 128 x 256 x 64; fp32 accumulator of 256 columns
 //   warps 2-5 epilogue: tcgen05.ld, fp32 -> bf16, 16-byte stores
+// The tile is 128 x 256 with one accumulator, or 128 x 224 with two (template argument): see TileCfg.
 // ---------------------------------------------------------------------------------------------
 constexpr int BM = 128, BN = 256;
 constexpr int kStages = 4;
-constexpr int kABytes = BM * 128, kBBytes = BN * 128, kSfaBytes = 1024, kSfbBytes = 2048;
-constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
+constexpr int kABytes = BM * 128, kSfaBytes = 1024, kSfbBytes = 2048;
+// TN = 256: one accumulator of 256 columns (the epilogue of a tile is not hidden).  TN = 224: two accumulators of 224
+// columns, the epilogue of a tile runs under the main loop of the next; the weight scales then come in the
+// 224-channel tile order (xq_mx_weights::sf_wide).  Tensor memory: 2 x 224 + 2 x 32 scale columns = 512.
+template <int TN>
+struct TileCfg {
+  static constexpr int kBBytes = TN * 128;
+  static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // a multiple of 1024 for both
+  static constexpr int kAccBufs = TN == 224 ? 2 : 1;
+  static constexpr int kSfaCol = TN == 224 ? 448 : 256, kSfbCol = kSfaCol + (TN == 224 ? 8 : 16);  // + 32 per stage parity
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+};
 constexpr int kThreads = 6 * 32;
 constexpr int kTmemCols = 512;
-constexpr int kSfaCol = 256, kSfbCol = 272;  // per stage parity: + 32 columns (8 for tokens, 16 for weights)
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
 
 struct MxParams {
   const uint8_t* sfa;  // token scale blocks
@@ -141,8 +151,8 @@ struct MxParams {
 
 // E2M1 operands (format 1 of kind::mxf4) at bits 7-9 and 10-12, both K-major; N >> 3 at bits 17-22; E8M0 scales
 // (bit 23); M >> 4 at bits 24-28; which bytes of the scale columns an instruction reads: bits 4-5 (B), 29-30 (A).
-__device__ __forceinline__ uint32_t mx_idesc(uint32_t sf_id) {
-  return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24) | (sf_id << 4) | (sf_id << 29);
+__device__ __forceinline__ uint32_t mx_idesc_n(uint32_t sf_id, int n) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(128 >> 4) << 24) | (sf_id << 4) | (sf_id << 29);
 }
 // 32 rows of 16 bytes, no swizzle: 8-row groups 128 bytes apart.
 __device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
@@ -161,8 +171,11 @@ __device__ __forceinline__ void umma_mxf4_ss(uint32_t d_tmem, uint64_t adesc, ui
       : "memory");
 }
 
+template <int TN>
 __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                                                               const MxParams p) {
+  using C = TileCfg<TN>;
+  constexpr int kBBytes = C::kBBytes, kStageBytes = C::kStageBytes, kAccBufs = C::kAccBufs;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* base = smem_raw + (((raw + 1023u) & ~1023u) - raw);
@@ -170,8 +183,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
   uint64_t* full = bars;
   uint64_t* empty = full + kStages;
   uint64_t* acc_full = empty + kStages;
-  uint64_t* acc_empty = acc_full + 1;
-  uint64_t* drain = acc_empty + 1;
+  uint64_t* acc_empty = acc_full + 2;
+  uint64_t* drain = acc_empty + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
   volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -183,8 +196,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
     }
-    mbar_init(acc_full, 1);
-    mbar_init(acc_empty, 4);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 4);
+    }
     mbar_init(drain, 1);
     *failed = 0;
     mbar_fence_init();
@@ -218,11 +233,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
           unsigned char* st = base + (size_t)s * kStageBytes;
           mbar_expect_tx(&full[s], kStageBytes);
           tma_load_2d(st, &mapA, kb * 128, tm * BM, &full[s]);
-          tma_load_2d(st + kABytes, &mapB, kb * 128, tn * BN, &full[s]);
+          tma_load_2d(st + kABytes, &mapB, kb * 128, tn * TN, &full[s]);
           const size_t kblocks = (size_t)(p.Kq >> 7);  // scale blocks along K per 128 rows
           bulk_g2s(st + kABytes + kBBytes, p.sfa + ((size_t)tm * kblocks + 2 * kb) * 512, kSfaBytes, &full[s]);
-          bulk_g2s(st + kABytes + kBBytes + kSfaBytes, p.sfb + ((size_t)(2 * tn) * kblocks + 2 * kb) * 512, 1024, &full[s]);
-          bulk_g2s(st + kABytes + kBBytes + kSfaBytes + 1024, p.sfb + ((size_t)(2 * tn + 1) * kblocks + 2 * kb) * 512, 1024, &full[s]);
+          if (TN == 224) {  // tile order: [128-code block][channels 0..127 | 128..223]
+            bulk_g2s(st + kABytes + kBBytes + kSfaBytes, p.sfb + (((size_t)tn * kblocks + 2 * kb) * 2) * 512, kSfbBytes, &full[s]);
+          } else {          // blocks of 128 channels: [channels 0..127 | 128..255][128-code block]
+            bulk_g2s(st + kABytes + kBBytes + kSfaBytes, p.sfb + ((size_t)(2 * tn) * kblocks + 2 * kb) * 512, 1024, &full[s]);
+            bulk_g2s(st + kABytes + kBBytes + kSfaBytes + 1024, p.sfb + ((size_t)(2 * tn + 1) * kblocks + 2 * kb) * 512, 1024, &full[s]);
+          }
         }
         __syncwarp();
       }
@@ -232,8 +251,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
     uint32_t it = 0, tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
-      if (tcount >= 1u) {
-        ok = mbar_wait_bounded(acc_empty, (tcount - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+      const uint32_t buf = kAccBufs == 2 ? (tcount & 1u) : 0u;
+      const uint32_t use = kAccBufs == 2 ? (tcount >> 1) : tcount;  // earlier uses of this accumulator
+      if (use >= 1u) {
+        ok = mbar_wait_bounded(&acc_empty[buf], (use - 1) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
         if (!ok) break;
       }
       tc_fence_after_sync();
@@ -246,23 +267,24 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
           const uint32_t a_addr = smem_u32(base + (size_t)s * kStageBytes);
           const uint32_t sfa_smem = a_addr + kABytes + kBBytes, sfb_smem = sfa_smem + kSfaBytes;
           // scale columns alternate between two sets so that a copy never lands under an MMA still in flight
-          const uint32_t sfa_t = tmem_base + kSfaCol + 32 * (it & 1), sfb_t = tmem_base + kSfbCol + 32 * (it & 1);
+          const uint32_t sfa_t = tmem_base + C::kSfaCol + 32 * (it & 1), sfb_t = tmem_base + C::kSfbCol + 32 * (it & 1);
 #pragma unroll
           for (int j = 0; j < 2; ++j) {  // K halves of 128 codes: 4 token columns, 8 weight columns each
             tmem_cp_32x128b_warpx4(sfa_t + 4 * j, sf_desc(sfa_smem + 512 * j));
-            tmem_cp_32x128b_warpx4(sfb_t + 8 * j, sf_desc(sfb_smem + 512 * j));             // channels 0..127 of the tile
-            tmem_cp_32x128b_warpx4(sfb_t + 8 * j + 4, sf_desc(sfb_smem + 1024 + 512 * j));  // channels 128..255
+            // channels 0..127 of the tile, then the rest
+            tmem_cp_32x128b_warpx4(sfb_t + 8 * j, sf_desc(sfb_smem + (TN == 224 ? 1024 * j : 512 * j)));
+            tmem_cp_32x128b_warpx4(sfb_t + 8 * j + 4, sf_desc(sfb_smem + (TN == 224 ? 1024 * j + 512 : 1024 + 512 * j)));
           }
           const uint64_t adesc = umma_desc_k128(a_addr), bdesc = umma_desc_k128(a_addr + kABytes);
 #pragma unroll
           for (int k = 0; k < 4; ++k)  // 64 codes = 32 bytes per instruction; its two scale bytes: 0-1 or 2-3 of the column
-            umma_mxf4_ss(tmem_base, adesc + 2 * k, bdesc + 2 * k, mx_idesc(2u * (k & 1)), (kb | k) != 0 ? 1u : 0u, sfa_t + 4 * (k >> 1),
-                         sfb_t + 8 * (k >> 1));
+            umma_mxf4_ss(tmem_base + buf * TN, adesc + 2 * k, bdesc + 2 * k, mx_idesc_n(2u * (k & 1), TN), (kb | k) != 0 ? 1u : 0u,
+                         sfa_t + 4 * (k >> 1), sfb_t + 8 * (k >> 1));
           umma_commit(&empty[s]);
         }
         __syncwarp();
       }
-      if (ok && lane == 0) umma_commit(acc_full);
+      if (ok && lane == 0) umma_commit(&acc_full[buf]);
       __syncwarp();
     }
     if (lane == 0) umma_commit(drain);
@@ -275,13 +297,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
       const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-      const int m = tm * BM + q * 32 + lane, n0 = tn * BN;
-      ok = mbar_wait_bounded(acc_full, tcount & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
+      const int m = tm * BM + q * 32 + lane, n0 = tn * TN;
+      const uint32_t buf = kAccBufs == 2 ? (tcount & 1u) : 0u;
+      const uint32_t use = kAccBufs == 2 ? (tcount >> 1) : tcount;
+      ok = mbar_wait_bounded(&acc_full[buf], use & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * TN;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int c = 0; c < TN / 32; ++c) {
         uint32_t v[32];
         tmem_ld_32x32(taddr + c * 32, v);
         tmem_ld_wait();
@@ -305,7 +329,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty);
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
   }
 
@@ -318,6 +342,25 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Weight scales in the order of 224-channel tiles (what the 224-column tile kernel copies): per tile and 128-code
+// block two blocks of 32 x 16 bytes, channels 0..127 and 128..223 of the tile.
+// ---------------------------------------------------------------------------------------------
+constexpr int WN = 224;
+
+__host__ __device__ inline size_t sf_wide_offset(int n, int g, int Kq) {
+  const int tile = n / WN, r = n - tile * WN, atom = r >> 7, ra = r & 127;
+  return (((size_t)tile * (Kq >> 7) + (g >> 2)) * 2 + atom) * 512 + (size_t)(ra & 31) * 16 + (size_t)(ra >> 5) * 4 + (g & 3);
+}
+
+__global__ void mx_sf_to_wide_kernel(const uint8_t* __restrict__ sf_blocks, int N, int Kq, uint8_t* __restrict__ sf_wide) {
+  const long long total = (long long)N * (Kq / 32);
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int n = (int)(i / (Kq / 32)), g = (int)(i % (Kq / 32));
+    sf_wide[sf_wide_offset(n, g, Kq)] = sf_blocks[xq_mx_sf_offset(n, g, Kq)];
   }
 }
 
@@ -346,10 +389,6 @@ struct MxDecodeParams {
   int32_t* status;
   int M, N, KB, Kq, S;
 };
-
-__device__ __forceinline__ uint32_t mx_idesc_n(uint32_t sf_id, int n) {
-  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(128 >> 4) << 24) | (sf_id << 4) | (sf_id << 29);
-}
 
 __global__ void __launch_bounds__(kThreads, 1) gemm_mx_decode_kernel(const __grid_constant__ CUtensorMap mapW,
                                                                      const __grid_constant__ CUtensorMap mapX, const MxDecodeParams p) {
@@ -594,14 +633,14 @@ cudaError_t launch_gemm_decode(const uint8_t* codes, const uint8_t* sfx, int M, 
   return cudaLaunchKernelEx(&cfg, gemm_mx_decode_kernel, mapW, mapX, p);
 }
 
-// codes / scale blocks of the tokens in device form -> out
-cudaError_t launch_gemm(const uint8_t* codes, const uint8_t* sfa, int M, const xq_mx_weights* w, void* out, int32_t* status,
-                        cudaStream_t st) {
+template <int TN>
+cudaError_t launch_gemm_tn(const uint8_t* codes, const uint8_t* sfa, int M, const xq_mx_weights* w, void* out, int32_t* status,
+                           cudaStream_t st) {
   CUtensorMap mapA, mapB;
-  if (!make_map(&mapA, codes, M, w->Kq, BM) || !make_map(&mapB, w->codes, w->Np, w->Kq, BN)) return cudaErrorInvalidValue;
+  if (!make_map(&mapA, codes, M, w->Kq, BM) || !make_map(&mapB, w->codes, w->Np, w->Kq, TN)) return cudaErrorInvalidValue;
   MxParams p;
   p.sfa = sfa;
-  p.sfb = w->sf;
+  p.sfb = TN == 224 ? w->sf_wide : w->sf;
   p.out = (__nv_bfloat16*)out;
   p.status = status;
   p.M = M;
@@ -609,13 +648,28 @@ cudaError_t launch_gemm(const uint8_t* codes, const uint8_t* sfa, int M, const x
   p.Kq = w->Kq;
   p.KB = w->Kq / 256;
   p.tiles_m = (M + BM - 1) / BM;
-  p.tiles_n = (w->N + BN - 1) / BN;
-  cudaError_t e = cudaFuncSetAttribute(gemm_mx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  p.tiles_n = (w->N + TN - 1) / TN;
+  constexpr size_t smem = TileCfg<TN>::kSmemBytes;
+  cudaError_t e = cudaFuncSetAttribute(gemm_mx_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int tiles = p.tiles_m * p.tiles_n;
   cudaLaunchAttribute attr[1];
-  cudaLaunchConfig_t cfg = pdl_config(dim3(tiles < w->sms ? tiles : w->sms), dim3(kThreads), kSmemBytes, st, attr);
-  return cudaLaunchKernelEx(&cfg, gemm_mx_kernel, mapA, mapB, p);
+  cudaLaunchConfig_t cfg = pdl_config(dim3(tiles < w->sms ? tiles : w->sms), dim3(kThreads), smem, st, attr);
+  return cudaLaunchKernelEx(&cfg, gemm_mx_kernel<TN>, mapA, mapB, p);
+}
+
+// codes / scale blocks of the tokens in device form -> out.  Two tile shapes; a simple cost model picks one: waves of
+// tiles over the multiprocessors times the tensor-core cycles of a tile's main loop (128 per 128 x 256 x 64 MMA, scaled
+// with the tile), plus the epilogue where it is not hidden behind the next tile (about 1500 cycles).
+cudaError_t launch_gemm(const uint8_t* codes, const uint8_t* sfa, int M, const xq_mx_weights* w, void* out, int32_t* status,
+                        cudaStream_t st) {
+  const int KB = w->Kq / 256, sms = w->sms, N = w->N;
+  auto waves = [&](int tiles) { return (double)((tiles + sms - 1) / sms); };
+  const int tm = (M + 127) / 128;
+  const double t256 = waves(tm * ((N + 255) / 256)) * (KB * 512.0 + 1500.0);
+  const double t224 = waves(tm * ((N + 223) / 224)) * (KB * 448.0) + 1500.0;
+  if (t224 <= t256) return launch_gemm_tn<224>(codes, sfa, M, w, out, status, st);
+  return launch_gemm_tn<256>(codes, sfa, M, w, out, status, st);
 }
 
 // Workspace: header (status word) | rotated rows fp32 | codes | scale blocks | scratch outputs of the rotate kernel.
@@ -688,6 +742,7 @@ xq_status make_mx_weights(int32_t N, int32_t K, int32_t Kp, xq_mx_weights** out,
   w->head_signs = nullptr;
   w->codes = nullptr;
   w->sf = nullptr;
+  w->sf_wide = nullptr;
   w->hp_signs = nullptr;
   if (cudaGetDevice(&w->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&w->sms, cudaDevAttrMultiProcessorCount, w->device) != cudaSuccess) {
@@ -695,7 +750,9 @@ xq_status make_mx_weights(int32_t N, int32_t K, int32_t Kp, xq_mx_weights** out,
     return XQ_ERR_CUDA;
   }
   const size_t cb = (size_t)w->Np * (w->Kq / 2), sb = sf_bytes(w->Np, w->Kq);
+  const size_t swb = (size_t)((N + WN - 1) / WN) * (w->Kq / 128) * 1024;
   if (cudaMalloc((void**)&w->codes, cb) != cudaSuccess || cudaMalloc((void**)&w->sf, sb) != cudaSuccess ||
+      cudaMalloc((void**)&w->sf_wide, swb) != cudaSuccess || cudaMemset(w->sf_wide, 127, swb) != cudaSuccess ||
       cudaMemset(w->codes, 0, cb) != cudaSuccess || cudaMemset(w->sf, 127, sb) != cudaSuccess ||
       !(heads > 1 ? xq_make_head_signs(pl, &w->head_signs) : xq_make_hp_signs(pl, &w->hp_signs))) {
     cudaGetLastError();
@@ -714,6 +771,7 @@ void xq_mx_weights_free(xq_mx_weights* w) {
   if (!w) return;
   if (w->codes) cudaFree(w->codes);
   if (w->sf) cudaFree(w->sf);
+  if (w->sf_wide) cudaFree(w->sf_wide);
   if (w->hp_signs) cudaFree(w->hp_signs);
   if (w->head_signs) cudaFree(w->head_signs);
   delete w;
@@ -776,6 +834,10 @@ xq_status mx_prepare_impl(const void* W_host, int32_t N, int32_t heads, int32_t 
       if (e == cudaSuccess) e = launch_quantize((const float*)dY.p, R, Kp, w->Kq, Kp, ccodes, w->Kq / 2, csf, nullptr, st);
     }
   }
+  if (e == cudaSuccess) {
+    mx_sf_to_wide_kernel<<<148 * 4, 256, 0, st>>>(w->sf, w->N, w->Kq, w->sf_wide);
+    e = cudaGetLastError();
+  }
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -824,6 +886,10 @@ xq_status xq_mx_weights_import(const uint8_t* codes_packed, const uint8_t* scale
   if (e == cudaSuccess) e = cudaMemcpyAsync(dS.p, scales, (size_t)N * (Kp / 32), cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) {
     mx_to_device_form_kernel<<<148 * 4, 256, 0, st>>>((const uint8_t*)dC.p, (const uint8_t*)dS.p, N, Kp, w->Kq, w->codes, w->sf);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) {
+    mx_sf_to_wide_kernel<<<148 * 4, 256, 0, st>>>(w->sf, w->N, w->Kq, w->sf_wide);
     e = cudaGetLastError();
   }
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
