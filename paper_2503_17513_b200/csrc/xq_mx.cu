@@ -115,13 +115,13 @@ __global__ void mx_from_device_form_kernel(const uint8_t* __restrict__ codes, co
 }
 
 // ---------------------------------------------------------------------------------------------
-// Product.  Tile: 128 tokens x 256 channels, K in blocks of 256 codes (one 128-byte row piece).
-//   warp 0   producer: per stage two TMA tiles (tokens 16 KiB, weights 32 KiB) and three bulk
-//            copies of scale blocks (tokens 1 KiB, weights 2 x 1 KiB)
+// Product.  Tile: 128 tokens x TN channels (TN = 224 or 256, see TileCfg), K in blocks of 256 codes
+// (one 128-byte row piece).
+//   warp 0   producer: per stage two TMA tiles (tokens 16 KiB, weights TN x 128 bytes) and the
+//            scale blocks as bulk copies (tokens 1 KiB, weights 2 KiB)
 //   warp 1   MMA issue: copies the scale blocks into tensor memory (tcgen05.cp), then four
-//            tcgen05.mma kind::mxf4 of 128 x 256 x 64; fp32 accumulator of 256 columns
+//            tcgen05.mma kind::mxf4 of 128 x TN x 64; fp32 accumulators of TN columns
 //   warps 2-5 epilogue: tcgen05.ld, fp32 -> bf16, 16-byte stores
-// The tile is 128 x 256 with one accumulator, or 128 x 224 with two (template argument): see TileCfg.
 // ---------------------------------------------------------------------------------------------
 constexpr int BM = 128, BN = 256;
 constexpr int kStages = 4;
