@@ -35,22 +35,25 @@ using namespace xqptx;
 
 namespace {
 
-constexpr int BMH = 128, BN = 256;                           // rows of one accumulator, columns
+constexpr int BMH = 128;                                     // rows of one accumulator
 constexpr int kPkStages = 4;
-constexpr int kPkBBytes = BN * 64;                           // packed weights of a K block: 16 KiB
-constexpr int kI8ABytes = BMH * 128, kI8BBytes = BN * 128;   // expanded: 16 KiB per 128 tokens, 32 KiB
+constexpr int kI8ABytes = BMH * 128;                         // expanded tokens: 16 KiB per 128 tokens
 constexpr int kUnpackWarps = 8;
 constexpr int kFirstEpiWarp = 4;
 constexpr int kTmemCols = 512;
 
-template <int MH>
+// MH accumulators of 128 tokens x BN channels per tile.  (1, 256) and (2, 128) use half of tensor memory per tile and
+// double-buffer it (the epilogue of a tile overlaps the main loop of the next); (2, 256) uses all 512 columns.
+template <int MH, int BN>
 struct Cfg {
-  static constexpr int kI8Stages = MH == 1 ? 3 : 2;
+  static constexpr int kPkBBytes = BN * 64;    // packed weights of a K block
+  static constexpr int kI8BBytes = BN * 128;   // expanded
   static constexpr int kI8StageBytes = MH * kI8ABytes + kI8BBytes;
+  static constexpr int kI8Stages = kI8StageBytes <= 48 * 1024 ? 3 : 2;
   static constexpr int kEpiWarps = 4 * MH;
   static constexpr int kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
   static constexpr int kThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;
-  static constexpr int kAccBufs = MH == 1 ? 2 : 1;
+  static constexpr int kAccBufs = MH * BN <= 256 ? 2 : 1;
   static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kI8Stages * kI8StageBytes + (size_t)kPkStages * kPkBBytes +
                                        kEpiWarps * 2 * BN * sizeof(float) /*scales, code sums*/ + 256 /*barriers, flags*/;
 };
@@ -82,10 +85,10 @@ __device__ __forceinline__ void expand_store(const uint4 v, unsigned char* tile,
   *reinterpret_cast<uint4*>(row + (((2 * j + 1) ^ x) << 4)) = hi;
 }
 
-template <int MH>
-__global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap mapA, const PrefillParams p) {
-  using C = Cfg<MH>;
-  constexpr int kI8Stages = C::kI8Stages, kI8StageBytes = C::kI8StageBytes, kAccBufs = C::kAccBufs;
+template <int MH, int BN>
+__global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap mapA, const PrefillParams p) {
+  using C = Cfg<MH, BN>;
+  constexpr int kI8Stages = C::kI8Stages, kI8StageBytes = C::kI8StageBytes, kAccBufs = C::kAccBufs, kPkBBytes = C::kPkBBytes;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* base = smem_raw + (((raw + 1023u) & ~1023u) - raw);
@@ -152,7 +155,7 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
         unsigned char* stage = pk + (size_t)s * kPkBBytes;
         if (lane == 0) mbar_expect_tx(&pk_full[s], kPkBBytes);
         __syncwarp();
-        if (lane < 16) bulk_g2s(stage + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
+        if (lane < BN / XQ_ROW_BLOCK) bulk_g2s(stage + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
       }
     }
   } else if (warp == 1) {
@@ -179,7 +182,7 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
 #pragma unroll
           for (int h = 0; h < MH; ++h) {
             const uint64_t adesc = umma_desc_k128(a_addr + h * kI8ABytes);
-            const uint32_t d_tmem = tmem_base + (kAccBufs == 2 ? buf : (uint32_t)h) * BN;
+            const uint32_t d_tmem = tmem_base + (buf * MH + (uint32_t)h) * BN;
 #pragma unroll
             for (int k = 0; k < 4; ++k) umma_i8_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
@@ -242,7 +245,7 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
       ok = mbar_wait_bounded(&acc_full[buf], use & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (kAccBufs == 2 ? buf : (uint32_t)eh) * BN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (buf * MH + (uint32_t)eh) * BN;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t v[32];
@@ -296,7 +299,7 @@ __global__ void __launch_bounds__(Cfg<MH>::kThreads, 1) gemm_prefill_kernel(cons
         // 16 channel blocks of 1 KiB, piece 16t + r of a block = codes 32t..32t+31 of channel r
         const unsigned char* src = pk + (size_t)s * kPkBBytes;
         unsigned char* dstB = i8 + (size_t)u * kI8StageBytes + MH * kI8ABytes;
-        constexpr int kPieces = BN * 4 / (kUnpackWarps * 32);  // 16-byte pieces per thread: 4
+        constexpr int kPieces = BN * 4 / (kUnpackWarps * 32);  // 16-byte pieces per thread
         uint4 v[kPieces];
 #pragma unroll
         for (int i = 0; i < kPieces; ++i) v[i] = *reinterpret_cast<const uint4*>(src + (size_t)(ut + i * kUnpackWarps * 32) * 16);
@@ -361,11 +364,12 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-template <int MH>
+template <int MH, int BN>
 cudaError_t launch_mh(const CUtensorMap& mapA, PrefillParams p, int sms, cudaStream_t st) {
-  using C = Cfg<MH>;
+  using C = Cfg<MH, BN>;
   p.tiles_m = (p.M + MH * BMH - 1) / (MH * BMH);
-  cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel<MH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+  p.tiles_n = (p.N + BN - 1) / BN;
+  cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel<MH, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int tiles = p.tiles_m * p.tiles_n;
   cudaLaunchConfig_t cfg = {};
@@ -378,13 +382,13 @@ cudaError_t launch_mh(const CUtensorMap& mapA, PrefillParams p, int sms, cudaStr
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_prefill_kernel<MH>, mapA, p);
+  return cudaLaunchKernelEx(&cfg, gemm_prefill_kernel<MH, BN>, mapA, p);
 }
 
 }  // namespace
 
 bool xq_prefill_supported(int32_t M, const xq_weights* w) {
-  return M >= 1 && w->Kp % 32 == 0 && w->N % 8 == 0 && w->Np % BN == 0;
+  return M >= 1 && w->Kp % 32 == 0 && w->N % 8 == 0 && w->Np % 256 == 0;
 }
 
 cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, uint8_t* A8, cudaStream_t st) {
@@ -427,11 +431,17 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int
   p.M = M;
   p.N = w->N;
   p.KB = w->Kpp / XQ_K_BLOCK;
-  p.tiles_n = (w->N + BN - 1) / BN;
+  p.tiles_n = 0;
   p.tiles_m = 0;
-  // 256-token tiles halve the weight expansion per MMA but leave fewer, coarser tiles: take them
-  // when they still fill the machine at least twice
-  const int tiles2 = ((M + 2 * BMH - 1) / (2 * BMH)) * p.tiles_n;
-  if (5 * tiles2 >= 3 * sms) return launch_mh<2>(mapA, p, sms, st);
-  return launch_mh<1>(mapA, p, sms, st);
+  // Three tile shapes; a cost model picks one: waves of tiles over the multiprocessors times the cycles of a tile
+  // (69 tensor-core cycles per 128 x 256 x 32 MMA; 128-token tiles expand every weight for half as many MMAs and run
+  // at about 0.62 of that rate; an epilogue that is not hidden costs about 2000 cycles).
+  const int KB = p.KB, tm1 = (M + BMH - 1) / BMH, tm2 = (M + 2 * BMH - 1) / (2 * BMH);
+  auto waves = [&](int tiles) { return (double)((tiles + sms - 1) / sms); };
+  const double t_1x256 = waves(tm1 * ((w->N + 255) / 256)) * (KB * 276.0 / 0.62);
+  const double t_2x256 = waves(tm2 * ((w->N + 255) / 256)) * (KB * 552.0 + 2000.0);
+  const double t_2x128 = waves(tm2 * ((w->N + 127) / 128)) * (KB * 276.0 / 0.80);  // N = 128 MMAs re-read the tokens twice as often
+  if (t_2x128 <= t_2x256 && t_2x128 <= t_1x256) return launch_mh<2, 128>(mapA, p, sms, st);
+  if (t_2x256 <= t_1x256) return launch_mh<2, 256>(mapA, p, sms, st);
+  return launch_mh<1, 256>(mapA, p, sms, st);
 }
