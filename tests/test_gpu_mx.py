@@ -240,3 +240,38 @@ def test_mx_heads_end_to_end(xq, oracle, M, N, heads, hd, hdp):
     assert rel_l2(got, want) <= E2E_REL_L2
     for m in range(M):
         assert rel_l2(got[m], want[m]) <= E2E_REL_L2
+
+
+def test_mx_edge_rows(xq, oracle):
+    """A zero row (unit scale bytes, zero codes), a single spike (every rotated value has the same magnitude: all
+    codes +-4 under one shared exponent), tiny and large magnitudes; few rows and many rows (both rotate kernels)."""
+    K, Kp = 2048, 2176
+    x = synth.activations(64, K, seed=19)
+    x[1] = 0
+    x[2] = 0
+    x[2, 5] = synth.f32_to_bf16_bits(np.array([3.0], dtype=np.float32))[0]
+    x[3] = synth.f32_to_bf16_bits((synth.bf16_bits_to_f32(x[3]) * 1e-30).astype(np.float32))
+    x[4] = synth.f32_to_bf16_bits((synth.bf16_bits_to_f32(x[4]) * 1e30).astype(np.float32))
+    pl = xq.xq_hadamard_plan(K, Kp)
+    opl = oracle.plan(K, Kp)
+    wb = synth.weights(64, K, seed=19, tag="edge")
+    w = xq.xq_mx_prepare_weights(wb, Kp)
+    for M in (6, 64):
+        codes = torch.empty((M, Kp // 2), dtype=torch.uint8, device="cuda")
+        sc = torch.empty((M, Kp // 32), dtype=torch.uint8, device="cuda")
+        Y = torch.empty((M, Kp), dtype=torch.float32, device="cuda")
+        xq.xq_mx_rotate_quant(dev(x[:M]), pl, codes, sc, Y)
+        c, s = unpack(codes.cpu().numpy()), sc.cpu().numpy()
+        _, c_ref, s_ref = oracle.rotate_quant_mx(opl, x[:M])
+        assert np.all(s[1] == 127) and not c[1].any()
+        assert len(set(s[2])) == 1 and set(np.unique(c[2] & 7)) == {6}   # |value| / 2^e = 4 everywhere
+        check_quantized(oracle, c, s, c_ref, s_ref)
+        # the fused kernels (layer call) see the same rows: outputs against the oracle, row by row
+        ws = xq.new_mx_workspace(M, w)
+        out = torch.empty((M, 64), dtype=torch.int16, device="cuda")
+        xq.xq_mx_expanded_linear(dev(x[:M]), w, out, ws)
+        got = synth.bf16_bits_to_f32(host_u16(out)).astype(np.float64)
+        want = synth.bf16_bits_to_f32(oracle.expanded_linear_mx(opl, x[:M], wb)[0]).astype(np.float64)
+        assert not got[1].any()
+        for m in range(M):
+            assert rel_l2(got[m], want[m]) <= E2E_REL_L2, m
