@@ -439,18 +439,19 @@ __global__ void unpack_codes_kernel(const uint8_t* __restrict__ packed, long lon
   }
 }
 
-// One thread per row of the block layout: the sum of its K'' signed nibbles (padding holds zeros).
+// One warp per row of the block layout: the sum of its K'' signed nibbles (padding holds zeros).
 __global__ void weight_sums_kernel(const uint8_t* __restrict__ blocks, int Np, int Kpp, int32_t* __restrict__ w_sum) {
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (n >= Np) return;
   const int k_groups = Kpp / XQ_K_GROUP;
   int acc = 0;
-  for (int kg = 0; kg < Kpp / 8; ++kg) {
+  for (int kg = lane; kg < Kpp / 8; kg += 32) {
     const uint32_t w = *reinterpret_cast<const uint32_t*>(blocks + xq_weight_word_offset(n, kg, k_groups));
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc += (int)(w << (28 - 4 * i)) >> 28;
   }
-  w_sum[n] = acc;
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) w_sum[n] = acc;
 }
 
 inline int grid_for(long long work, int threads) {
@@ -521,7 +522,7 @@ cudaError_t xq_launch_relayout_from_blocks(const uint8_t* blocks, int32_t Np, in
 }
 
 cudaError_t xq_launch_weight_sums(const uint8_t* blocks, int32_t Np, int32_t Kpp, int32_t* w_sum, cudaStream_t st) {
-  weight_sums_kernel<<<(Np + 127) / 128, 128, 0, st>>>(blocks, Np, Kpp, w_sum);
+  weight_sums_kernel<<<(Np + 3) / 4, 128, 0, st>>>(blocks, Np, Kpp, w_sum);
   return cudaGetLastError();
 }
 
