@@ -155,17 +155,17 @@ def rotate_bytes(M, K, Kp):
 
 def run_reference(args, table, layers, M, heavy):
     """CPU oracle on the host cores.  A step is a bounded sample of the workload -- the online path of
-    ONE layer's linears for min(M, 8) tokens and min(N, 128) output channels per linear (weights prepared
+    ONE layer's linears for min(M, 32) tokens and min(N, 512) output channels per linear (weights prepared
     beforehand, as on the GPU) -- so that K steps end within minutes whatever K is; tokens/s is scaled
     linearly to all layers, all tokens and all channels (the path is independent per token and channel)."""
     import oracle
 
     oracle.build()
-    Ms = min(M, 8)
+    Ms = min(M, 32)  # the same sample as the cpu_baseline leg: smaller ones let fixed call overheads dominate the scaled time
     prepared = {}
     xs = {}
     for name, (K, Kp, N, *hh) in table.items():
-        Ns = min(N, 128)
+        Ns = min(N, 512)
         heads = hh[0] if hh else 1
         pl = oracle.plan(K // heads, Kp // heads)
         xs[name] = synth.activations(Ms, K, seed=0, tag=name, heavy_tail=heavy)
@@ -210,7 +210,7 @@ def run_reference(args, table, layers, M, heavy):
     t_layer = sum(times) / len(times)
     t_step = t_layer * layers * (M / Ms)
     value = M / t_step
-    sample = (f"{len(times)} timed steps; per step: online path of one layer's linears for {Ms} tokens and up to 128 output channels per linear "
+    sample = (f"{len(times)} timed steps; per step: online path of one layer's linears for {Ms} tokens and up to 512 output channels per linear "
               f"(GEMM time scaled to full N), scaled to {layers} layers and M={M}")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": len(times),
