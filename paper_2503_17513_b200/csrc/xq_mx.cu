@@ -684,6 +684,7 @@ int mx_decode_splits(const xq_mx_weights* w) {
   if (S < 1) S = 1;
   if (S > KB) S = KB;
   if (S > 3) S = 3;  // the last CTA of a tile adds S partial tiles one after the other: few, long slices
+  if (KB <= kDStages + 1) S = 1;  // the whole K fits the stages requested before the tokens arrive: nothing to gain from slices
   if (tiles > (int)((XQ_WS_COUNTER_BYTES - XQ_WS_HEADER_BYTES) / 4)) S = 1;  // one counter per tile
   return S;
 }
