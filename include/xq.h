@@ -21,7 +21,10 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls taking a
  *    stream only enqueue work; they do not synchronize unless stated.
  *  - bf16 tensors are raw 16-bit patterns.  Device pointers must be 16-byte aligned.
- *  - No global state: calls on distinct streams with distinct workspaces may run concurrently.
+ *  - The device that was current when a weights object was made must be current in every call
+ *    that takes the object (XQ_ERR_INVALID_ARG otherwise).
+ *  - No global state, except in xq_expanded_linear_static (see there): calls on distinct streams
+ *    with distinct workspaces may run concurrently.
  */
 #ifndef XQ_H_
 #define XQ_H_
@@ -241,9 +244,14 @@ xq_status xq_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_w
  *
  * Here the intermediate results (packed INT4 codes of the M tokens, their M scales, the status
  * word) are kept in a fixed 4 MiB array that is part of the library image; every GPU on which
- * the library is used holds those 4 MiB until the process exits.  The call itself performs no
- * allocation of any kind: it looks up the array, clears the status word and enqueues the same
- * two kernels as xq_expanded_linear on `stream`.
+ * the library is used holds those 4 MiB until the process exits.  The call asks for no memory,
+ * neither from the CUDA allocator nor from the host heap: it looks up the array, clears the status
+ * word and enqueues the same two kernels as xq_expanded_linear on `stream`.  What the CUDA
+ * runtime does by itself the first time a kernel of the library runs on a device (loading the
+ * module, which is also when the 4 MiB array comes into being) happens in the first call; so do
+ * an occupancy query and a driver entry-point lookup whose answers the library keeps (behind two
+ * short host mutexes that every later call also takes for a table lookup).  From the second
+ * call for a given token-count class on a device, the amount of free device memory no longer moves.
  *
  * Limit: 256 + roundup256(M * Kp / 2) + roundup256(4 * M) bytes, plus roundup256(M * Kp) when
  * M > 32, must fit in 4 MiB (about 1280 tokens at Kp = 2176, 180 at Kp = 15360); larger calls
@@ -261,6 +269,15 @@ xq_status xq_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_w
 xq_status xq_expanded_linear_static(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w,
                                     void* out_bf16_dev, void* stream);
 
+/* Diagnostic, host only, nothing is launched (no counterpart in the paper): which kernel the quantized
+ * product of M tokens against w runs in, and its tile.  *kind = 0: the split-K weight-stream kernel
+ * of M <= 32 tokens (tile_tokens = tokens padded to 8, 16 or 32; tile_channels = 16); 1: the
+ * tcgen05 tile kernel (tile_tokens x tile_channels one of 128 x 256, 256 x 256, 256 x 128); 2: the
+ * one-thread-per-output kernel (1 x 1).  Tests use it to name the tile shape a case exercised.
+ * Errors: INVALID_ARG (null pointer, M < 1, wrong current device), CUDA. */
+xq_status xq_gemm_kernel_info(int32_t M, const xq_weights* w, int32_t* kind, int32_t* tile_tokens,
+                              int32_t* tile_channels);
+
 /* Synchronizes `stream` and returns the sticky device status stored in the workspace (XQ_OK,
  * XQ_ERR_TIMEOUT or XQ_ERR_BOUNDS), or XQ_ERR_CUDA if the stream itself reports an error. */
 xq_status xq_poll_status(const void* ws_dev, void* stream);
@@ -271,6 +288,15 @@ xq_status xq_poll_status(const void* ws_dev, void* stream);
  * the workspace status word and returns normally; xq_poll_status then reports XQ_ERR_TIMEOUT and
  * the CUDA context stays usable.  xq_workspace_init clears the status again. */
 xq_status xq_selftest_wait_timeout(void* ws_dev, size_t ws_bytes, void* stream);
+
+/* Measurement aid (no counterpart in the paper): enqueues one kernel in which every multiprocessor
+ * issues iters * 4 tensor-core instructions of the kind the prefill product uses
+ * (tcgen05.mma kind::i8, 128 x 256 x 32, operands resident in shared memory, no loads, no unpacking)
+ * and returns in *ops_out (optional) the integer operations that launch performs, 2 per
+ * multiply-add.  Timed with events by the caller, this gives the INT8 issue rate of the tensor pipe
+ * on the device at hand: the ceiling the prefill kernel is measured against.  1 <= iters <= 2^22.
+ * ws: any initialised workspace (status word for the bounded wait). */
+xq_status xq_selftest_i8_mma_rate(int32_t iters, void* ws_dev, size_t ws_bytes, void* stream, double* ops_out);
 
 const char* xq_status_string(xq_status s);
 

@@ -328,7 +328,7 @@ xq_status xq_weights_import(const int8_t* codes, const float* s_w, int32_t N, in
 }
 
 xq_status xq_weights_export(const xq_weights* w, int8_t* codes, float* s_w) {
-  if (!w || !codes || !s_w) return XQ_ERR_INVALID_ARG;
+  if (!w || !codes || !s_w || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   const size_t count = (size_t)w->N * w->Kp;
   DevBuf dCodes, dCanon;
   if (dCodes.alloc(count) != cudaSuccess || dCanon.alloc(count / 2) != cudaSuccess) {
@@ -404,7 +404,7 @@ xq_status gemm_impl(const uint8_t* Xq, const float* s_x, const int32_t* zp, bool
                     int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!Xq || !s_x || !out || (asym && !zp)) return XQ_ERR_INVALID_ARG;
+  if (!Xq || !s_x || !out || (asym && !zp) || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   if (zp && (reinterpret_cast<uintptr_t>(zp) & 3u)) return XQ_ERR_INVALID_ARG;
   if (!aligned16(Xq) || !aligned16(out) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
       (acc_opt && !aligned16(acc_opt)))
@@ -422,7 +422,7 @@ xq_status linear_impl(const void* X, int32_t M, int64_t ldx, const xq_weights* w
                       size_t ws_bytes, void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!X || !out) return XQ_ERR_INVALID_ARG;
+  if (!X || !out || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   if (ldx < w->K || (ldx % 8) != 0 || !aligned16(X) || !aligned16(out)) return XQ_ERR_INVALID_ARG;
   const xq_ws_layout L = xq_ws_compute(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
@@ -488,7 +488,7 @@ xq_status linear_host_impl(const void* X_host, int32_t M, const xq_weights* w, b
                            size_t ws_bytes, void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!X_host || !out_host) return XQ_ERR_INVALID_ARG;
+  if (!X_host || !out_host || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   const xq_ws_layout L = xq_ws_compute(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
   uint8_t* base = (uint8_t*)ws;
@@ -532,6 +532,22 @@ xq_status xq_selftest_wait_timeout(void* ws, size_t ws_bytes, void* stream) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
   }
+  return XQ_OK;
+}
+
+xq_status xq_selftest_i8_mma_rate(int32_t iters, void* ws, size_t ws_bytes, void* stream, double* ops_out) {
+  if (!ws || ws_bytes < XQ_WS_HEADER_BYTES || !aligned16(ws)) return XQ_ERR_WORKSPACE;
+  if (iters < 1 || iters > (1 << 22)) return XQ_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  if (xq_launch_i8_mma_rate(iters, (int32_t*)ws, sms, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  if (ops_out) *ops_out = (double)sms * iters * 4.0 * 2.0 * 128.0 * 256.0 * 32.0;
   return XQ_OK;
 }
 

@@ -81,3 +81,30 @@ cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, const int32_t* zp
                                             w->Kpp / XQ_K_GROUP, (__nv_bfloat16*)out, acc_opt);
   return cudaGetLastError();
 }
+
+// Which of the three product kernels xq_launch_gemm takes for M tokens against w (the same tests, nothing launched).
+extern "C" xq_status xq_gemm_kernel_info(int32_t M, const xq_weights* w, int32_t* kind, int32_t* tile_tokens, int32_t* tile_channels) {
+  if (!w || M < 1 || !kind || !tile_tokens || !tile_channels) return XQ_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return XQ_ERR_CUDA;
+  }
+  if (dev != w->device) return XQ_ERR_INVALID_ARG;
+  int mt = 0, cluster = 0;
+  if (M <= XQ_DECODE_MAX_M && xq_decode_shape(M, w, &mt, &cluster)) {
+    *kind = 0;
+    *tile_tokens = mt;
+    *tile_channels = 16;
+  } else if (xq_gemm_wants_a8(M, w)) {
+    const int c = xq_prefill_tile_choice(M, w, w->sms);
+    *kind = 1;
+    *tile_tokens = c == 0 ? 128 : 256;
+    *tile_channels = c == 2 ? 128 : 256;
+  } else {
+    *kind = 2;
+    *tile_tokens = 1;
+    *tile_channels = 1;
+  }
+  return XQ_OK;
+}

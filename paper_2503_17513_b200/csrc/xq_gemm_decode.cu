@@ -522,6 +522,14 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
 
 }  // namespace
 
+bool xq_decode_shape(int32_t M, const xq_weights* w, int* padded_tokens, int* cluster) {
+  const DecodePlan d = decode_plan(M, w);
+  if (d.stages < 16) return false;
+  *padded_tokens = 8 * d.nt;
+  *cluster = d.C;
+  return true;
+}
+
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
                                   void* out, int32_t* acc_opt, int32_t* status, cudaStream_t st) {
   const DecodePlan d = decode_plan(M, w);

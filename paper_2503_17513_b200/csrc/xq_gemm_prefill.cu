@@ -348,6 +348,57 @@ __global__ void expand_tokens_kernel(const uint4* __restrict__ Xq, long long pie
   }
 }
 
+// Issue-rate probe of the tensor core for this kernel's MMA (measurement only): every CTA holds one operand stage
+// of pseudo-random bytes in the layout the product kernel uses and one thread issues `iters` K blocks of four
+// 128 x 256 x 32 kind::i8 MMAs each, alternating between two accumulators; nothing is loaded or unpacked meanwhile.
+// Operations per CTA: iters * 4 * 2 * 128 * 256 * 32.
+__global__ void __launch_bounds__(128, 1) i8_mma_rate_kernel(int iters, int32_t* status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  unsigned char* base = smem_raw + (((raw + 1023u) & ~1023u) - raw);
+  __shared__ uint64_t done;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int failed;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  for (int i = tid; i < (kI8ABytes + 256 * 128) / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(base)[i] = (uint32_t)(i * 2654435761u + blockIdx.x * 40503u) & 0xF0F0F0F0u;
+  if (tid == 0) {
+    mbar_init(&done, 1);
+    failed = 0;
+    mbar_fence_init();
+  }
+  fence_proxy_async_smem();
+  if (warp == 0) {
+    tmem_alloc(&tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_slot;
+  if (warp == 0) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_s8(BMH, 256);
+      const uint32_t a_addr = smem_u32(base);
+      const uint64_t adesc = umma_desc_k128(a_addr), bdesc = umma_desc_k128(a_addr + kI8ABytes);
+      for (int it = 0; it < iters; ++it) {
+        const uint32_t d_tmem = tmem_base + (uint32_t)(it & 1) * 256u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) umma_i8_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (it >> 1 | k) != 0 ? 1u : 0u);
+      }
+      umma_commit(&done);
+    }
+    __syncwarp();
+    mbar_wait_bounded(&done, 0, &failed, status, (int)XQ_ERR_TIMEOUT);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -407,6 +458,21 @@ cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, ui
   return cudaLaunchKernelEx(&cfg, expand_tokens_kernel, (const uint4*)Xq, pieces, (uint4*)A8);
 }
 
+// Three tile shapes; a cost model picks one: waves of tiles over the multiprocessors times the cycles of a tile
+// (69 tensor-core cycles per 128 x 256 x 32 MMA; 128-token tiles expand every weight for half as many MMAs and run
+// at about 0.62 of that rate; an epilogue that is not hidden costs about 2000 cycles).
+// Returns 0 for 128 tokens x 256 channels, 1 for 256 x 256, 2 for 256 x 128.
+int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms) {
+  const int KB = w->Kpp / XQ_K_BLOCK, tm1 = (M + BMH - 1) / BMH, tm2 = (M + 2 * BMH - 1) / (2 * BMH);
+  auto waves = [&](int tiles) { return (double)((tiles + sms - 1) / sms); };
+  const double t_1x256 = waves(tm1 * ((w->N + 255) / 256)) * (KB * 276.0 / 0.62);
+  const double t_2x256 = waves(tm2 * ((w->N + 255) / 256)) * (KB * 552.0 + 2000.0);
+  const double t_2x128 = waves(tm2 * ((w->N + 127) / 128)) * (KB * 276.0 / 0.80);  // N = 128 MMAs re-read the tokens twice as often
+  if (t_2x128 <= t_2x256 && t_2x128 <= t_1x256) return 2;
+  if (t_2x256 <= t_1x256) return 1;
+  return 0;
+}
+
 cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
                                    void* out, int32_t* acc_opt, int32_t* status, int sms, cudaStream_t st) {
   EncodeTiledFn enc = encode_tiled_fn();
@@ -433,15 +499,17 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int
   p.KB = w->Kpp / XQ_K_BLOCK;
   p.tiles_n = 0;
   p.tiles_m = 0;
-  // Three tile shapes; a cost model picks one: waves of tiles over the multiprocessors times the cycles of a tile
-  // (69 tensor-core cycles per 128 x 256 x 32 MMA; 128-token tiles expand every weight for half as many MMAs and run
-  // at about 0.62 of that rate; an epilogue that is not hidden costs about 2000 cycles).
-  const int KB = p.KB, tm1 = (M + BMH - 1) / BMH, tm2 = (M + 2 * BMH - 1) / (2 * BMH);
-  auto waves = [&](int tiles) { return (double)((tiles + sms - 1) / sms); };
-  const double t_1x256 = waves(tm1 * ((w->N + 255) / 256)) * (KB * 276.0 / 0.62);
-  const double t_2x256 = waves(tm2 * ((w->N + 255) / 256)) * (KB * 552.0 + 2000.0);
-  const double t_2x128 = waves(tm2 * ((w->N + 127) / 128)) * (KB * 276.0 / 0.80);  // N = 128 MMAs re-read the tokens twice as often
-  if (t_2x128 <= t_2x256 && t_2x128 <= t_1x256) return launch_mh<2, 128>(mapA, p, sms, st);
-  if (t_2x256 <= t_1x256) return launch_mh<2, 256>(mapA, p, sms, st);
-  return launch_mh<1, 256>(mapA, p, sms, st);
+  switch (xq_prefill_tile_choice(M, w, sms)) {
+    case 2: return launch_mh<2, 128>(mapA, p, sms, st);
+    case 1: return launch_mh<2, 256>(mapA, p, sms, st);
+    default: return launch_mh<1, 256>(mapA, p, sms, st);
+  }
+}
+
+cudaError_t xq_launch_i8_mma_rate(int iters, int32_t* status, int sms, cudaStream_t st) {
+  const size_t smem = 1024 + kI8ABytes + 256 * 128;
+  cudaError_t e = cudaFuncSetAttribute(i8_mma_rate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  i8_mma_rate_kernel<<<sms, 128, smem, st>>>(iters, status);
+  return cudaGetLastError();
 }

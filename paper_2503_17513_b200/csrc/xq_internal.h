@@ -43,6 +43,17 @@ struct xq_weights {
   int sms;             // multiprocessors of that device
 };
 
+// True when `device` (the one a weights object lives on) is the current device: the kernels dereference the
+// object's pointers, so a call made with another device current is refused on the host.
+inline bool xq_on_device(int device) {
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return cur == device;
+}
+
 // Byte offset of the 32-bit word holding codes 8*kg .. 8*kg+7 of row n (k_groups = K'' / 32).
 __host__ __device__ inline size_t xq_weight_word_offset(int n, int kg, int k_groups) {
   const int blk = n >> 4, r = n & 15, grp = kg >> 2, word = kg & 3;
@@ -135,6 +146,10 @@ cudaError_t xq_launch_weight_sums(const uint8_t* blocks, int32_t Np, int32_t Kpp
 // zp (optional, here and below): per-token zero points; the epilogue then removes zp[m] * w_sum[n].
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
                                   void* out, int32_t* acc_opt, int32_t* status, cudaStream_t st);
+// True when M tokens against w run in the decode kernel; then also its padded token count and cluster size.
+bool xq_decode_shape(int32_t M, const xq_weights* w, int* padded_tokens, int* cluster);
+// Tile shape the tensor-core kernel picks: 0 = 128 tokens x 256 channels, 1 = 256 x 256, 2 = 256 x 128.
+int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms);
 // Tensor-core path: takes the tokens one code per byte (16 x code, even codes of every word first),
 // as written by the rotate kernels' optional output or by xq_launch_expand_tokens.
 bool xq_prefill_supported(int32_t M, const xq_weights* w);
@@ -145,6 +160,8 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int
 // kernel write the byte-per-code tokens).
 cudaError_t xq_launch_selftest_wait_timeout(int32_t* status, cudaStream_t st);
 bool xq_gemm_wants_a8(int32_t M, const xq_weights* w);
+// Tensor-core issue-rate probe: one CTA per multiprocessor, iters * 4 MMAs of 128 x 256 x 32 (kind::i8) each.
+cudaError_t xq_launch_i8_mma_rate(int iters, int32_t* status, int sms, cudaStream_t st);
 // a8_ready: the a8 region of the workspace already holds the byte-per-code tokens.
 cudaError_t xq_launch_gemm(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w, void* out,
                            int32_t* acc_opt, void* ws, const xq_ws_layout& L, bool a8_ready, cudaStream_t st);

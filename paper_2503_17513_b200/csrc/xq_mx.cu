@@ -904,7 +904,7 @@ xq_status xq_mx_weights_import(const uint8_t* codes_packed, const uint8_t* scale
 }
 
 xq_status xq_mx_weights_export(const xq_mx_weights* w, uint8_t* codes, uint8_t* scales) {
-  if (!w || !codes || !scales) return XQ_ERR_INVALID_ARG;
+  if (!w || !codes || !scales || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   DevBuf dC, dS;
   const size_t nc = (size_t)w->N * w->Kp, ns = (size_t)w->N * (w->Kp / 32);
   if (dC.alloc(nc) != cudaSuccess || dS.alloc(ns) != cudaSuccess) {
@@ -958,7 +958,7 @@ xq_status xq_mx_gemm(const uint8_t* codes, const uint8_t* scales, int32_t M, con
                      void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!codes || !scales || !out || !aligned16(codes) || !aligned16(out)) return XQ_ERR_INVALID_ARG;
+  if (!codes || !scales || !out || !aligned16(codes) || !aligned16(out) || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   const MxWs L = mx_ws(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
   uint8_t* base = (uint8_t*)ws;
@@ -978,7 +978,7 @@ xq_status xq_mx_gemm(const uint8_t* codes, const uint8_t* scales, int32_t M, con
 xq_status xq_mx_gemm_staged(int32_t M, const xq_mx_weights* w, void* out, void* ws, size_t ws_bytes, void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!out || !aligned16(out)) return XQ_ERR_INVALID_ARG;
+  if (!out || !aligned16(out) || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   const MxWs L = mx_ws(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
   uint8_t* base = (uint8_t*)ws;
@@ -995,7 +995,7 @@ xq_status xq_mx_rotate_quant_staged(const void* X, int32_t M, int64_t ldx, const
                                     void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!X) return XQ_ERR_INVALID_ARG;
+  if (!X || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   if (ldx < w->K || (ldx % 8) != 0 || !aligned16(X)) return XQ_ERR_INVALID_ARG;
   const MxWs L = mx_ws(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
@@ -1036,7 +1036,7 @@ xq_status xq_mx_expanded_linear_host(const void* X_host, int32_t M, const xq_mx_
                                      void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!X_host || !out_host || w->K % 8 != 0) return XQ_ERR_INVALID_ARG;
+  if (!X_host || !out_host || w->K % 8 != 0 || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   const MxWs L = mx_ws(M, w);
   if (!ws || !aligned16(ws) || ws_bytes < L.total) return XQ_ERR_WORKSPACE;
   uint8_t* base = (uint8_t*)ws;

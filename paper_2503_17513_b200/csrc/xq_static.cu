@@ -46,7 +46,7 @@ extern "C" xq_status xq_expanded_linear_static(const void* X, int32_t M, int64_t
                                                void* stream) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
-  if (!X || !out) return XQ_ERR_INVALID_ARG;
+  if (!X || !out || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   if (ldx < w->K || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u))
     return XQ_ERR_INVALID_ARG;
   // [status header | packed codes M x K'/2 | scales M | byte-per-code tokens M x K' when M > 32]

@@ -42,7 +42,7 @@ EXPORTS = [
     "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
     "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
     "xq_mx_expanded_linear_host", "xq_mx_gemm_staged", "xq_mx_rotate_quant_staged",
-    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads",
+    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads", "xq_gemm_kernel_info", "xq_selftest_i8_mma_rate",
 ]
 
 
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.xq_poll_status.argtypes = [vp, vp]
         L.xq_expanded_linear_static.argtypes = [vp, i32, i64, vp, vp, vp]
         L.xq_selftest_wait_timeout.argtypes = [vp, sz, vp]
+        L.xq_selftest_i8_mma_rate.argtypes = [i32, vp, sz, vp, ctypes.POINTER(ctypes.c_double)]
+        L.xq_gemm_kernel_info.argtypes = [i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
         for name in EXPORTS:
             if name not in ("xq_status_string", "xq_weights_free", "xq_workspace_bytes", "xq_weights_heads", "xq_mx_weights_free",
                             "xq_mx_workspace_bytes", "xq_mx_weights_heads"):
@@ -288,6 +290,21 @@ def xq_expanded_linear_static(X, w: Weights, out, M=None, ldx=None, stream=None)
 def xq_selftest_wait_timeout(ws, stream=None) -> None:
     """Enqueue the self-test kernel whose bounded wait runs out after about a second."""
     _check(lib().xq_selftest_wait_timeout(_dp(ws), ws.numel() * ws.element_size(), _stream(stream)), "xq_selftest_wait_timeout")
+
+
+def xq_gemm_kernel_info(M: int, w: Weights):
+    """(kind, tile_tokens, tile_channels) of the product kernel that M tokens against w run in."""
+    kind, tt, tc = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _check(lib().xq_gemm_kernel_info(M, w.handle, ctypes.byref(kind), ctypes.byref(tt), ctypes.byref(tc)), "xq_gemm_kernel_info")
+    return kind.value, tt.value, tc.value
+
+
+def xq_selftest_i8_mma_rate(iters: int, ws, stream=None) -> float:
+    """Enqueue the tensor-core issue-rate probe; returns the integer operations the launch performs."""
+    ops = ctypes.c_double()
+    _check(lib().xq_selftest_i8_mma_rate(iters, _dp(ws), ws.numel() * ws.element_size(), _stream(stream), ctypes.byref(ops)),
+           "xq_selftest_i8_mma_rate")
+    return ops.value
 
 
 def xq_poll_status(ws, stream=None) -> int:

@@ -313,3 +313,15 @@ def test_full_size_sampled_rows(xq, oracle, tag, M, N, K, Kp, heavy, nsample):
     diff = codes.astype(np.int32) - qw.astype(np.int32)
     assert np.abs(diff).max() <= 1 and np.count_nonzero(diff) / diff.size <= CODE_MISMATCH_FRAC
     assert np.allclose(s_back, s_w, rtol=2e-6)
+    # The product alone at full size, with no rounding-tie allowance in the way: the codes and scales that the GPU
+    # itself made for these rows (the same rotate kernel the layer call ran) and the weights it prepared go through
+    # the oracle's integer product and one-rounding epilogue; every output of the layer is within one bf16 ulp.
+    Xq_g = torch.empty((M, Kp // 2), dtype=torch.uint8, device="cuda")
+    sx_g = torch.empty((M,), dtype=torch.float32, device="cuda")
+    xq.xq_rotate_quant(dev(x), w.plan, Xq_g, sx_g)
+    ridx = torch.from_numpy(rows).cuda()
+    qx_g = oracle.unpack_int4(Xq_g[ridx].cpu().numpy())
+    want_g = synth.bf16_bits_to_f32(oracle.epilogue(oracle.gemm_i64(qx_g, codes), sx_g[ridx].cpu().numpy(), s_back)).astype(np.float64)
+    got64 = got.astype(np.float64)
+    assert np.all(np.abs(got64 - want_g) <= np.abs(want_g) * 2.0**-7 + 1e-30), tag
+    assert np.mean(got64 == want_g) > 0.99

@@ -1,0 +1,159 @@
+"""Bit-exact accumulators on every tile shape of the tcgen05 INT4 product kernel, each case naming the
+shape it ran on (asked from the library with xq_gemm_kernel_info, nothing is assumed).
+
+The quantized product Q(XR) Q(W~) of the paper's Sec. 3 is an integer sum, so given identical codes
+the int32 accumulators must equal the oracle's int64 sums exactly, whatever tile shape, tile count
+per CTA, K length or tail the launch has.  Cases here reach the three shapes the kernel can pick
+(128 tokens x 256 channels, 256 x 256, 256 x 128) at the layer sizes the benchmark times, and the
+extreme codes (-8 against -8 and against 7) at the longest K' of the paper's Table 1, where the
+16 x 16 factor carried by the nibble expansion makes the partial sums largest.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2503_17513_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TILE_KERNEL = 1
+
+
+@pytest.fixture(scope="module")
+def xq():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2503_17513_b200 import xq as binding
+
+    binding.lib()
+    return binding
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda()
+    return torch.from_numpy(a).cuda()
+
+
+def host_u16(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().view(torch.int16).numpy().view(np.uint16)
+
+
+def sample_rows(M, count, seed=13):
+    rows = np.sort(np.random.default_rng(seed).choice(M, size=min(count, M), replace=False))
+    rows[-1] = M - 1  # the last row of the last tile is always among them
+    return rows
+
+
+# (M, N, K, Kp, tile the library must report, token rows compared: None = all)
+TILE_CASES = [
+    (384, 9728, 250, 256, (128, 256), None),
+    (2048, 8192, 2048, 2176, (256, 256), None),       # gate / up of the 1B prefill workload
+    (512, 14336, 4096, 4352, (256, 256), None),       # gate / up of the 8B workload, all channels
+    (2048, 2048, 8192, 8704, (256, 128), None),       # down of the 1B prefill workload
+    (4096, 14336, 4096, 4352, (256, 256), 64),        # the 8B prefill launches as the benchmark times them
+    (4096, 4096, 14336, 15360, (256, 256), 64),
+    (8192, 4096, 4096, 4096, (256, 128), 64),         # the expansion sweep at its two ends
+    (8192, 4096, 4096, 5120, (256, 256), 64),
+]
+IDS = [f"M{c[0]}-N{c[1]}-Kp{c[3]}-{c[4][0]}x{c[4][1]}" for c in TILE_CASES]
+
+
+@pytest.mark.parametrize("M,N,K,Kp,tile,nrows", TILE_CASES, ids=IDS)
+def test_tile_shape_accumulators_bit_exact(xq, oracle, M, N, K, Kp, tile, nrows):
+    qx = synth.int4_codes(M, Kp, seed=21, tag=f"tx{M}")
+    qw = synth.int4_codes(N, Kp, seed=21, tag=f"tw{N}")
+    s_x = synth.scales(M, seed=21, tag="x")
+    s_w = synth.scales(N, seed=21, tag="w")
+    w = xq.xq_weights_import(qw, s_w, K)
+    assert xq.xq_gemm_kernel_info(M, w) == (TILE_KERNEL, *tile)
+    ws = xq.new_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    xq.xq_w4a4_gemm(dev(oracle.pack_int4(qx)), dev(s_x), M, w, out, ws, acc=acc)
+    assert xq.xq_poll_status(ws) == xq.OK
+    rows = np.arange(M) if nrows is None else sample_rows(M, nrows)
+    ridx = torch.from_numpy(rows).cuda()
+    acc_ref = oracle.gemm_i64(qx[rows], qw)
+    assert np.array_equal(acc[ridx].cpu().numpy().astype(np.int64), acc_ref)
+    want = synth.bf16_bits_to_f32(oracle.epilogue(acc_ref, s_x[rows], s_w)).astype(np.float64)
+    got = synth.bf16_bits_to_f32(host_u16(out[ridx])).astype(np.float64)
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0**-7 + 1e-30)  # one bf16 ulp
+    assert np.mean(got == want) > 0.99
+
+
+ASYM_TILE_CASES = [
+    (384, 9728, 250, 256, (128, 256), None),
+    (2048, 8192, 2048, 2176, (256, 256), 256),
+    (2048, 2048, 8192, 8704, (256, 128), 256),
+    (4096, 4096, 14336, 15360, (256, 256), 64),
+]
+
+
+@pytest.mark.parametrize("M,N,K,Kp,tile,nrows", ASYM_TILE_CASES, ids=[f"M{c[0]}-N{c[1]}-Kp{c[3]}-{c[4][0]}x{c[4][1]}" for c in ASYM_TILE_CASES])
+def test_tile_shape_zero_point_epilogue_bit_exact(xq, oracle, M, N, K, Kp, tile, nrows):
+    """The zero-point term of asymmetric tokens (Sec. 4), sum (u - z) qw, on the same tile shapes."""
+    ux = (synth.int4_codes(M, Kp, seed=22, tag=f"ux{M}").astype(np.int16) + 8).astype(np.uint8)
+    z = (synth.int4_codes(M, 1, seed=22, tag=f"z{M}").astype(np.int32) + 8)[:, 0].copy()
+    qw = synth.int4_codes(N, Kp, seed=22, tag=f"w{N}")
+    s_x = synth.scales(M, seed=22, tag="x")
+    s_w = synth.scales(N, seed=22, tag="w")
+    w = xq.xq_weights_import(qw, s_w, K)
+    assert xq.xq_gemm_kernel_info(M, w) == (TILE_KERNEL, *tile)
+    ws = xq.new_workspace(M, w)
+    Xq = dev(oracle.pack_int4((ux.astype(np.int16) - 8).astype(np.int8)))
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    xq.xq_w4a4_gemm_asym(Xq, dev(s_x), dev((z - 8).astype(np.int32)), M, w, out, ws, acc=acc)
+    assert xq.xq_poll_status(ws) == xq.OK
+    rows = np.arange(M) if nrows is None else sample_rows(M, nrows)
+    ridx = torch.from_numpy(rows).cuda()
+    acc_u = oracle.gemm_u_i64(ux[rows], qw)
+    acc_ref = acc_u - z[rows, None].astype(np.int64) * qw.astype(np.int64).sum(axis=1)[None, :]
+    assert np.array_equal(acc[ridx].cpu().numpy().astype(np.int64), acc_ref)
+    want = synth.bf16_bits_to_f32(oracle.epilogue_asym(acc_u, s_x[rows], z[rows], s_w, qw)).astype(np.float64)
+    got = synth.bf16_bits_to_f32(host_u16(out[ridx])).astype(np.float64)
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0**-7 + 1e-30)
+
+
+# (M, N, K, Kp, tile): the largest partial sums the kernel can meet -- every product is (-8)(-8) = 64 or (-8)(7) = -56,
+# times 256 inside the tensor core, over the two longest K' of Table 1.
+EXTREME_CASES = [
+    (64, 256, 14336, 18432, (256, 128)),
+    (200, 256, 14336, 22016, (256, 128)),
+    (1024, 9472, 14336, 18432, (256, 256)),
+    (1024, 9472, 14336, 22016, (256, 256)),
+    (384, 9728, 14336, 22016, (128, 256)),
+]
+
+
+@pytest.mark.parametrize("M,N,K,Kp,tile", EXTREME_CASES, ids=[f"M{c[0]}-N{c[1]}-Kp{c[3]}-{c[4][0]}x{c[4][1]}" for c in EXTREME_CASES])
+def test_tile_shape_extreme_codes_closed_form(xq, oracle, M, N, K, Kp, tile):
+    qx = np.full((M, Kp), -8, dtype=np.int8)
+    qw = np.full((N, Kp), -8, dtype=np.int8)
+    qw[1::3] = 7
+    w = xq.xq_weights_import(qw, np.ones(N, np.float32), K)
+    assert xq.xq_gemm_kernel_info(M, w) == (TILE_KERNEL, *tile)
+    ws = xq.new_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    xq.xq_w4a4_gemm(dev(oracle.pack_int4(qx)), torch.ones(M, device="cuda"), M, w, out, ws, acc=acc)
+    assert xq.xq_poll_status(ws) == xq.OK
+    want = np.full(N, 64 * Kp, dtype=np.int64)
+    want[1::3] = -56 * Kp
+    a = acc.cpu().numpy().astype(np.int64)
+    assert np.array_equal(a, np.broadcast_to(want, (M, N)))
+    # the outputs: bf16 of the closed form (scales are one)
+    got = synth.bf16_bits_to_f32(host_u16(out)).astype(np.float64)
+    ref = synth.bf16_bits_to_f32(oracle.epilogue(np.broadcast_to(want, (M, N)).copy(), np.ones(M, np.float32), np.ones(N, np.float32)))
+    assert np.array_equal(got, ref.astype(np.float64))
+
+
+def test_i8_mma_rate_probe_runs_and_reports_its_operations(xq):
+    """The tensor-core issue-rate probe (the measured INT8 ceiling of the benchmark) completes, leaves the status
+    word clean and counts 2 x 128 x 256 x 32 operations per instruction, four instructions per iteration and SM."""
+    w = xq.xq_weights_import(synth.int4_codes(32, 64), synth.scales(32), 64)
+    ws = xq.new_workspace(4, w)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    ops = xq.xq_selftest_i8_mma_rate(50, ws)
+    assert xq.xq_poll_status(ws) == xq.OK
+    assert ops == sms * 50 * 4 * 2 * 128 * 256 * 32

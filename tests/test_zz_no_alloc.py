@@ -32,16 +32,18 @@ def _f32(t):
     return synth.bf16_bits_to_f32(t.cpu().numpy().view(np.uint16)).astype(np.float64)
 
 
-def test_static_scratch_matches_workspace_path_twice_in_a_row():
+def test_static_scratch_matches_workspace_path_twice_in_a_row(oracle):
     assert torch.cuda.is_available(), "GPU tests need a CUDA device"
     from paper_2503_17513_b200 import xq
 
     xq.lib()
     K, Kp, N = 2048, 2176, 512
-    w = xq.xq_prepare_weights(synth.weights(N, K, seed=5, tag="na"), Kp)
+    wb = synth.weights(N, K, seed=5, tag="na")
+    w = xq.xq_prepare_weights(wb, Kp)
     # a decode-sized call, then a larger one that takes the tensor-core path, then the first again
     for M, tag in [(16, "a"), (160, "b"), (16, "c")]:
-        X = _dev(synth.activations(M, K, seed=5, tag=tag, heavy_tail=(M > 32)))
+        x_bits = synth.activations(M, K, seed=5, tag=tag, heavy_tail=(M > 32))
+        X = _dev(x_bits)
         want = torch.empty((M, N), dtype=torch.int16, device="cuda")
         ws = xq.new_workspace(M, w)
         xq.xq_expanded_linear(X, w, want, ws)
@@ -52,6 +54,17 @@ def test_static_scratch_matches_workspace_path_twice_in_a_row():
         a, b = _f32(got), _f32(want)
         assert np.linalg.norm(a - b) <= E2E_REL_L2 * np.linalg.norm(b)
         assert torch.equal(got, want), "same kernels, same inputs: the outputs are the same bits"
+        # and directly against the CPU oracle, within the end-to-end bound of the other tests
+        ref_bits, _ = oracle.expanded_linear(oracle.plan(K, Kp), x_bits, wb)
+        ref = synth.bf16_bits_to_f32(ref_bits).astype(np.float64)
+        assert np.linalg.norm(a - ref) <= E2E_REL_L2 * np.linalg.norm(ref)
+        # a warm call takes no device memory: the free amount is the same before and after a second call
+        free_before, _ = torch.cuda.mem_get_info()
+        xq.xq_expanded_linear_static(X, w, got)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
+        assert torch.equal(got, want)
 
 
 def test_static_scratch_refuses_what_does_not_fit():
