@@ -233,6 +233,13 @@ xq_status xq_mx_expanded_linear_host(const void* X_bf16_host, int32_t M, const x
 xq_status xq_expanded_linear_host(const void* X_bf16_host, int32_t M, const xq_weights* w,
                                   void* out_bf16_host, void* ws_dev, size_t ws_bytes, void* stream);
 
+/* xq_expanded_linear_host without the final synchronization: the two copies and the layer are only
+ * enqueued on `stream` (pinned host memory; with pageable memory the runtime makes the copies
+ * synchronous).  X_host must stay untouched and out_host is valid only after the caller has
+ * synchronized the stream; several layers may be enqueued back to back and awaited once. */
+xq_status xq_expanded_linear_host_enqueue(const void* X_bf16_host, int32_t M, const xq_weights* w,
+                                          void* out_bf16_host, void* ws_dev, size_t ws_bytes, void* stream);
+
 /* The whole layer for callers that cannot allocate device memory.  (No counterpart in the paper:
  * this is a deployment variant of xq_expanded_linear, same arithmetic, same kernels.)
  *

@@ -485,7 +485,7 @@ xq_status xq_expanded_linear_asym(const void* X, int32_t M, int64_t ldx, const x
 namespace {
 
 xq_status linear_host_impl(const void* X_host, int32_t M, const xq_weights* w, bool asym, void* out_host, void* ws,
-                           size_t ws_bytes, void* stream) {
+                           size_t ws_bytes, void* stream, bool sync = true) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X_host || !out_host || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
@@ -504,7 +504,7 @@ xq_status linear_host_impl(const void* X_host, int32_t M, const xq_weights* w, b
   xq_status s = linear_impl(base + L.xstage, M, ldx, w, asym, base + L.ostage, ws, ws_bytes, stream);
   if (s != XQ_OK) return s;
   e = cudaMemcpyAsync(out_host, base + L.ostage, (size_t)M * w->N * 2, cudaMemcpyDeviceToHost, st);
-  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess && sync) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return XQ_ERR_CUDA;
@@ -524,6 +524,11 @@ xq_status xq_expanded_linear_host(const void* X_host, int32_t M, const xq_weight
 xq_status xq_expanded_linear_host_asym(const void* X_host, int32_t M, const xq_weights* w, void* out_host, void* ws,
                                        size_t ws_bytes, void* stream) {
   return linear_host_impl(X_host, M, w, true, out_host, ws, ws_bytes, stream);
+}
+
+xq_status xq_expanded_linear_host_enqueue(const void* X_host, int32_t M, const xq_weights* w, void* out_host, void* ws,
+                                          size_t ws_bytes, void* stream) {
+  return linear_host_impl(X_host, M, w, false, out_host, ws, ws_bytes, stream, false);
 }
 
 xq_status xq_selftest_wait_timeout(void* ws, size_t ws_bytes, void* stream) {

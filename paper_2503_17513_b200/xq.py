@@ -42,7 +42,7 @@ EXPORTS = [
     "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
     "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
     "xq_mx_expanded_linear_host", "xq_mx_gemm_staged", "xq_mx_rotate_quant_staged",
-    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads", "xq_gemm_kernel_info", "xq_selftest_i8_mma_rate",
+    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads", "xq_gemm_kernel_info", "xq_selftest_i8_mma_rate", "xq_expanded_linear_host_enqueue",
 ]
 
 
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
         L.xq_expanded_linear_asym.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host_asym.argtypes = [vp, i32, vp, vp, vp, sz, vp]
+        L.xq_expanded_linear_host_enqueue.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_rotate_quant_heads.argtypes = [vp, i32, i64, i32, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp, vp]
         L.xq_prepare_weights_heads.argtypes = [vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
         L.xq_weights_heads.argtypes = [vp]
@@ -269,6 +270,14 @@ def xq_expanded_linear_host(X_host, w: Weights, out_host, ws, M=None, stream=Non
     _check(lib().xq_expanded_linear_host(ctypes.c_void_p(X_host.data_ptr()), M, w.handle,
                                          ctypes.c_void_p(out_host.data_ptr()), _dp(ws), ws.numel() * ws.element_size(),
                                          _stream(stream)), "xq_expanded_linear_host")
+
+
+def xq_expanded_linear_host_enqueue(X_host, w: Weights, out_host, ws, M=None, stream=None) -> None:
+    """As xq_expanded_linear_host, but only enqueued: synchronize the stream before reading out_host."""
+    M = X_host.shape[0] if M is None else M
+    _check(lib().xq_expanded_linear_host_enqueue(ctypes.c_void_p(X_host.data_ptr()), M, w.handle,
+                                                 ctypes.c_void_p(out_host.data_ptr()), _dp(ws), ws.numel() * ws.element_size(),
+                                                 _stream(stream)), "xq_expanded_linear_host_enqueue")
 
 
 def xq_expanded_linear_host_asym(X_host, w: Weights, out_host, ws, M=None, stream=None) -> None:
