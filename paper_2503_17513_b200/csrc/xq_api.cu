@@ -431,6 +431,14 @@ xq_status linear_impl(const void* X, int32_t M, int64_t ldx, const xq_weights* w
   float* sx = (float*)(base + L.sx);
   int32_t* zp = asym ? (int32_t*)(base + L.zp) : nullptr;
   cudaStream_t st = (cudaStream_t)stream;
+  if (M <= XQ_DECODE_MAX_M) {  // one launch: the online step inside the product kernel
+    const cudaError_t e = xq_launch_linear_decode(X, ldx, Xq, sx, zp, M, w, out, (int32_t*)ws, st);
+    if (e == cudaSuccess) return XQ_OK;
+    if (e != cudaErrorNotSupported) {
+      cudaGetLastError();
+      return XQ_ERR_CUDA;
+    }
+  }
   uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + L.a8 : nullptr;
   if (xq_launch_rotate_for(w, X, M, ldx, Xq, sx, A8, zp, st) != cudaSuccess ||
       xq_launch_gemm(Xq, sx, zp, M, w, out, nullptr, ws, L, A8 != nullptr, st) != cudaSuccess) {

@@ -22,12 +22,24 @@
 // memory), and after one cluster barrier the owner sums the C * S tiles and applies the epilogue
 // (exact >> 8, scales, bf16, 16-byte stores).  No global scratch, no atomics, and no CTA waits on
 // another outside the cluster barrier.
+//
+// Fused form (the whole layer in one launch, paper Sec. 3 "online": X_hat = X H_hat computed at inference, then
+// the product).  The weights do not depend on the tokens, so every CTA requests its first ring-full before
+// anything else; meanwhile CTA r (r < M) pads, rotates and quantizes token row r with the routine of
+// xq_rotate_row.cuh (its scratch lies where the token slice and the partial tiles go later), writes the packed
+// codes and the scale to the workspace and publishes a per-row flag (release); every CTA then waits, time-bounded,
+// for the M flags (acquire) and reads its K slice of the codes from L2.  Rotating CTAs never wait before they
+// publish, so the launch makes progress whenever its first M CTAs run; a wait that runs out records
+// XQ_ERR_TIMEOUT and the CTA leaves through the normal exits.  Flags carry the launch's generation number, kept
+// in the workspace header and advanced by the last CTA to leave, so that replays of a captured launch need no
+// host-side reset.
 #include <cuda_bf16.h>
 
 #include <mutex>
 
 #include "xq_internal.h"
 #include "xq_ptx.cuh"
+#include "xq_rotate_row.cuh"
 
 using namespace xqptx;
 
@@ -59,7 +71,97 @@ struct DecodeParams {
   int max_blocks;   // blocks in the longest cluster range
   int log2S;        // sub-slices per block and CTA: S = 1 << log2S
   int P;            // ring pieces per work item
+  int region_bytes; // token slice + partial tiles (fused form: or the rotation scratch, whichever is larger)
+  // fused online step: the first M CTAs rotate and quantize the token rows into Xq / sx / zp (workspace)
+  const __nv_bfloat16* X;
+  long long ldx;
+  xq_hadamard_plan_t plan;
+  float gamma;
+  const __nv_bfloat16* Hsigns;  // bf16 image of H_p^T
+  uint8_t* Xq_w;
+  float* sx_w;
+  int32_t* zp_w;                // null: symmetric codes
+  uint32_t* sync_words;         // workspace header words: [1] generation, [2] CTAs that have left, [32 + r] flag of row r
+  int rot_threads;              // threads of a row group: 32 x tiles of 16 output rows x column chunks
 };
+
+// Workspace header words of the fused form.
+constexpr int kGenWord = 1, kExitWord = 2, kFlagWord0 = 32;
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Rows blockIdx.x, blockIdx.x + gridDim.x, ... < M through pad + rotate + quantize by the first rot_threads threads
+// of the CTA; each finished row is published with its flag.  `region` is this CTA's scratch.
+template <int LOG2NB, int KS>
+__device__ __noinline__ void fused_rotate_rows(const DecodeParams& p, unsigned char* region, int tid) {
+  const xq_hadamard_plan_t& pl = p.plan;
+  const int n = 1 << pl.log2n, pitch = n + 8, NB = 1 << LOG2NB, NC = n / NB;
+  const int P16 = (pl.p + 15) / 16 * 16, hpitch = P16 + 8;
+  const int nthreads = p.rot_threads, warp = tid >> 5, lane = tid & 31, mt = warp / NC;
+  const xqrot::RowLayout L = xqrot::row_layout(pl);
+  __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(region + L.xs);
+  __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(region + L.hs);
+  const xqrot::RowSmem sm = {Xs, reinterpret_cast<uint32_t*>(region + L.outp), nullptr, reinterpret_cast<float*>(region + L.red),
+                             reinterpret_cast<float*>(region + L.exch)};
+  const xqrot::NamedSync sync = {2, nthreads};
+  // constants of the plan first: nothing here depends on the preceding kernel
+  for (int i = tid; i < P16 * hpitch / 8; i += nthreads) cp_async16(Hs + 8 * i, p.Hsigns + 8 * i);
+  for (int i = tid; i < KS * 16 * pitch / 8; i += nthreads) reinterpret_cast<uint4*>(Xs)[i] = make_uint4(0, 0, 0, 0);
+  cp_async_wait_all();
+  sync();
+  uint32_t afrag[KS][4];
+  xqrot::load_afrag<KS>(afrag, Hs, P16, hpitch, mt, lane);
+  pdl_wait();
+  const uint32_t want = ld_acquire_u32(p.sync_words + kGenWord) + 1u;
+  const xqrot::RowOut out = {p.Xq_w, p.sx_w, nullptr, nullptr, p.zp_w, nullptr, 0};
+  const int chunks = pl.K / 8;
+  for (int row = blockIdx.x; row < p.M; row += gridDim.x) {
+    const __nv_bfloat16* x = p.X + (long long)row * p.ldx;
+    for (int i = tid; i < chunks; i += nthreads) {
+      const int c = 8 * i, a = c >> pl.log2n, b = c & (n - 1);
+      cp_async16(Xs + a * pitch + b, x + c);
+    }
+    cp_async_wait_all();
+    sync();
+    xqrot::rotate_row<LOG2NB, KS>(pl, p.gamma, afrag, sm, out, row, tid, nthreads, sync);
+    // rotate_row ends with the group's barrier: every thread's stores of the row precede it
+    if (tid == 0) {
+      __threadfence();
+      st_release_u32(p.sync_words + kFlagWord0 + row, want);
+    }
+  }
+}
+
+__device__ __forceinline__ void fused_rotate_dispatch(const DecodeParams& p, unsigned char* region, int tid) {
+  const int n = 1 << p.plan.log2n, ks = ((p.plan.K + n - 1) / n + 15) / 16;
+  switch (p.plan.log2n) {
+    case 5:
+      if (ks == 1) fused_rotate_rows<5, 1>(p, region, tid);
+      else if (ks == 2) fused_rotate_rows<5, 2>(p, region, tid);
+      else if (ks == 3) fused_rotate_rows<5, 3>(p, region, tid);
+      else fused_rotate_rows<5, 4>(p, region, tid);
+      break;
+    case 6:
+      if (ks == 1) fused_rotate_rows<6, 1>(p, region, tid);
+      else if (ks == 2) fused_rotate_rows<6, 2>(p, region, tid);
+      else if (ks == 3) fused_rotate_rows<6, 3>(p, region, tid);
+      else fused_rotate_rows<6, 4>(p, region, tid);
+      break;
+    default:
+      if (ks == 1) fused_rotate_rows<7, 1>(p, region, tid);
+      else if (ks == 2) fused_rotate_rows<7, 2>(p, region, tid);
+      else if (ks == 3) fused_rotate_rows<7, 3>(p, region, tid);
+      else fused_rotate_rows<7, 4>(p, region, tid);
+      break;
+  }
+}
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -77,7 +179,7 @@ __device__ __forceinline__ void st_cluster_v2(void* local_ptr, uint32_t rank, in
   asm volatile("st.shared::cluster.v2.s32 [%0], {%1, %2};" ::"r"(remote), "r"(v.x), "r"(v.y) : "memory");
 }
 
-template <int NT, int C>  // NT token tiles of 8 (M <= 8 NT), clusters of C CTAs
+template <int NT, int C, bool FUSED>  // NT token tiles of 8 (M <= 8 NT), clusters of C CTAs; FUSED: rotate + quantize inside
 __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -90,7 +192,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   // partial tiles of the blocks this CTA finishes: [owned block][source CTA, sub-slice][16 channels][MT tokens]
   const int S = 1 << p.log2S, srcs = C * S;
   int* tiles = reinterpret_cast<int*>(act + (size_t)MT * p.act_pitch);
-  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + (size_t)((p.max_blocks + C - 1) / C) * srcs * 16 * MT);
+  uint64_t* full = reinterpret_cast<uint64_t*>(act + p.region_bytes);
   uint64_t* empty = full + p.stages;
   volatile int* failed = reinterpret_cast<volatile int*>(empty + p.stages);
 
@@ -201,14 +303,48 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
     // the epilogue's channel scales: bring them into L2 now, they are constants
     for (int i = tid * 32; i < n_blk * 16; i += kConsumerThreads * 32)
       if (b0 * 16 + i < p.N) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.sw + b0 * 16 + i));
+    bool ok = true;
+    if (FUSED) {
+      // the online step of the layer, inside this launch: this CTA's token rows (if it has any), then the flags of all
+      if (blockIdx.x < p.M && tid < p.rot_threads) fused_rotate_dispatch(p, act, tid);
+      else pdl_wait();
+      bar_sync(1, kConsumerThreads);  // the scratch of the rotation is free: the token slice goes there
+      if (warp == 0) {
+        const uint32_t want = ld_acquire_u32(p.sync_words + kGenWord) + 1u;
+        bool seen = true;
+        if (lane < p.M) {
+          const uint32_t* flag = p.sync_words + kFlagWord0 + lane;
+          uint64_t t0 = 0;
+          for (uint32_t i = 1; ld_acquire_u32(flag) != want; ++i) {
+            if ((i & 31u) == 0u) {
+              const uint64_t now = globaltimer_ns();
+              if (t0 == 0) t0 = now;
+              if (*failed || now - t0 > 1000000000ull) {
+                seen = false;
+                break;
+              }
+            }
+          }
+        }
+        if (!__all_sync(0xffffffffu, seen) && lane == 0) {
+          *failed = 1;
+          atomicExch(p.status, (int)XQ_ERR_TIMEOUT);
+        }
+      }
+    }
     // token rows beyond M are zero
     for (int i = tid; i < (MT - p.M) * (p.act_pitch / 16); i += kConsumerThreads)
       reinterpret_cast<uint4*>(act + (size_t)p.M * p.act_pitch)[i] = make_uint4(0, 0, 0, 0);
-    pdl_wait();
+    if (FUSED) {
+      bar_sync(1, kConsumerThreads);
+      ok = !*failed;
+    } else {
+      pdl_wait();
+    }
     // Expand this CTA's K slice of the packed tokens once, in fragment order: chunk c of four
     // groups takes 128 bytes per token, word t of group i (even codes, odd codes) at
     // c * 128 + t * 32 + i * 8.
-    {
+    if (ok) {
       const int total = p.M * L;
       constexpr int kBatch = 6;
       for (int base = tid; base < total; base += kBatch * kConsumerThreads) {
@@ -218,7 +354,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
           const int i = base + u * kConsumerThreads;
           if (i < total) {
             const int m = i / L, l = i - m * L;
-            v[u] = __ldg(reinterpret_cast<const uint4*>(p.Xq + (size_t)m * (p.Kp / 2)) + g0 + l);
+            const uint4* src = reinterpret_cast<const uint4*>(p.Xq + (size_t)m * (p.Kp / 2)) + g0 + l;
+            v[u] = FUSED ? __ldcg(src) : __ldg(src);  // fused: written by other CTAs of this launch, read from L2
           }
         }
 #pragma unroll
@@ -244,7 +381,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
     if (C > 1) cluster_wait_acquire();  // every CTA of the cluster has started: remote stores are legal
 
     const int ag = lane >> 2, at = lane & 3;  // MMA fragment coordinates: channel row / token column, word
-    bool ok = true;
     for (int r = 0; r < rounds && ok; ++r) {
       const int t = r * kConsumerWarps + warp;
       if (t >= n_items) break;
@@ -324,8 +460,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
   if (warp < kConsumerWarps && tid < mine * p.M * 2) {
     const int h = tid & 1, bm = tid >> 1, jj = bm / p.M, m = bm - jj * p.M;
     const int n0 = (b0 + rank + jj * C) * 16 + 8 * h;
-    e_sx = p.sx[m];
-    if (p.zp) e_z = p.zp[m];
+    e_sx = FUSED ? __ldcg(p.sx + m) : p.sx[m];
+    if (p.zp) e_z = FUSED ? __ldcg(p.zp + m) : p.zp[m];
     if (n0 + 8 <= p.N && (p.N & 7) == 0) {
       e_s0 = *reinterpret_cast<const float4*>(p.sw + n0);
       e_s1 = *reinterpret_cast<const float4*>(p.sw + n0 + 4);
@@ -343,7 +479,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       int z = 0;
       int4 w0 = make_int4(0, 0, 0, 0), w1 = w0;
       if (p.zp) {  // issued ahead of the tile reads (w_sum covers the padded rows)
-        z = pre ? e_z : p.zp[m];
+        z = pre ? e_z : (FUSED ? __ldcg(p.zp + m) : p.zp[m]);
         w0 = *reinterpret_cast<const int4*>(p.wsum + n0);
         w1 = *reinterpret_cast<const int4*>(p.wsum + n0 + 4);
       }
@@ -361,7 +497,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         v[0] -= z * w0.x; v[1] -= z * w0.y; v[2] -= z * w0.z; v[3] -= z * w0.w;
         v[4] -= z * w1.x; v[5] -= z * w1.y; v[6] -= z * w1.z; v[7] -= z * w1.w;
       }
-      const float sxm = pre ? e_sx : p.sx[m];
+      const float sxm = pre ? e_sx : (FUSED ? __ldcg(p.sx + m) : p.sx[m]);
       const size_t o = (size_t)m * p.N + n0;
       if (n0 + 8 <= p.N && (p.N & 7) == 0) {
         const float4 s0 = pre ? e_s0 : *reinterpret_cast<const float4*>(p.sw + n0);
@@ -389,26 +525,36 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       }
     }
   }
+  if (FUSED && tid == 0) {
+    // this CTA is past the row flags (its warp 0 waited for them): once every CTA has said so, the flags of this
+    // launch are history and the generation moves on for the next launch on this workspace
+    __threadfence();
+    if (atomicAdd(p.sync_words + kExitWord, 1u) == gridDim.x - 1) {
+      p.sync_words[kExitWord] = 0u;
+      __threadfence();
+      atomicAdd(p.sync_words + kGenWord, 1u);
+    }
+  }
 }
 
 struct DecodePlan {
-  int nt, C, stages, act_pitch, max_blocks, grid, log2S, P;
+  int nt, C, stages, act_pitch, max_blocks, grid, log2S, P, region;
   size_t smem;
 };
 
 // Cached answers of cudaOccupancyMaxActiveClusters, keyed by (device, variant, shared memory).
 struct ClusterCacheEntry {
-  int device, nt, C;
+  int device, nt, C, fused;
   size_t smem;
   int clusters;
 };
 std::mutex g_cache_mutex;
-ClusterCacheEntry g_cache[64];
+ClusterCacheEntry g_cache[128];
 int g_cache_size = 0;
 
-template <int NT, int C>
+template <int NT, int C, bool FUSED>
 cudaError_t launch_variant(const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
-  auto kern = gemm_decode_kernel<NT, C>;
+  auto kern = gemm_decode_kernel<NT, C, FUSED>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -433,38 +579,45 @@ cudaError_t launch_variant(const DecodeParams& p, int grid, size_t smem, cudaStr
   return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
-cudaError_t dispatch(int nt, int C, const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
+template <bool FUSED>
+cudaError_t dispatch_f(int nt, int C, const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
   if (C == 1) {
-    if (nt == 1) return launch_variant<1, 1>(p, grid, smem, st, max_clusters);
-    if (nt == 2) return launch_variant<2, 1>(p, grid, smem, st, max_clusters);
-    return launch_variant<4, 1>(p, grid, smem, st, max_clusters);
+    if (nt == 1) return launch_variant<1, 1, FUSED>(p, grid, smem, st, max_clusters);
+    if (nt == 2) return launch_variant<2, 1, FUSED>(p, grid, smem, st, max_clusters);
+    return launch_variant<4, 1, FUSED>(p, grid, smem, st, max_clusters);
   }
   if (C == 2) {
-    if (nt == 1) return launch_variant<1, 2>(p, grid, smem, st, max_clusters);
-    if (nt == 2) return launch_variant<2, 2>(p, grid, smem, st, max_clusters);
-    return launch_variant<4, 2>(p, grid, smem, st, max_clusters);
+    if (nt == 1) return launch_variant<1, 2, FUSED>(p, grid, smem, st, max_clusters);
+    if (nt == 2) return launch_variant<2, 2, FUSED>(p, grid, smem, st, max_clusters);
+    return launch_variant<4, 2, FUSED>(p, grid, smem, st, max_clusters);
   }
-  if (nt == 1) return launch_variant<1, 4>(p, grid, smem, st, max_clusters);
-  if (nt == 2) return launch_variant<2, 4>(p, grid, smem, st, max_clusters);
-  return launch_variant<4, 4>(p, grid, smem, st, max_clusters);
+  if (nt == 1) return launch_variant<1, 4, FUSED>(p, grid, smem, st, max_clusters);
+  if (nt == 2) return launch_variant<2, 4, FUSED>(p, grid, smem, st, max_clusters);
+  return launch_variant<4, 4, FUSED>(p, grid, smem, st, max_clusters);
 }
 
-int max_active_clusters(int device, int nt, int C, size_t smem) {
+cudaError_t dispatch(bool fused, int nt, int C, const DecodeParams& p, int grid, size_t smem, cudaStream_t st, int* max_clusters) {
+  return fused ? dispatch_f<true>(nt, C, p, grid, smem, st, max_clusters) : dispatch_f<false>(nt, C, p, grid, smem, st, max_clusters);
+}
+
+int max_active_clusters(int device, int nt, int C, bool fused, size_t smem) {
   std::lock_guard<std::mutex> lock(g_cache_mutex);
   for (int i = 0; i < g_cache_size; ++i)
-    if (g_cache[i].device == device && g_cache[i].nt == nt && g_cache[i].C == C && g_cache[i].smem == smem) return g_cache[i].clusters;
+    if (g_cache[i].device == device && g_cache[i].nt == nt && g_cache[i].C == C && g_cache[i].fused == (int)fused && g_cache[i].smem == smem)
+      return g_cache[i].clusters;
   int n = 0;
   DecodeParams dummy = {};
-  if (dispatch(nt, C, dummy, C, smem, nullptr, &n) != cudaSuccess) {
+  if (dispatch(fused, nt, C, dummy, C, smem, nullptr, &n) != cudaSuccess) {
     cudaGetLastError();
     n = 0;
   }
-  if (g_cache_size < 64) g_cache[g_cache_size++] = {device, nt, C, smem, n};
+  if (g_cache_size < 128) g_cache[g_cache_size++] = {device, nt, C, (int)fused, smem, n};
   return n;
 }
 
-// Shared-memory plan for M tokens; stages == 0 means the shape does not fit this kernel.
-DecodePlan decode_plan(int M, const xq_weights* w) {
+// Shared-memory plan for M tokens; stages == 0 means the shape does not fit this kernel.  rot_bytes > 0: the fused
+// form, whose rotation scratch shares the region of the token slice and the partial tiles.
+DecodePlan decode_plan(int M, const xq_weights* w, size_t rot_bytes = 0) {
   DecodePlan d = {};
   if (M < 1 || M > XQ_DECODE_MAX_M || w->Kp % XQ_K_GROUP != 0) return d;
   d.nt = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
@@ -496,12 +649,13 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
       if (P < 1 || P > item_chunks_min) break;  // every piece holds at least one chunk
       const size_t tiles = (size_t)((max_blocks + C - 1) / C) * C * S * 16 * MT * 4;
       const size_t misc = 2 * kMaxStages * 8 + 64 + 128;
-      if (act + tiles + misc + 16 * (size_t)kStageBytes > cap) break;
-      const int room = (int)((cap - act - tiles - misc) / kStageBytes);
+      const size_t region = ((act + tiles > rot_bytes ? act + tiles : rot_bytes) + 127) / 128 * 128;
+      if (region + misc + 16 * (size_t)kStageBytes > cap) break;
+      const int room = (int)((cap - region - misc) / kStageBytes);
       const int want = ((max_blocks << log2S) + kConsumerWarps - 1) / kConsumerWarps * P * kConsumerWarps;
       const int stg = (room >= 48 && want > 32) ? 48 : ((room >= 32 && want > 16) ? 32 : 16);
-      const size_t smem = act + tiles + misc + (size_t)stg * kStageBytes;
-      const int fit = max_active_clusters(w->device, d.nt, C, smem);
+      const size_t smem = region + misc + (size_t)stg * kStageBytes;
+      const int fit = max_active_clusters(w->device, d.nt, C, rot_bytes > 0, smem);
       if (fit < 1) break;
       if (pass == 1 || fit >= clusters) {
         d.C = C;
@@ -512,6 +666,7 @@ DecodePlan decode_plan(int M, const xq_weights* w) {
         d.smem = smem;
         d.log2S = log2S;
         d.P = P;
+        d.region = (int)region;
         return d;
       }
       clusters = fit;
@@ -530,11 +685,10 @@ bool xq_decode_shape(int32_t M, const xq_weights* w, int* padded_tokens, int* cl
   return true;
 }
 
-cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
-                                  void* out, int32_t* acc_opt, int32_t* status, cudaStream_t st) {
-  const DecodePlan d = decode_plan(M, w);
-  if (d.stages < 16) return cudaErrorNotSupported;
-  DecodeParams p;
+namespace {
+void fill_params(DecodeParams& p, const DecodePlan& d, const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
+                 void* out, int32_t* acc_opt, int32_t* status) {
+  p = {};
   p.W = w->packed;
   p.sw = w->s_w;
   p.Xq = Xq;
@@ -554,5 +708,42 @@ cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int3
   p.max_blocks = d.max_blocks;
   p.log2S = d.log2S;
   p.P = d.P;
-  return dispatch(d.nt, d.C, p, d.grid, d.smem, st, nullptr);
+  p.region_bytes = d.region;
+}
+}  // namespace
+
+cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
+                                  void* out, int32_t* acc_opt, int32_t* status, cudaStream_t st) {
+  const DecodePlan d = decode_plan(M, w);
+  if (d.stages < 16) return cudaErrorNotSupported;
+  DecodeParams p;
+  fill_params(p, d, Xq, sx, zp, M, w, out, acc_opt, status);
+  return dispatch(false, d.nt, d.C, p, d.grid, d.smem, st, nullptr);
+}
+
+bool xq_linear_decode_supported(int32_t M, const xq_weights* w) {
+  if (M < 1 || M > XQ_DECODE_MAX_M || w->heads != 1 || !w->hp_signs || !xqrot::plan_supported(w->plan)) return false;
+  return decode_plan(M, w, xqrot::row_layout(w->plan).total).stages >= 16;
+}
+
+cudaError_t xq_launch_linear_decode(const void* X, int64_t ldx, uint8_t* Xq, float* sx, int32_t* zp, int32_t M, const xq_weights* w,
+                                    void* out, int32_t* header, cudaStream_t st) {
+  if (M < 1 || M > XQ_DECODE_MAX_M || w->heads != 1 || !w->hp_signs || !xqrot::plan_supported(w->plan)) return cudaErrorNotSupported;
+  const xq_hadamard_plan_t& pl = w->plan;
+  const DecodePlan d = decode_plan(M, w, xqrot::row_layout(pl).total);
+  if (d.stages < 16) return cudaErrorNotSupported;
+  DecodeParams p;
+  fill_params(p, d, Xq, sx, zp, M, w, out, nullptr, header);
+  p.X = (const __nv_bfloat16*)X;
+  p.ldx = ldx;
+  p.plan = pl;
+  p.gamma = (float)(1.0 / sqrt((double)pl.Kp));
+  p.Hsigns = (const __nv_bfloat16*)w->hp_signs;
+  p.Xq_w = Xq;
+  p.sx_w = sx;
+  p.zp_w = zp;
+  p.sync_words = (uint32_t*)header;
+  const int n = 1 << pl.log2n;
+  p.rot_threads = 32 * ((pl.p + 15) / 16) * (n > 128 ? 2 : 1);
+  return dispatch(true, d.nt, d.C, p, d.grid, d.smem, st, nullptr);
 }

@@ -146,6 +146,13 @@ cudaError_t xq_launch_weight_sums(const uint8_t* blocks, int32_t Np, int32_t Kpp
 // zp (optional, here and below): per-token zero points; the epilogue then removes zp[m] * w_sum[n].
 cudaError_t xq_launch_gemm_decode(const uint8_t* Xq, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
                                   void* out, int32_t* acc_opt, int32_t* status, cudaStream_t st);
+// The whole layer for M <= 32 tokens in one launch: the decode kernel with the online step (pad, rotate, quantize)
+// inside.  Xq, sx, zp (zp null: symmetric codes) are workspace arrays the kernel fills and reads; header is the
+// workspace header (status word, generation, exit count, row flags).  cudaErrorNotSupported (nothing launched) when
+// the plan or the shape is not one it takes.
+bool xq_linear_decode_supported(int32_t M, const xq_weights* w);
+cudaError_t xq_launch_linear_decode(const void* X, int64_t ldx, uint8_t* Xq, float* sx, int32_t* zp, int32_t M, const xq_weights* w,
+                                    void* out, int32_t* header, cudaStream_t st);
 // True when M tokens against w run in the decode kernel; then also its padded token count and cluster size.
 bool xq_decode_shape(int32_t M, const xq_weights* w, int* padded_tokens, int* cluster);
 // Tile shape the tensor-core kernel picks: 0 = 128 tokens x 256 channels, 1 = 256 x 256, 2 = 256 x 128.

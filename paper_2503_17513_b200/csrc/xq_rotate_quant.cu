@@ -6,6 +6,7 @@
 #include "xq_internal.h"
 #include "xq_hadamard.cuh"
 #include "xq_ptx.cuh"
+#include "xq_rotate_row.cuh"
 
 using namespace xqhad;
 
@@ -102,18 +103,8 @@ __global__ void __launch_bounds__(256) rotate_quant_general_kernel(const __nv_bf
 }
 
 // ---------------------------------------------------------------------------------------------
-// Tensor-core kernel for p > 1, 32 <= n <= 256, ceil(K / n) <= 64.
-//
-// With the row viewed as V[a][b] (a < p, b < n) the layer needs Y = H_p^T V S_n.  The outer
-// factor goes first, on the raw bf16 inputs: +-1 times bf16 is exact and the sums accumulate in
-// fp32, so H_p^T V runs as m16n8k16 bf16 MMAs (A = H_p^T built from the character table, B = V
-// read from shared memory with a transposing ldmatrix).  Warp (mt, bc) owns 16 rows a' and a
-// chunk of NB = min(n, 128) columns b, so the Sylvester butterflies along b stay inside the
-// warp: bit 0 inside a thread, bits 1-2 across the four lanes of a quad, higher bits across
-// accumulator registers.  For n = 256 the last butterfly crosses the two column chunks through
-// shared memory.  absmax, scale, rounding and nibble packing follow in registers; the packed row
-// leaves through shared memory as 128-bit stores (and, on request, as the byte-per-code operand
-// format of the tcgen05 GEMM).
+// Tensor-core kernel for p > 1, 32 <= n <= 256, ceil(K / n) <= 64: one CTA per row, all of its warps on
+// that row (the row routine and its description: xq_rotate_row.cuh).
 // ---------------------------------------------------------------------------------------------
 template <int LOG2NB, int KS>
 __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx,
@@ -124,13 +115,12 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
   // sfb != null: MXFP4 instead of per-row INT4 -- a shared exponent per 32 channels, E2M1 codes; Xq then has the row
   // pitch Kq / 2 and the scale bytes go to sfb in the block layout of the block-scaled GEMM (sx, zp, A8opt unused).
   constexpr int NB = 1 << LOG2NB;  // columns per warp
-  constexpr int NT8 = NB / 8;      // n-tiles per warp
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int K = pl.K, Kp = pl.Kp, p = pl.p, n = 1 << pl.log2n, q = pl.q;
   const int NC = n / NB;            // column chunks (1 or 2)
   const int pitch = n + 8;          // bf16 elements per staged row (conflict-free ldmatrix)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int mt = warp / NC, bc = warp - mt * NC;
+  const int mt = warp / NC;
   const int nthreads = blockDim.x;
 
   __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
@@ -154,11 +144,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
     for (int i = tid; i < P16 * hpitch / 8; i += nthreads) xqptx::cp_async16(Hs + 8 * i, Hsigns + 8 * i);
     xqptx::cp_async_wait_all();
     __syncthreads();
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      if (16 * ks < P16) ldmatrix_x4(afrag[ks], Hs + (16 * mt + (lane & 15)) * hpitch + 16 * ks + (lane >> 4) * 8);
-      else afrag[ks][0] = afrag[ks][1] = afrag[ks][2] = afrag[ks][3] = 0u;
-    }
+    xqrot::load_afrag<KS>(afrag, Hs, P16, hpitch, mt, lane);
   } else {
   build_chi(q, chi2, sq);
 #pragma unroll
@@ -181,6 +167,8 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
   xqptx::pdl_wait();
   __syncthreads();
 
+  const xqrot::RowSmem sm = {Xs, outp, sfs, red, exch};
+  const xqrot::RowOut out = {Xq, sx, Yopt, A8opt, zp, sfb, Kq};
   const int chunks = K / 8;  // 16-byte pieces of a row
   for (int row = blockIdx.x; row < M; row += gridDim.x) {
     const __nv_bfloat16* x = X + (long long)row * ldx;
@@ -190,166 +178,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
     }
     xqptx::cp_async_wait_all();
     __syncthreads();
-
-    float acc[NT8][4];
-#pragma unroll
-    for (int j = 0; j < NT8; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      const __nv_bfloat16* base = Xs + (16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8) * pitch + bc * NB + ((lane >> 4) & 1) * 8;
-#pragma unroll
-      for (int jp = 0; jp < NT8 / 2; ++jp) {
-        uint32_t bfr[4];
-        ldmatrix_x4_trans(bfr, base + 16 * jp);
-        xqptx::mma_bf16_16x8x16(acc[2 * jp], afrag[ks], bfr[0], bfr[1]);
-        xqptx::mma_bf16_16x8x16(acc[2 * jp + 1], afrag[ks], bfr[2], bfr[3]);
-      }
-    }
-    // Sylvester butterflies along b = 8 j + 2 t + e
-#pragma unroll
-    for (int j = 0; j < NT8; ++j) {
-      const float u0 = acc[j][0], u1 = acc[j][1], u2 = acc[j][2], u3 = acc[j][3];
-      acc[j][0] = u0 + u1; acc[j][1] = u0 - u1; acc[j][2] = u2 + u3; acc[j][3] = u2 - u3;
-    }
-#pragma unroll
-    for (int bit = 1; bit <= 2; ++bit) {
-      const float sgn = (t & bit) ? -1.f : 1.f;
-#pragma unroll
-      for (int j = 0; j < NT8; ++j)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float o = __shfl_xor_sync(0xffffffffu, acc[j][e], bit);
-          acc[j][e] = fmaf(sgn, acc[j][e], o);
-        }
-    }
-#pragma unroll
-    for (int s = 1; s < NT8; s <<= 1)
-#pragma unroll
-      for (int j = 0; j < NT8; ++j)
-        if (!(j & s)) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float u = acc[j][e], w = acc[j | s][e];
-            acc[j][e] = u + w;
-            acc[j | s][e] = u - w;
-          }
-        }
-    if (NC == 2) {
-      // last butterfly (bit log2(NB) of b) between the two column chunks
-      float* mine = exch + ((size_t)(16 * mt + g) * n + bc * NB + 2 * t);
-#pragma unroll
-      for (int j = 0; j < NT8; ++j) {
-        *reinterpret_cast<float2*>(mine + 8 * j) = make_float2(acc[j][0], acc[j][1]);
-        *reinterpret_cast<float2*>(mine + 8 * n + 8 * j) = make_float2(acc[j][2], acc[j][3]);
-      }
-      __syncthreads();
-      const float* other = exch + ((size_t)(16 * mt + g) * n + (bc ^ 1) * NB + 2 * t);
-      const float sgn = bc ? -1.f : 1.f;
-#pragma unroll
-      for (int j = 0; j < NT8; ++j) {
-        const float2 o0 = *reinterpret_cast<const float2*>(other + 8 * j);
-        const float2 o1 = *reinterpret_cast<const float2*>(other + 8 * n + 8 * j);
-        acc[j][0] = fmaf(sgn, acc[j][0], o0.x);
-        acc[j][1] = fmaf(sgn, acc[j][1], o0.y);
-        acc[j][2] = fmaf(sgn, acc[j][2], o1.x);
-        acc[j][3] = fmaf(sgn, acc[j][3], o1.y);
-      }
-    }
-    // scale by 1/sqrt(K'), per-token absmax
-    // (rows of the tile padding hold zeros: harmless, the asymmetric range contains zero anyway)
-    float vmax = 0.f, vmin = 0.f;
-#pragma unroll
-    for (int j = 0; j < NT8; ++j)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        acc[j][e] *= gamma;
-        vmax = fmaxf(vmax, acc[j][e]);
-        vmin = fminf(vmin, acc[j][e]);
-      }
-    RowQuant rq = row_quant_sym(0.f);
-    if (sfb) {
-      // MXFP4: the group of 32 channels is four neighbouring column tiles of one row, spread over the quad
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const int a2 = 16 * mt + g + 8 * r;
-#pragma unroll
-        for (int gq = 0; gq < NT8 / 4; ++gq) {
-          float gm = 0.f;
-#pragma unroll
-          for (int j = 4 * gq; j < 4 * gq + 4; ++j) gm = fmaxf(gm, fmaxf(fabsf(acc[j][2 * r]), fabsf(acc[j][2 * r + 1])));
-          gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, 1));
-          gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, 2));
-          const int e = mx_shared_exp(gm);
-          const float inv = mx_inv_scale(e);
-#pragma unroll
-          for (int j = 4 * gq; j < 4 * gq + 4; ++j) {
-            uint32_t w = mx_e2m1_pair(acc[j][2 * r] * inv, acc[j][2 * r + 1] * inv) << (8 * t);
-            w |= __shfl_xor_sync(0xffffffffu, w, 1);
-            w |= __shfl_xor_sync(0xffffffffu, w, 2);
-            if (t == 0 && a2 < p) outp[(a2 * n + bc * NB) / 8 + j] = w;
-          }
-          if (t == 0 && a2 < p) sfs[(a2 * n + bc * NB) / 32 + gq] = (uint8_t)(e + 127);
-        }
-      }
-    } else if (zp) {
-      vmax = block_max(vmax, red);
-      vmin = -block_max(-vmin, red);
-      rq = row_quant_asym(vmin, vmax);
-    } else {
-      rq = row_quant_sym(block_max(fmaxf(vmax, -vmin), red));
-    }
-    const float s = rq.s;
-    // quantize, pack: the quad's four bytes of one (row, j) form one word of 8 codes
-#pragma unroll
-    for (int r = 0; r < 2 && !sfb; ++r) {
-      const int a2 = 16 * mt + g + 8 * r;
-#pragma unroll
-      for (int j = 0; j < NT8; ++j) {
-        const int lo = row_code(rq, acc[j][2 * r]);
-        const int hi = row_code(rq, acc[j][2 * r + 1]);
-        uint32_t w = (uint32_t)((lo & 0xF) | ((hi & 0xF) << 4)) << (8 * t);
-        w |= __shfl_xor_sync(0xffffffffu, w, 1);
-        w |= __shfl_xor_sync(0xffffffffu, w, 2);
-        if (t == 0 && a2 < p) outp[(a2 * n + bc * NB) / 8 + j] = w;
-      }
-    }
-    if (Yopt) {
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const int a2 = 16 * mt + g + 8 * r;
-        if (a2 < p) {
-          float* yrow = Yopt + (long long)row * Kp + a2 * n + bc * NB + 2 * t;
-#pragma unroll
-          for (int j = 0; j < NT8; ++j) *reinterpret_cast<float2*>(yrow + 8 * j) = make_float2(acc[j][2 * r], acc[j][2 * r + 1]);
-        }
-      }
-    }
-    __syncthreads();
-    if (tid == 0 && !sfb) {
-      sx[row] = s;
-      if (zp) zp[row] = rq.z;
-    }
-    if (sfb) {
-      // scale bytes into their blocks; padding up to Kq: unit scales and zero codes (never a NaN scale byte)
-      for (int i = tid; i < Kq / 32; i += nthreads) sfb[xq_mx_sf_offset(row, i, Kq)] = i < Kp / 32 ? sfs[i] : (uint8_t)127;
-      for (int i = tid; i < (Kq - Kp) / 8; i += nthreads) *reinterpret_cast<uint32_t*>(Xq + (long long)row * (Kq / 2) + Kp / 2 + 4 * i) = 0u;
-    }
-    uint4* dst = reinterpret_cast<uint4*>(Xq + (long long)row * ((sfb ? Kq : Kp) / 2));
-    for (int i = tid; i < Kp / 32; i += nthreads) {
-      const uint4 v = reinterpret_cast<const uint4*>(outp)[i];
-      dst[i] = v;
-      if (A8opt) {
-        uint4 e0, e1;
-        xqptx::split16(v.x, e0.x, e0.y);
-        xqptx::split16(v.y, e0.z, e0.w);
-        xqptx::split16(v.z, e1.x, e1.y);
-        xqptx::split16(v.w, e1.z, e1.w);
-        uint4* d8 = reinterpret_cast<uint4*>(A8opt + (long long)row * Kp);
-        d8[2 * i] = e0;
-        d8[2 * i + 1] = e1;
-      }
-    }
-    __syncthreads();
+    xqrot::rotate_row<LOG2NB, KS>(pl, gamma, afrag, sm, out, row, tid, nthreads, xqrot::CtaSync());
   }
 }
 
@@ -361,7 +190,7 @@ cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_p
   size_t smem = (size_t)KS * 16 * (n + 8) * 2 + (size_t)pl.Kp / 2 + (size_t)pl.Kp / 32 + 16 + 128 + (size_t)(3 * pl.q + 1) + 32;
   if (mx) Xq = mx->codes;
   if (Hsigns) smem += (size_t)MT * 16 * (MT * 16 + 8) * 2;
-  if (NC == 2) smem += (size_t)MT * 16 * n * 4;
+  if (NC == 2) smem += (size_t)MT * 8 * n * 4;
   auto kern = rotate_quant_tc_kernel<LOG2NB, KS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
@@ -468,9 +297,7 @@ cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const 
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
   const int n = 1 << pl.log2n;
   const int rows_a = (pl.K + n - 1) / n;
-  const int MT = (pl.p + 15) / 16;
-  const bool tc = pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 8 && pl.K % 8 == 0 && rows_a <= 64 &&
-                  MT * (n > 128 ? 2 : 1) <= 16;
+  const bool tc = xqrot::plan_supported(pl);
   // many rows, or an order that only the multi-row-group kernel and the general kernel take
   if ((M >= XQ_ROTATE_ROWS_MIN_M || !tc) && xq_rotate_rows_supported(pl))
     return xq_launch_rotate_rows(X, M, ldx, pl, Xq, sx, Yopt, A8opt, zp, sms, st);
@@ -495,9 +322,7 @@ cudaError_t xq_launch_rotate_tc_mx(const void* X, int32_t M, int64_t ldx, const 
   const float gamma = (float)(1.0 / sqrt((double)pl.Kp));
   const int n = 1 << pl.log2n;
   const int rows_a = (pl.K + n - 1) / n;
-  const int MT = (pl.p + 15) / 16;
-  const bool tc = pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 8 && pl.K % 8 == 0 && rows_a <= 64 &&
-                  MT * (n > 128 ? 2 : 1) <= 16;
+  const bool tc = xqrot::plan_supported(pl);
   if (!tc || pl.Kp % 32 != 0) return cudaErrorNotSupported;
   const int ks = (rows_a + 15) / 16;
   switch (pl.log2n) {
