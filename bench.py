@@ -385,6 +385,8 @@ class Bench:
                         xq.xq_mx_expanded_linear(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
                     elif asym:
                         xq.xq_expanded_linear_asym(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
+                    elif args.one_launch and M <= 32:
+                        xq.xq_expanded_linear_one_launch(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
                     else:
                         xq.xq_expanded_linear(X[n], Wt[n][l], out[n], wsp[n], stream=stream)
 
@@ -530,6 +532,8 @@ def main():
     ap.add_argument("--only", action="store_true", help="time the named workload alone (no per_workload object)")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--one-launch", action="store_true",
+                    help="M <= 32: run each linear as xq_expanded_linear_one_launch (the online step inside the product kernel)")
     ap.add_argument("--fmt", default="int4", choices=["int4", "mxfp4"],
                     help="number format of weights and activations: INT4 with per-row scales (default) or MXFP4")
     ap.add_argument("--act", default="sym", choices=["sym", "asym"],

@@ -128,6 +128,21 @@ xq_status xq_w4a4_gemm(const uint8_t* Xq_dev, const float* s_x_dev, int32_t M, c
 xq_status xq_expanded_linear(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w,
                              void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
 
+/* xq_expanded_linear for M <= 32 tokens as ONE kernel launch (Sec. 3: the rotation of the activations is an online
+ * step of the layer; here it runs inside the product's launch).  Every CTA first requests its share of the weights,
+ * which do not depend on the tokens; CTA r < M meanwhile pads, rotates and quantizes token row r, writes codes and
+ * scale to the workspace and counts the row as published; every CTA waits, time-bounded, until M rows are counted
+ * and goes on as xq_w4a4_gemm does.  asym != 0: asymmetric codes (as xq_expanded_linear_asym).  The output bits
+ * are those of xq_expanded_linear.  Measured on B200 inside a captured, programmatically chained stream the two-kernel
+ * form is the faster one (the chain already overlaps the next product's weight requests with the rotation); this
+ * form halves the number of launches, which is what counts where the host's launch rate is the limit.
+ * Limits: the plans of the tensor-core row routine (p > 1, 32 <= 2^k <= 256, K a multiple of 8, at most 64 input
+ * rows of 2^k channels, at most 16 warps per row) on weights made by xq_prepare_weights / xq_weights_import with
+ * p <= 256; otherwise UNSUPPORTED_ORDER (also M > 32).  The two counters it keeps in the workspace header are back at zero
+ * when the launch ends; after a device-side time-out re-initialise the workspace. */
+xq_status xq_expanded_linear_one_launch(const void* X_bf16_dev, int32_t M, int64_t ldx, const xq_weights* w, int32_t asym,
+                                        void* out_bf16_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
 /* The same three calls with per-token ASYMMETRIC activation codes (Sec. 4: the setting of the
  * paper's experiments; weights stay symmetric per channel).  For each row, with y as above,
  * lo = min(0, min y), hi = max(0, max y):

@@ -418,8 +418,10 @@ xq_status gemm_impl(const uint8_t* Xq, const float* s_x, const int32_t* zp, bool
   return XQ_OK;
 }
 
+// one_launch: the form for M <= 32 tokens with the online step inside the product kernel (UNSUPPORTED_ORDER when the
+// plan or the shape is not one it takes); otherwise the rotate + quantize kernel followed by the product kernel.
 xq_status linear_impl(const void* X, int32_t M, int64_t ldx, const xq_weights* w, bool asym, void* out, void* ws,
-                      size_t ws_bytes, void* stream) {
+                      size_t ws_bytes, void* stream, bool one_launch = false) {
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X || !out || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
@@ -431,13 +433,11 @@ xq_status linear_impl(const void* X, int32_t M, int64_t ldx, const xq_weights* w
   float* sx = (float*)(base + L.sx);
   int32_t* zp = asym ? (int32_t*)(base + L.zp) : nullptr;
   cudaStream_t st = (cudaStream_t)stream;
-  if (M <= XQ_DECODE_MAX_M) {  // one launch: the online step inside the product kernel
+  if (one_launch) {
     const cudaError_t e = xq_launch_linear_decode(X, ldx, Xq, sx, zp, M, w, out, (int32_t*)ws, st);
     if (e == cudaSuccess) return XQ_OK;
-    if (e != cudaErrorNotSupported) {
-      cudaGetLastError();
-      return XQ_ERR_CUDA;
-    }
+    cudaGetLastError();
+    return e == cudaErrorNotSupported ? XQ_ERR_UNSUPPORTED_ORDER : XQ_ERR_CUDA;
   }
   uint8_t* A8 = xq_gemm_wants_a8(M, w) ? base + L.a8 : nullptr;
   if (xq_launch_rotate_for(w, X, M, ldx, Xq, sx, A8, zp, st) != cudaSuccess ||
@@ -486,6 +486,11 @@ xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_wei
 xq_status xq_expanded_linear_asym(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out, void* ws,
                                   size_t ws_bytes, void* stream) {
   return linear_impl(X, M, ldx, w, true, out, ws, ws_bytes, stream);
+}
+
+xq_status xq_expanded_linear_one_launch(const void* X, int32_t M, int64_t ldx, const xq_weights* w, int32_t asym, void* out,
+                                        void* ws, size_t ws_bytes, void* stream) {
+  return linear_impl(X, M, ldx, w, asym != 0, out, ws, ws_bytes, stream, true);
 }
 
 }  // extern "C"

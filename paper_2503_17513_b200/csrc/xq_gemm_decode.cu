@@ -27,12 +27,11 @@
 // the product).  The weights do not depend on the tokens, so every CTA requests its first ring-full before
 // anything else; meanwhile CTA r (r < M) pads, rotates and quantizes token row r with the routine of
 // xq_rotate_row.cuh (its scratch lies where the token slice and the partial tiles go later), writes the packed
-// codes and the scale to the workspace and publishes a per-row flag (release); every CTA then waits, time-bounded,
-// for the M flags (acquire) and reads its K slice of the codes from L2.  Rotating CTAs never wait before they
+// codes and the scale to the workspace and counts the row as published (release); every CTA then waits, time-bounded,
+// until M rows are counted (acquire) and reads its K slice of the codes from L2.  Rotating CTAs never wait before they
 // publish, so the launch makes progress whenever its first M CTAs run; a wait that runs out records
-// XQ_ERR_TIMEOUT and the CTA leaves through the normal exits.  Flags carry the launch's generation number, kept
-// in the workspace header and advanced by the last CTA to leave, so that replays of a captured launch need no
-// host-side reset.
+// XQ_ERR_TIMEOUT and the CTA leaves through the normal exits.  The last CTA to leave puts the two counters in the
+// workspace header back to zero, so that replays of a captured launch need no host-side reset.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -81,24 +80,24 @@ struct DecodeParams {
   uint8_t* Xq_w;
   float* sx_w;
   int32_t* zp_w;                // null: symmetric codes
-  uint32_t* sync_words;         // workspace header words: [1] generation, [2] CTAs that have left, [32 + r] flag of row r
+  uint32_t* sync_words;         // workspace header words: [1] token rows published so far, [2] CTAs that have left
   int rot_threads;              // threads of a row group: 32 x tiles of 16 output rows x column chunks
 };
 
-// Workspace header words of the fused form.
-constexpr int kGenWord = 1, kExitWord = 2, kFlagWord0 = 32;
+// Workspace header words of the fused form: both are zero between launches (the last CTA to leave clears them).
+constexpr int kRowsWord = 1, kExitWord = 2;
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release_u32(uint32_t* p, uint32_t v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void add_release_u32(uint32_t* p, uint32_t v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 // Rows blockIdx.x, blockIdx.x + gridDim.x, ... < M through pad + rotate + quantize by the first rot_threads threads
-// of the CTA; each finished row is published with its flag.  `region` is this CTA's scratch.
+// of the CTA; each finished row is published by counting it (release).  `region` is this CTA's scratch.
 template <int LOG2NB, int KS>
 __device__ __noinline__ void fused_rotate_rows(const DecodeParams& p, unsigned char* region, int tid) {
   const xq_hadamard_plan_t& pl = p.plan;
@@ -119,7 +118,6 @@ __device__ __noinline__ void fused_rotate_rows(const DecodeParams& p, unsigned c
   uint32_t afrag[KS][4];
   xqrot::load_afrag<KS>(afrag, Hs, P16, hpitch, mt, lane);
   pdl_wait();
-  const uint32_t want = ld_acquire_u32(p.sync_words + kGenWord) + 1u;
   const xqrot::RowOut out = {p.Xq_w, p.sx_w, nullptr, nullptr, p.zp_w, nullptr, 0};
   const int chunks = pl.K / 8;
   for (int row = blockIdx.x; row < p.M; row += gridDim.x) {
@@ -132,34 +130,22 @@ __device__ __noinline__ void fused_rotate_rows(const DecodeParams& p, unsigned c
     sync();
     xqrot::rotate_row<LOG2NB, KS>(pl, p.gamma, afrag, sm, out, row, tid, nthreads, sync);
     // rotate_row ends with the group's barrier: every thread's stores of the row precede it
-    if (tid == 0) {
-      __threadfence();
-      st_release_u32(p.sync_words + kFlagWord0 + row, want);
-    }
+    if (tid == 0) add_release_u32(p.sync_words + kRowsWord, 1u);
   }
 }
 
 __device__ __forceinline__ void fused_rotate_dispatch(const DecodeParams& p, unsigned char* region, int tid) {
   const int n = 1 << p.plan.log2n, ks = ((p.plan.K + n - 1) / n + 15) / 16;
-  switch (p.plan.log2n) {
-    case 5:
-      if (ks == 1) fused_rotate_rows<5, 1>(p, region, tid);
-      else if (ks == 2) fused_rotate_rows<5, 2>(p, region, tid);
-      else if (ks == 3) fused_rotate_rows<5, 3>(p, region, tid);
-      else fused_rotate_rows<5, 4>(p, region, tid);
-      break;
-    case 6:
-      if (ks == 1) fused_rotate_rows<6, 1>(p, region, tid);
-      else if (ks == 2) fused_rotate_rows<6, 2>(p, region, tid);
-      else if (ks == 3) fused_rotate_rows<6, 3>(p, region, tid);
-      else fused_rotate_rows<6, 4>(p, region, tid);
-      break;
-    default:
-      if (ks == 1) fused_rotate_rows<7, 1>(p, region, tid);
-      else if (ks == 2) fused_rotate_rows<7, 2>(p, region, tid);
-      else if (ks == 3) fused_rotate_rows<7, 3>(p, region, tid);
-      else fused_rotate_rows<7, 4>(p, region, tid);
-      break;
+  if (p.plan.log2n == 5) {
+    if (ks == 1) fused_rotate_rows<5, 1>(p, region, tid);
+    else if (ks == 2) fused_rotate_rows<5, 2>(p, region, tid);
+    else if (ks == 3) fused_rotate_rows<5, 3>(p, region, tid);
+    else fused_rotate_rows<5, 4>(p, region, tid);
+  } else {  // chunks of 64 columns
+    if (ks == 1) fused_rotate_rows<6, 1>(p, region, tid);
+    else if (ks == 2) fused_rotate_rows<6, 2>(p, region, tid);
+    else if (ks == 3) fused_rotate_rows<6, 3>(p, region, tid);
+    else fused_rotate_rows<6, 4>(p, region, tid);
   }
 }
 
@@ -256,6 +242,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
     if (active && !exists(n)) active = false;
     uint32_t idle = 0;
     uint64_t t_idle = 0;
+    const uint64_t stream_policy = l2_policy_evict_first();  // the weights pass once: keep L2 for the tokens and scales
     while (__any_sync(0xffffffffu, active)) {
       bool ready = false;
       int stage = 0;
@@ -274,7 +261,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         const uint32_t bytes = (uint32_t)ng * XQ_GROUP_BYTES;
         const unsigned char* src = p.W + ((size_t)(b0 + (t >> p.log2S)) * p.k_groups + g0 + 4 * c_lo) * XQ_GROUP_BYTES;
         mbar_expect_tx(&full[stage], bytes);
-        bulk_g2s(ring + (size_t)stage * kStageBytes, src, bytes, &full[stage]);
+        bulk_g2s_hint(ring + (size_t)stage * kStageBytes, src, bytes, &full[stage], stream_policy);
         if (stage == lane) ++use_a; else ++use_b;
         n = next_n(n);
         if (!exists(n)) active = false;
@@ -310,12 +297,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
       else pdl_wait();
       bar_sync(1, kConsumerThreads);  // the scratch of the rotation is free: the token slice goes there
       if (warp == 0) {
-        const uint32_t want = ld_acquire_u32(p.sync_words + kGenWord) + 1u;
+        // one lane per CTA watches the count of published rows, with a pause between looks: the word sits in one L2
+        // slice that every weight stream also crosses
         bool seen = true;
-        if (lane < p.M) {
-          const uint32_t* flag = p.sync_words + kFlagWord0 + lane;
+        if (lane == 0) {
           uint64_t t0 = 0;
-          for (uint32_t i = 1; ld_acquire_u32(flag) != want; ++i) {
+          for (uint32_t i = 1; ld_acquire_u32(p.sync_words + kRowsWord) < (uint32_t)p.M; ++i) {
+            __nanosleep(100);
             if ((i & 31u) == 0u) {
               const uint64_t now = globaltimer_ns();
               if (t0 == 0) t0 = now;
@@ -325,11 +313,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
               }
             }
           }
+          if (!seen) {
+            *failed = 1;
+            atomicExch(p.status, (int)XQ_ERR_TIMEOUT);
+          }
         }
-        if (!__all_sync(0xffffffffu, seen) && lane == 0) {
-          *failed = 1;
-          atomicExch(p.status, (int)XQ_ERR_TIMEOUT);
-        }
+        __syncwarp();
       }
     }
     // token rows beyond M are zero
@@ -526,13 +515,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
     }
   }
   if (FUSED && tid == 0) {
-    // this CTA is past the row flags (its warp 0 waited for them): once every CTA has said so, the flags of this
-    // launch are history and the generation moves on for the next launch on this workspace
-    __threadfence();
+    // this CTA is past the row count (its warp 0 waited for it): once every CTA has said so, both words go back to
+    // zero for the next launch on this workspace (which looks at them only after this grid has completed)
     if (atomicAdd(p.sync_words + kExitWord, 1u) == gridDim.x - 1) {
+      p.sync_words[kRowsWord] = 0u;
       p.sync_words[kExitWord] = 0u;
-      __threadfence();
-      atomicAdd(p.sync_words + kGenWord, 1u);
     }
   }
 }
@@ -743,7 +730,6 @@ cudaError_t xq_launch_linear_decode(const void* X, int64_t ldx, uint8_t* Xq, flo
   p.sx_w = sx;
   p.zp_w = zp;
   p.sync_words = (uint32_t*)header;
-  const int n = 1 << pl.log2n;
-  p.rot_threads = 32 * ((pl.p + 15) / 16) * (n > 128 ? 2 : 1);
+  p.rot_threads = 32 * ((pl.p + 15) / 16) * xqrot::row_chunks(pl);
   return dispatch(true, d.nt, d.C, p, d.grid, d.smem, st, nullptr);
 }

@@ -61,6 +61,21 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, u
                : "memory");
 }
 
+// The same with an L2 eviction hint.  evict-first suits data that is read once (a weight stream): it leaves the
+// small tensors that the same kernel reads with latency on the critical path (token rows, codes, scales, sign
+// images) resident in L2 instead of being pushed out by the stream.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar, uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                   smem_u32(dst_smem)),
+               "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+               : "memory");
+}
+
 // Time-bounded wait shared by the pipelined kernels: polls the barrier phase for at most about
 // one second of wall time.  On expiry (or when another thread of the CTA already gave up) it
 // raises the CTA-wide flag `*failed`, records `timeout_code` in the global status word and

@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
   constexpr int NB = 1 << LOG2NB;  // columns per warp
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int K = pl.K, Kp = pl.Kp, p = pl.p, n = 1 << pl.log2n, q = pl.q;
-  const int NC = n / NB;            // column chunks (1 or 2)
+  const int NC = n / NB;            // column chunks (1, 2 or 4)
   const int pitch = n + 8;          // bf16 elements per staged row (conflict-free ldmatrix)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int mt = warp / NC;
@@ -186,11 +186,11 @@ template <int LOG2NB, int KS>
 cudaError_t launch_tc(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t& pl, float gamma, uint8_t* Xq, float* sx,
                       float* Yopt, uint8_t* A8opt, const void* Hsigns, int32_t* zp, int sms, cudaStream_t st,
                       const xq_mx_out* mx = nullptr) {
-  const int n = 1 << pl.log2n, NB = 1 << LOG2NB, NC = n / NB, MT = (pl.p + 15) / 16;
+  const int n = 1 << pl.log2n, NB = 1 << LOG2NB, NC = n / NB, MT = (pl.p + 15) / 16;  // NC = xqrot::row_chunks(pl)
   size_t smem = (size_t)KS * 16 * (n + 8) * 2 + (size_t)pl.Kp / 2 + (size_t)pl.Kp / 32 + 16 + 128 + (size_t)(3 * pl.q + 1) + 32;
   if (mx) Xq = mx->codes;
   if (Hsigns) smem += (size_t)MT * 16 * (MT * 16 + 8) * 2;
-  if (NC == 2) smem += (size_t)MT * 8 * n * 4;
+  if (NC > 1) smem += (size_t)MT * 8 * (n + 8) * 4;
   auto kern = rotate_quant_tc_kernel<LOG2NB, KS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
@@ -305,8 +305,7 @@ cudaError_t xq_launch_rotate_quant(const void* X, int32_t M, int64_t ldx, const 
     const int ks = (rows_a + 15) / 16;
     switch (pl.log2n) {
       case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
-      case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
-      default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
+      default: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, Hsigns, zp, sms, st);
     }
   }
   const size_t smem = sizeof(float) * (2 * (size_t)pl.Kp + 32) + (size_t)(3 * pl.q + 1) + 16;
@@ -327,8 +326,7 @@ cudaError_t xq_launch_rotate_tc_mx(const void* X, int32_t M, int64_t ldx, const 
   const int ks = (rows_a + 15) / 16;
   switch (pl.log2n) {
     case 5: return launch_tc_ks<5>(ks, X, M, ldx, pl, gamma, mx.codes, nullptr, nullptr, nullptr, Hsigns, nullptr, sms, st, &mx);
-    case 6: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, mx.codes, nullptr, nullptr, nullptr, Hsigns, nullptr, sms, st, &mx);
-    default: return launch_tc_ks<7>(ks, X, M, ldx, pl, gamma, mx.codes, nullptr, nullptr, nullptr, Hsigns, nullptr, sms, st, &mx);
+    default: return launch_tc_ks<6>(ks, X, M, ldx, pl, gamma, mx.codes, nullptr, nullptr, nullptr, Hsigns, nullptr, sms, st, &mx);
   }
 }
 

@@ -6,10 +6,11 @@
 // For p > 1, 32 <= n <= 256, ceil(K / n) <= 64.  With the row viewed as V[a][b] (a < p, b < n) the layer needs
 // Y = H_p^T V S_n.  The outer factor goes first, on the raw bf16 inputs: +-1 times bf16 is exact and the sums
 // accumulate in fp32, so H_p^T V runs as m16n8k16 bf16 MMAs (A = H_p^T, B = V read from shared memory with a
-// transposing ldmatrix).  Warp (mt, bc) owns 16 rows a' and a chunk of NB = min(n, 128) columns b, so the
-// Sylvester butterflies along b stay inside the warp: bit 0 inside a thread, bits 1-2 across the four lanes of a
-// quad, higher bits across accumulator registers.  For n = 256 the last butterfly crosses the two column chunks
-// through shared memory.  absmax, scale, rounding and nibble packing follow in registers; the packed row leaves
+// transposing ldmatrix).  Warp (mt, bc) owns 16 rows a' and a chunk of NB = min(n, 64) columns b, so the
+// Sylvester butterflies over the low bits of b stay inside the warp: bit 0 inside a thread, bits 1-2 across the four
+// lanes of a quad, higher bits across accumulator registers.  For n = 128 and 256 the last one or two butterflies
+// cross the two or four column chunks through shared memory (short chunks keep the accumulators at 32 registers
+// and put up to 16 warps on one row: the row's latency is what counts here).  absmax, scale, rounding and nibble packing follow in registers; the packed row leaves
 // through shared memory as 128-bit stores (and, on request, as the byte-per-code operand format of the tcgen05
 // GEMM).
 #pragma once
@@ -52,7 +53,7 @@ struct RowSmem {
   uint32_t* outp;      // Kp / 8 words: the packed row
   uint8_t* sfs;        // Kp / 32 scale bytes (MXFP4)
   float* red;          // 32 floats
-  float* exch;         // n = 256 only: [MT * 8][n] floats
+  float* exch;         // n > 64 only: [MT * 8][n + 8] floats
 };
 
 // Where a row's results go.
@@ -83,7 +84,7 @@ __device__ __forceinline__ void rotate_row(const xq_hadamard_plan_t& pl, float g
   constexpr int NB = 1 << LOG2NB;  // columns per warp
   constexpr int NT8 = NB / 8;      // n-tiles per warp
   const int Kp = pl.Kp, p = pl.p, n = 1 << pl.log2n;
-  const int NC = n / NB;            // column chunks (1 or 2)
+  const int NC = n / NB;            // column chunks (1, 2 or 4)
   const int pitch = n + 8;          // bf16 elements per staged row (conflict-free ldmatrix)
   const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int mt = warp / NC, bc = warp - mt * NC;
@@ -138,22 +139,39 @@ __device__ __forceinline__ void rotate_row(const xq_hadamard_plan_t& pl, float g
           acc[j | s][e] = u - w;
         }
       }
-  if (NC == 2) {
-    // last butterfly (bit log2(NB) of b) between the two column chunks, through shared memory: first the rows g of
-    // every tile, then the rows g + 8 (half the buffer of doing both at once)
-    const float sgn = bc ? -1.f : 1.f;
+  if (NC > 1) {
+    // the butterflies over the top bits of b run between the column chunks (warps), through shared memory: every warp
+    // writes its chunk, reads the others and combines them level by level, exactly as the register levels do.  First
+    // the rows g of every tile, then the rows g + 8 (half the buffer of doing both at once).
+    const float s0 = (bc & 1) ? -1.f : 1.f, s1 = (bc & 2) ? -1.f : 1.f;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      float* mine = exch + ((size_t)(8 * mt + g) * n + bc * NB + 2 * t);
+      float* rowp = exch + (size_t)(8 * mt + g) * (n + 8) + 2 * t;  // pitch n + 8: the eight rows of a store fall into distinct banks
 #pragma unroll
-      for (int j = 0; j < NT8; ++j) *reinterpret_cast<float2*>(mine + 8 * j) = make_float2(acc[j][2 * h], acc[j][2 * h + 1]);
+      for (int j = 0; j < NT8; ++j) *reinterpret_cast<float2*>(rowp + bc * NB + 8 * j) = make_float2(acc[j][2 * h], acc[j][2 * h + 1]);
       sync();
-      const float* other = exch + ((size_t)(8 * mt + g) * n + (bc ^ 1) * NB + 2 * t);
+      if (NC == 2) {
+        const float* other = rowp + (bc ^ 1) * NB;
 #pragma unroll
-      for (int j = 0; j < NT8; ++j) {
-        const float2 ov = *reinterpret_cast<const float2*>(other + 8 * j);
-        acc[j][2 * h] = fmaf(sgn, acc[j][2 * h], ov.x);
-        acc[j][2 * h + 1] = fmaf(sgn, acc[j][2 * h + 1], ov.y);
+        for (int j = 0; j < NT8; ++j) {
+          const float2 ov = *reinterpret_cast<const float2*>(other + 8 * j);
+          acc[j][2 * h] = fmaf(s0, acc[j][2 * h], ov.x);
+          acc[j][2 * h + 1] = fmaf(s0, acc[j][2 * h + 1], ov.y);
+        }
+      } else {  // NC == 4: v[c] = x[c & ~1] + (-1)^(c & 1) x[c | 1], then y[c] = v[c & ~2] + (-1)^(c >> 1 & 1) v[c | 2]
+        const float* p1 = rowp + (bc ^ 1) * NB;
+        const float* p2 = rowp + (bc ^ 2) * NB;
+        const float* p3 = rowp + (bc ^ 3) * NB;
+#pragma unroll
+        for (int j = 0; j < NT8; ++j) {
+          const float2 o1 = *reinterpret_cast<const float2*>(p1 + 8 * j);
+          const float2 o2 = *reinterpret_cast<const float2*>(p2 + 8 * j);
+          const float2 o3 = *reinterpret_cast<const float2*>(p3 + 8 * j);
+          const float vx = fmaf(s0, acc[j][2 * h], o1.x), vy = fmaf(s0, acc[j][2 * h + 1], o1.y);  // level 1 of this chunk
+          const float wx = fmaf(s0, o2.x, o3.x), wy = fmaf(s0, o2.y, o3.y);                        // level 1 of chunk bc ^ 2
+          acc[j][2 * h] = fmaf(s1, vx, wx);
+          acc[j][2 * h + 1] = fmaf(s1, vy, wy);
+        }
       }
       if (h == 0) sync();  // the second half overwrites what the first half's readers read
     }
@@ -255,6 +273,11 @@ __device__ __forceinline__ void rotate_row(const xq_hadamard_plan_t& pl, float g
   sync();
 }
 
+// Column chunks (warps per tile of 16 output rows) of a row group: chunks of min(n, 64) columns.
+__host__ __device__ inline int row_chunks(const xq_hadamard_plan_t& pl) { return pl.log2n > 6 ? 1 << (pl.log2n - 6) : 1; }
+// log2 of the chunk length: the LOG2NB template argument of rotate_row for this plan.
+__host__ __device__ inline int row_log2nb(const xq_hadamard_plan_t& pl) { return pl.log2n > 6 ? 6 : pl.log2n; }
+
 // Shared memory of one row group in the order Xs | outp | red | Hs (image of H_p^T, [P16][P16 + 8] bf16) | exch.
 struct RowLayout {
   size_t xs, outp, red, hs, exch, total;
@@ -272,7 +295,7 @@ __host__ __device__ inline RowLayout row_layout(const xq_hadamard_plan_t& pl) {
   L.hs = off;
   off += ((size_t)P16 * (P16 + 8) * 2 + 15) / 16 * 16;
   L.exch = off;
-  if (n > 128) off += (size_t)(P16 / 2) * n * 4;
+  if (n > 64) off += (size_t)(P16 / 2) * (n + 8) * 4;
   L.total = off;
   return L;
 }
@@ -280,7 +303,7 @@ __host__ __device__ inline RowLayout row_layout(const xq_hadamard_plan_t& pl) {
 // True when the plan is one rotate_row takes (and the warp count of a row group fits 16 warps).
 __host__ __device__ inline bool plan_supported(const xq_hadamard_plan_t& pl) {
   const int n = 1 << pl.log2n, rows_a = (pl.K + n - 1) / n, MT = (pl.p + 15) / 16;
-  return pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 8 && pl.K % 8 == 0 && rows_a <= 64 && MT * (n > 128 ? 2 : 1) <= 16;
+  return pl.p > 1 && pl.log2n >= 5 && pl.log2n <= 8 && pl.K % 8 == 0 && rows_a <= 64 && MT * row_chunks(pl) <= 16;
 }
 
 }  // namespace xqrot

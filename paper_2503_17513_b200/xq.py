@@ -42,7 +42,7 @@ EXPORTS = [
     "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
     "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
     "xq_mx_expanded_linear_host", "xq_mx_gemm_staged", "xq_mx_rotate_quant_staged",
-    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads", "xq_gemm_kernel_info", "xq_selftest_i8_mma_rate", "xq_expanded_linear_host_enqueue",
+    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads", "xq_gemm_kernel_info", "xq_selftest_i8_mma_rate", "xq_expanded_linear_host_enqueue", "xq_expanded_linear_one_launch",
 ]
 
 
@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
         L.xq_rotate_quant_asym.argtypes = [vp, i32, i64, ctypes.POINTER(HadamardPlan), vp, vp, vp, vp, vp]
         L.xq_w4a4_gemm_asym.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_asym.argtypes = [vp, i32, i64, vp, vp, vp, sz, vp]
+        L.xq_expanded_linear_one_launch.argtypes = [vp, i32, i64, vp, i32, vp, vp, sz, vp]
         L.xq_expanded_linear_host.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host_asym.argtypes = [vp, i32, vp, vp, vp, sz, vp]
         L.xq_expanded_linear_host_enqueue.argtypes = [vp, i32, vp, vp, vp, sz, vp]
@@ -243,6 +244,13 @@ def xq_expanded_linear(X, w: Weights, out, ws, M=None, ldx=None, stream=None) ->
     ldx = X.stride(0) if ldx is None else ldx
     _check(lib().xq_expanded_linear(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, _dp(out), _dp(ws),
                                     ws.numel() * ws.element_size(), _stream(stream)), "xq_expanded_linear")
+
+
+def xq_expanded_linear_one_launch(X, w: Weights, out, ws, asym=False, M=None, ldx=None, stream=None) -> None:
+    M = X.shape[0] if M is None else M
+    ldx = X.stride(0) if ldx is None else ldx
+    _check(lib().xq_expanded_linear_one_launch(ctypes.c_void_p(X.data_ptr()), M, ldx, w.handle, int(bool(asym)), _dp(out), _dp(ws),
+                                               ws.numel() * ws.element_size(), _stream(stream)), "xq_expanded_linear_one_launch")
 
 
 def xq_rotate_quant_asym(X, plan: HadamardPlan, Xq, s_x, zp, Y_f32=None, M=None, ldx=None, stream=None) -> None:
