@@ -614,8 +614,18 @@ DecodePlan decode_plan(int M, const xq_weights* w, size_t rot_bytes = 0) {
   // between CTAs (no cluster barrier, no remote stores) if the whole token slice fits.
   const size_t weight_bytes = (size_t)n_blocks * 16 * (w->Kp / 2);
   const int c_first = (weight_bytes / (size_t)w->sms < 64 * 1024 && M * groups <= 1200) ? 1 : 2;  // and few tokens to expand
-  for (int C = c_first; C <= 4; C *= 2) {
-    if (groups < 4 * C) break;
+  // More than 8 tokens: every CTA reads its K slice of all tokens from L2, the same lines as every other cluster, and that
+  // read is what the kernel waits for before its first MMA; clusters of four cut it to a quarter (measured: 4-12 % of
+  // the step at 16 and 32 tokens).  The smaller cluster sizes follow as fall-backs.
+  const int order_many[3] = {4, 2, 1}, order_few[3] = {c_first, 2 * c_first, c_first == 1 ? 4 : 0};
+  for (int ci = 0; ci < 3; ++ci) {
+    const int C = M > 8 ? order_many[ci] : order_few[ci];
+    if (C == 0 || C > 4) break;
+    if (M > 8 && C == 1 && c_first != 1) break;
+    if (groups < 4 * C) {
+      if (M > 8) continue;
+      break;
+    }
     const int Lmax = (groups + C - 1) / C, Lmin = groups / C;
     const int chunks = (Lmax + 3) / 4, chunks_min = (Lmin + 3) / 4;
     const int pitch = chunks * 128 + 16;  // 16 (mod 128): conflict-free 128-bit fragment reads
