@@ -77,6 +77,24 @@ xq_status xq_hadamard_plan(int32_t K, int32_t Kp, xq_hadamard_plan_t* out);
 xq_status xq_prepare_weights(const void* W_bf16_host, int32_t N, int32_t K, int32_t Kp,
                              void* stream, xq_weights** out);
 
+/* Offline step with the weight quantizer of the paper's experiments (Sec. 4 "Quantization Details": GPTQ with
+ * act-order on per-channel symmetric 4-bit weights; Sec. 3.1 Remark 2 bounds its error under expansion).  The rows of
+ * W are expanded and rotated as in xq_prepare_weights; then, instead of rounding every value to the nearest grid
+ * point, the channels are visited in descending order of diag(H) and the error of every quantized column is fed into
+ * the columns still to come, so that tr((W~ - Q) H (W~ - Q)^T) is descended on.  H_host: HOST, double [Kp, Kp],
+ * row-major, symmetric: the Hessian X_hat^T X_hat of the layer's expanded, rotated calibration activations (rows of
+ * xq_rotate_quant's Y output).  damp times the mean of diag(H) is added to the diagonal first (0.01 is customary; the
+ * Hessian of expanded activations has rank <= K < Kp, so some damping is needed); a channel with H[c][c] = 0 gets
+ * zero codes.  Every row keeps the scale absmax / 7 of its rotated values; codes lie in [-8, 7].  fp64 on the device;
+ * allocates about 8 (Kp^2 + 3 N Kp) bytes of device memory for the duration of the call; synchronizes `stream`.
+ * Errors as xq_prepare_weights; INVALID_ARG also when H is not positive definite after damping.
+ * xq_gptq_codes is the quantizer alone, on rows that are already rotated (HOST double [N, Kp]): codes int8 [N, Kp] and
+ * scales float [N] to the HOST (what xq_weights_import takes). */
+xq_status xq_prepare_weights_gptq(const void* W_bf16_host, int32_t N, int32_t K, int32_t Kp, const double* H_host,
+                                  double damp, void* stream, xq_weights** out);
+xq_status xq_gptq_codes(const double* Wt_host, const double* H_host, int32_t N, int32_t Kp, double damp,
+                        int8_t* codes_host, float* s_w_host, void* stream);
+
 /* Build a weights object from already quantized values (HOST): codes int8 [N, Kp] row-major with
  * values in -8..7 (INVALID_ARG otherwise), s_w float [N].  Synchronizes `stream`. */
 xq_status xq_weights_import(const int8_t* codes_host, const float* s_w_host, int32_t N, int32_t K,

@@ -42,7 +42,7 @@ EXPORTS = [
     "xq_mx_prepare_weights", "xq_mx_weights_import", "xq_mx_weights_export", "xq_mx_weights_info", "xq_mx_weights_free",
     "xq_mx_workspace_bytes", "xq_mx_rotate_quant", "xq_mx_gemm", "xq_mx_expanded_linear",
     "xq_mx_expanded_linear_host", "xq_mx_gemm_staged", "xq_mx_rotate_quant_staged",
-    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads", "xq_gemm_kernel_info", "xq_selftest_i8_mma_rate", "xq_expanded_linear_host_enqueue", "xq_expanded_linear_one_launch",
+    "xq_mx_prepare_weights_heads", "xq_mx_weights_heads", "xq_gemm_kernel_info", "xq_selftest_i8_mma_rate", "xq_expanded_linear_host_enqueue", "xq_expanded_linear_one_launch", "xq_prepare_weights_gptq", "xq_gptq_codes",
 ]
 
 
@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.xq_hadamard_plan.argtypes = [i32, i32, ctypes.POINTER(HadamardPlan)]
         L.xq_prepare_weights.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
         L.xq_weights_import.argtypes = [vp, vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.xq_prepare_weights_gptq.argtypes = [vp, i32, i32, i32, vp, ctypes.c_double, vp, ctypes.POINTER(vp)]
+        L.xq_gptq_codes.argtypes = [vp, vp, i32, i32, ctypes.c_double, vp, vp, vp]
         L.xq_weights_export.argtypes = [vp, vp, vp]
         L.xq_weights_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
                                       ctypes.POINTER(HadamardPlan)]
@@ -175,6 +177,29 @@ def xq_prepare_weights(W_bf16_host: np.ndarray, Kp: int, stream=None) -> Weights
     h = ctypes.c_void_p()
     _check(lib().xq_prepare_weights(_hp(W), N, K, Kp, _stream(stream), ctypes.byref(h)), "xq_prepare_weights")
     return Weights(h.value)
+
+
+def xq_prepare_weights_gptq(W_bf16_host: np.ndarray, Kp: int, H_host: np.ndarray, damp: float = 0.01, stream=None) -> Weights:
+    """W: host uint16 bf16 bit patterns [N, K]; H: host float64 [Kp, Kp], the Hessian of the rotated calibration activations."""
+    W = np.ascontiguousarray(W_bf16_host, dtype=np.uint16)
+    H = np.ascontiguousarray(H_host, dtype=np.float64)
+    N, K = W.shape
+    assert H.shape == (Kp, Kp)
+    h = ctypes.c_void_p()
+    _check(lib().xq_prepare_weights_gptq(_hp(W), N, K, Kp, _hp(H), float(damp), _stream(stream), ctypes.byref(h)), "xq_prepare_weights_gptq")
+    return Weights(h.value)
+
+
+def xq_gptq_codes(Wt_host: np.ndarray, H_host: np.ndarray, damp: float = 0.01, stream=None):
+    """GPTQ with act-order on already rotated rows (host float64 [N, Kp]): returns (codes int8 [N, Kp], scales float32 [N])."""
+    Wt = np.ascontiguousarray(Wt_host, dtype=np.float64)
+    H = np.ascontiguousarray(H_host, dtype=np.float64)
+    N, Kp = Wt.shape
+    assert H.shape == (Kp, Kp)
+    codes = np.empty((N, Kp), dtype=np.int8)
+    s_w = np.empty((N,), dtype=np.float32)
+    _check(lib().xq_gptq_codes(_hp(Wt), _hp(H), N, Kp, float(damp), _hp(codes), _hp(s_w), _stream(stream)), "xq_gptq_codes")
+    return codes, s_w
 
 
 def xq_prepare_weights_heads(W_bf16_host: np.ndarray, heads: int, head_dim_p: int, stream=None) -> Weights:
