@@ -60,7 +60,8 @@ FALLBACK_BF16_TFLOPS = (1590.0, 1400.0)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (mean over the linears of a layer), from the
 # ncu captures summarised in profiles/ (file named per entry); a workload that was not captured reports null.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    ("1b-decode", 32): (6.57e6, "profiles/gemm_decode_1b_decode_m32.txt"),
+    ("1b-decode", 32): (6.58e6, "profiles/gemm_decode_1b_decode_m32.txt"),
+    ("8b-decode", 16): ((13.47 + 31.32 + 31.32 + 31.49) * 1e6 / 4, "profiles/gemm_decode_8b_decode_m16.txt"),
     ("8b-prefill", 4096): ((31.802368 + 4.061952 + 51.203840 + 64.903936 + 51.312128 + 65.464064 + 158.099968 + 22.970624) * 1e6 / 4,
                            "profiles/gemm_prefill_8b_prefill_m4096.txt"),
 }
