@@ -100,7 +100,7 @@ extern "C" xq_status xq_gemm_kernel_info(int32_t M, const xq_weights* w, int32_t
     const int c = xq_prefill_tile_choice(M, w, w->sms);
     *kind = 1;
     *tile_tokens = c == 0 ? 128 : 256;
-    *tile_channels = c == 2 ? 128 : 256;
+    *tile_channels = c == 2 ? 128 : (c == 3 ? 224 : 256);
   } else {
     *kind = 2;
     *tile_tokens = 1;

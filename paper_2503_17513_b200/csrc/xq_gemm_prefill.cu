@@ -68,6 +68,7 @@ struct PrefillParams {
   int32_t* acc_opt;
   int32_t* status;
   int M, N, KB;        // KB = K'' / 128 (k blocks of the padded weights)
+  int row_blocks;      // blocks of 16 channels in the padded weights
   int tiles_m, tiles_n;
 };
 
@@ -144,8 +145,12 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
       const int tn = tile / p.tiles_m;
-      // lane l < 16 fetches channel block l of the tile: 16 channels x 128 codes = 1 KiB contiguous
-      const unsigned char* wsrc = p.W + ((size_t)(tn * (BN / XQ_ROW_BLOCK) + (lane & 15)) * p.KB) * (4 * XQ_GROUP_BYTES);
+      // lane l < BN / 16 fetches channel block l of the tile: 16 channels x 128 codes = 1 KiB contiguous; the last tile of
+      // a 224-wide tiling may reach past the padded rows: those blocks are not fetched (their stage rows keep stale
+      // bytes, which only feed accumulator columns the epilogue never stores)
+      const int blk0 = tn * (BN / XQ_ROW_BLOCK);
+      const int nblk = min(BN / XQ_ROW_BLOCK, p.row_blocks - blk0);
+      const unsigned char* wsrc = p.W + ((size_t)(blk0 + (lane < nblk ? lane : 0)) * p.KB) * (4 * XQ_GROUP_BYTES);
       for (int kb = 0; kb < p.KB; ++kb, ++it) {
         const int s = it % kPkStages;
         if (it >= (uint32_t)kPkStages) {
@@ -153,9 +158,9 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
           if (!ok) break;
         }
         unsigned char* stage = pk + (size_t)s * kPkBBytes;
-        if (lane == 0) mbar_expect_tx(&pk_full[s], kPkBBytes);
+        if (lane == 0) mbar_expect_tx(&pk_full[s], (uint32_t)nblk * (4 * XQ_GROUP_BYTES));
         __syncwarp();
-        if (lane < BN / XQ_ROW_BLOCK) bulk_g2s(stage + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
+        if (lane < nblk) bulk_g2s(stage + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
       }
     }
   } else if (warp == 1) {
@@ -299,14 +304,18 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
         // 16 channel blocks of 1 KiB, piece 16t + r of a block = codes 32t..32t+31 of channel r
         const unsigned char* src = pk + (size_t)s * kPkBBytes;
         unsigned char* dstB = i8 + (size_t)u * kI8StageBytes + MH * kI8ABytes;
-        constexpr int kPieces = BN * 4 / (kUnpackWarps * 32);  // 16-byte pieces per thread
+        constexpr int kTotal = BN * 4;                                               // 16-byte pieces of the tile
+        constexpr int kPieces = (kTotal + kUnpackWarps * 32 - 1) / (kUnpackWarps * 32);  // per thread (the last may be missing)
         uint4 v[kPieces];
-#pragma unroll
-        for (int i = 0; i < kPieces; ++i) v[i] = *reinterpret_cast<const uint4*>(src + (size_t)(ut + i * kUnpackWarps * 32) * 16);
 #pragma unroll
         for (int i = 0; i < kPieces; ++i) {
           const int q = ut + i * kUnpackWarps * 32;
-          expand_store(v[i], dstB, ((q >> 6) << 4) + (q & 15), (q >> 4) & 3);
+          if (kTotal % (kUnpackWarps * 32) == 0 || q < kTotal) v[i] = *reinterpret_cast<const uint4*>(src + (size_t)q * 16);
+        }
+#pragma unroll
+        for (int i = 0; i < kPieces; ++i) {
+          const int q = ut + i * kUnpackWarps * 32;
+          if (kTotal % (kUnpackWarps * 32) == 0 || q < kTotal) expand_store(v[i], dstB, ((q >> 6) << 4) + (q & 15), (q >> 4) & 3);
         }
         fence_proxy_async_smem();
         __syncwarp();
@@ -461,13 +470,18 @@ cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, ui
 // Three tile shapes; a cost model picks one: waves of tiles over the multiprocessors times the cycles of a tile
 // (69 tensor-core cycles per 128 x 256 x 32 MMA; 128-token tiles expand every weight for half as many MMAs and run
 // at about 0.62 of that rate; an epilogue that is not hidden costs about 2000 cycles).
-// Returns 0 for 128 tokens x 256 channels, 1 for 256 x 256, 2 for 256 x 128.
+// A fourth shape, 256 tokens x 224 channels, costs 7/8 of the 256 x 256 tile and exists for the wave count: 14336 =
+// 64 x 224 channels in 256-token rows are 6.9 waves on 148 SMs instead of 6.05 (which runs as 7), 8192 channels
+// and 2048 tokens are exactly 2 waves.
+// Returns 0 for 128 tokens x 256 channels, 1 for 256 x 256, 2 for 256 x 128, 3 for 256 x 224.
 int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms) {
   const int KB = w->Kpp / XQ_K_BLOCK, tm1 = (M + BMH - 1) / BMH, tm2 = (M + 2 * BMH - 1) / (2 * BMH);
   auto waves = [&](int tiles) { return (double)((tiles + sms - 1) / sms); };
   const double t_1x256 = waves(tm1 * ((w->N + 255) / 256)) * (KB * 276.0 / 0.62);
   const double t_2x256 = waves(tm2 * ((w->N + 255) / 256)) * (KB * 552.0 + 2000.0);
   const double t_2x128 = waves(tm2 * ((w->N + 127) / 128)) * (KB * 276.0 / 0.80);  // N = 128 MMAs re-read the tokens twice as often
+  const double t_2x224 = waves(tm2 * ((w->N + 223) / 224)) * (KB * 483.0 + 1750.0);
+  if (t_2x224 < 0.97 * t_2x256 && t_2x224 < t_2x128 && t_2x224 < t_1x256) return 3;  // only for a clear gain
   if (t_2x128 <= t_2x256 && t_2x128 <= t_1x256) return 2;
   if (t_2x256 <= t_1x256) return 1;
   return 0;
@@ -497,9 +511,11 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int
   p.M = M;
   p.N = w->N;
   p.KB = w->Kpp / XQ_K_BLOCK;
+  p.row_blocks = w->Np / XQ_ROW_BLOCK;
   p.tiles_n = 0;
   p.tiles_m = 0;
   switch (xq_prefill_tile_choice(M, w, sms)) {
+    case 3: return launch_mh<2, 224>(mapA, p, sms, st);
     case 2: return launch_mh<2, 128>(mapA, p, sms, st);
     case 1: return launch_mh<2, 256>(mapA, p, sms, st);
     default: return launch_mh<1, 256>(mapA, p, sms, st);

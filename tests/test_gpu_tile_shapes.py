@@ -4,7 +4,7 @@ shape it ran on (asked from the library with xq_gemm_kernel_info, nothing is ass
 The quantized product Q(XR) Q(W~) of the paper's Sec. 3 is an integer sum, so given identical codes
 the int32 accumulators must equal the oracle's int64 sums exactly, whatever tile shape, tile count
 per CTA, K length or tail the launch has.  Cases here reach the three shapes the kernel can pick
-(128 tokens x 256 channels, 256 x 256, 256 x 128) at the layer sizes the benchmark times, and the
+(128 tokens x 256 channels, 256 x 256, 256 x 128, 256 x 224) at the layer sizes the benchmark times, and the
 extreme codes (-8 against -8 and against 7) at the longest K' of the paper's Table 1, where the
 16 x 16 factor carried by the nibble expansion makes the partial sums largest.
 """
@@ -47,10 +47,13 @@ def sample_rows(M, count, seed=13):
 # (M, N, K, Kp, tile the library must report, token rows compared: None = all)
 TILE_CASES = [
     (384, 9728, 250, 256, (128, 256), None),
-    (2048, 8192, 2048, 2176, (256, 256), None),       # gate / up of the 1B prefill workload
-    (512, 14336, 4096, 4352, (256, 256), None),       # gate / up of the 8B workload, all channels
+    (2048, 8192, 2048, 2176, (256, 224), None),       # gate / up of the 1B prefill workload: the last 224-wide tile is ragged
+    (2048, 4096, 2048, 2176, (256, 256), None),
+    (512, 14336, 4096, 4352, (256, 224), None),       # gate / up of the 8B workload, all channels (64 x 224)
     (2048, 2048, 8192, 8704, (256, 128), None),       # down of the 1B prefill workload
-    (4096, 14336, 4096, 4352, (256, 256), 64),        # the 8B prefill launches as the benchmark times them
+    (2048, 3072, 2048, 2176, (256, 224), None),       # qkv of the 1B prefill workload: tiles reach past the padded rows
+    (4096, 14336, 4096, 4352, (256, 224), 64),        # the 8B prefill launches as the benchmark times them
+    (4096, 6144, 4096, 4352, (256, 256), 64),
     (4096, 4096, 14336, 15360, (256, 256), 64),
     (8192, 4096, 4096, 4096, (256, 128), 64),         # the expansion sweep at its two ends
     (8192, 4096, 4096, 5120, (256, 256), 64),
@@ -83,7 +86,8 @@ def test_tile_shape_accumulators_bit_exact(xq, oracle, M, N, K, Kp, tile, nrows)
 
 ASYM_TILE_CASES = [
     (384, 9728, 250, 256, (128, 256), None),
-    (2048, 8192, 2048, 2176, (256, 256), 256),
+    (2048, 8192, 2048, 2176, (256, 224), 256),
+    (2048, 4096, 2048, 2176, (256, 256), 256),
     (2048, 2048, 8192, 8704, (256, 128), 256),
     (4096, 4096, 14336, 15360, (256, 256), 64),
 ]
@@ -123,6 +127,7 @@ EXTREME_CASES = [
     (1024, 9472, 14336, 18432, (256, 256)),
     (1024, 9472, 14336, 22016, (256, 256)),
     (384, 9728, 14336, 22016, (128, 256)),
+    (512, 14336, 14336, 22016, (256, 224)),
 ]
 
 
