@@ -36,7 +36,6 @@ using namespace xqptx;
 namespace {
 
 constexpr int BMH = 128;                                     // rows of one accumulator
-constexpr int kPkStages = 4;
 constexpr int kI8ABytes = BMH * 128;                         // expanded tokens: 16 KiB per 128 tokens
 constexpr int kUnpackWarps = 8;
 constexpr int kFirstEpiWarp = 4;
@@ -49,13 +48,16 @@ struct Cfg {
   static constexpr int kPkBBytes = BN * 64;    // packed weights of a K block
   static constexpr int kI8BBytes = BN * 128;   // expanded
   static constexpr int kI8StageBytes = MH * kI8ABytes + kI8BBytes;
-  static constexpr int kI8Stages = kI8StageBytes <= 48 * 1024 ? 3 : 2;
+  // stages: as many expanded ones as fit (a stage's hand-over chain -- commit, unpack wakes, expands, MMA wakes -- is
+  // longer than its MMAs, so two stages leave the tensor pipe waiting); 256 x 256 has room for two only
+  static constexpr int kI8Stages = kI8StageBytes <= 60 * 1024 ? 3 : 2;
+  static constexpr int kPkStages = (BN == 224) ? 3 : 4;
   static constexpr int kEpiWarps = 4 * MH;
   static constexpr int kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
   static constexpr int kThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;
   static constexpr int kAccBufs = MH * BN <= 256 ? 2 : 1;
   static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kI8Stages * kI8StageBytes + (size_t)kPkStages * kPkBBytes +
-                                       kEpiWarps * 2 * BN * sizeof(float) /*scales, code sums*/ + 256 /*barriers, flags*/;
+                                       kEpiWarps * 64 * sizeof(float) /*scales, code sums of 32 channels per warp*/ + 256 /*barriers, flags*/;
 };
 
 struct PrefillParams {
@@ -90,13 +92,14 @@ template <int MH, int BN>
 __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap mapA, const PrefillParams p) {
   using C = Cfg<MH, BN>;
   constexpr int kI8Stages = C::kI8Stages, kI8StageBytes = C::kI8StageBytes, kAccBufs = C::kAccBufs, kPkBBytes = C::kPkBBytes;
+  constexpr int kPkStages = C::kPkStages;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* base = smem_raw + (((raw + 1023u) & ~1023u) - raw);
   unsigned char* i8 = base;                                        // kI8Stages x [A (MH x 16 KiB) | B 32 KiB], 1024-aligned
   unsigned char* pk = i8 + (size_t)kI8Stages * kI8StageBytes;      // kPkStages x 16 KiB of packed weights
   float* sw_tile = reinterpret_cast<float*>(pk + (size_t)kPkStages * kPkBBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sw_tile + C::kEpiWarps * 2 * BN);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sw_tile + C::kEpiWarps * 64);
   uint64_t* pk_full = bars;
   uint64_t* pk_empty = pk_full + kPkStages;
   uint64_t* i8_full = pk_empty + kPkStages;
@@ -229,8 +232,10 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
     // ---------------- epilogue ------------------------------------------------------------------
     const int q = warp & 3;                        // tensor-memory lane quarter this warp may read
     const int eh = (warp - kFirstEpiWarp) >> 2;    // which 128-row half of the tile (MH = 2)
-    float* sw_mine = sw_tile + (warp - kFirstEpiWarp) * 2 * BN;  // a private copy per warp: no cross-warp barrier
-    int* ws_mine = reinterpret_cast<int*>(sw_mine + BN);         // code sums of the tile's channels (asymmetric tokens)
+    // the scales and code sums of the 32 channels being stored, a private copy per warp (no cross-warp barrier); the
+    // values of the next 32 travel in a register of each lane meanwhile
+    float* sw_mine = sw_tile + (warp - kFirstEpiWarp) * 64;
+    int* ws_mine = reinterpret_cast<int*>(sw_mine + 32);
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
@@ -238,12 +243,8 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
       const uint32_t buf = kAccBufs == 2 ? (tcount & 1u) : 0u;
       const uint32_t use = kAccBufs == 2 ? (tcount >> 1) : tcount;
       const int n0 = tn * BN;
-      __syncwarp();
-      for (int i = lane; i < BN; i += 32) {
-        sw_mine[i] = (n0 + i < p.N) ? p.sw[n0 + i] : 0.f;
-        ws_mine[i] = (p.zp && n0 + i < p.N) ? p.wsum[n0 + i] : 0;
-      }
-      __syncwarp();
+      float sw_next = (n0 + lane < p.N) ? p.sw[n0 + lane] : 0.f;
+      int ws_next = (p.zp && n0 + lane < p.N) ? p.wsum[n0 + lane] : 0;
       const int m = (tm * MH + eh) * BMH + q * 32 + lane;
       const float sxm = m < p.M ? p.sx[m] : 0.f;
       const int zpm = (p.zp && m < p.M) ? p.zp[m] : 0;
@@ -253,6 +254,15 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (buf * MH + (uint32_t)eh) * BN;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
+        __syncwarp();
+        sw_mine[lane] = sw_next;
+        ws_mine[lane] = ws_next;
+        __syncwarp();
+        if (c + 1 < BN / 32) {
+          const int nn = n0 + (c + 1) * 32 + lane;
+          sw_next = nn < p.N ? p.sw[nn] : 0.f;
+          ws_next = (p.zp && nn < p.N) ? p.wsum[nn] : 0;
+        }
         uint32_t v[32];
         tmem_ld_32x32(taddr + c * 32, v);
         tmem_ld_wait();
@@ -265,7 +275,7 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
               int a[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e)  // every product carries 16 x 16; sum (c - z) qw = sum c qw - z sum qw
-                a[e] = ((int)v[8 * g8 + e] >> 8) - zpm * ws_mine[c * 32 + 8 * g8 + e];
+                a[e] = ((int)v[8 * g8 + e] >> 8) - zpm * ws_mine[8 * g8 + e];
               if (p.acc_opt) {
                 *reinterpret_cast<int4*>(p.acc_opt + o + 8 * g8) = make_int4(a[0], a[1], a[2], a[3]);
                 *reinterpret_cast<int4*>(p.acc_opt + o + 8 * g8 + 4) = make_int4(a[4], a[5], a[6], a[7]);
@@ -273,8 +283,8 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
               uint32_t h[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const float f0 = (float)a[2 * e] * sxm * sw_mine[c * 32 + 8 * g8 + 2 * e];
-                const float f1 = (float)a[2 * e + 1] * sxm * sw_mine[c * 32 + 8 * g8 + 2 * e + 1];
+                const float f0 = (float)a[2 * e] * sxm * sw_mine[8 * g8 + 2 * e];
+                const float f1 = (float)a[2 * e + 1] * sxm * sw_mine[8 * g8 + 2 * e + 1];
                 const __nv_bfloat162 b2 = __halves2bfloat162(__float2bfloat16_rn(f0), __float2bfloat16_rn(f1));
                 h[e] = *reinterpret_cast<const uint32_t*>(&b2);
               }
