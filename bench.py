@@ -533,6 +533,9 @@ def main():
     ap.add_argument("--only", action="store_true", help="time the named workload alone (no per_workload object)")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gptq-report", action="store_true",
+                    help="instead of timing: GPTQ (act-order) against round-to-nearest on the down projection at the paper's "
+                         "Table 1 sizes of the 1B model, objective relative to the layer's energy per K' (one JSON line)")
     ap.add_argument("--one-launch", action="store_true",
                     help="M <= 32: run each linear as xq_expanded_linear_one_launch (the online step inside the product kernel)")
     ap.add_argument("--fmt", default="int4", choices=["int4", "mxfp4"],
@@ -567,6 +570,11 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     if args.fmt == "mxfp4":
         assert args.act == "sym", "--fmt mxfp4 has its own quantizer: --act does not apply"
+
+    if args.gptq_report:
+        if rank == 0:
+            gptq_report()
+        return
 
     b = Bench(args, rank, local_rank, world, dist)
     head = b.run(args.workload, M, args.steps, args.warmup, headline=True)
@@ -603,6 +611,53 @@ def main():
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def gptq_report(rows=256, tokens=2048):
+    """Sec. 3.1 Remark 2 on synthetic data: the down projection of the 1B shape (K = 8192) at the expansion sizes of the
+    paper's Table 1, `rows` output channels, Hessian from `tokens` synthetic calibration tokens.  Rotated activations and
+    weights come from the library's rotate kernel (its fp32 dump), the Hessian and the objectives are plain fp64 matrix
+    products (torch: bookkeeping of the report, not the path), the codes from xq_gptq_codes and from round-to-nearest."""
+    import torch
+
+    from paper_2503_17513_b200 import xq
+
+    K = 8192
+    x = synth.activations(tokens, K, seed=7, tag="gptq-cal", heavy_tail=True)
+    wb = synth.weights(rows, K, seed=7, tag="gptq-down")
+    X = torch.from_numpy(x.view(np.int16)).cuda()
+    Wb = torch.from_numpy(wb.view(np.int16)).cuda()
+    out = {}
+    for Kp in (8192, 8960, 9728, 10240, 12288):
+        pl = xq.xq_hadamard_plan(K, Kp)
+
+        def rotated(T, n):
+            Xq = torch.empty((n, Kp // 2), dtype=torch.uint8, device="cuda")
+            sx = torch.empty((n,), dtype=torch.float32, device="cuda")
+            Y = torch.empty((n, Kp), dtype=torch.float32, device="cuda")
+            xq.xq_rotate_quant(T, pl, Xq, sx, Y)
+            return Y.double()
+
+        Y, Wt = rotated(X, tokens), rotated(Wb, rows)
+        H = Y.T @ Y
+        t0 = time.perf_counter()
+        codes, s_w = xq.xq_gptq_codes(Wt.cpu().numpy(), H.cpu().numpy(), damp=0.01)
+        t_gptq = time.perf_counter() - t0
+        s_rtn = torch.clamp(Wt.abs().amax(dim=1) / 7.0, min=0).float().double()
+        s_rtn[s_rtn == 0] = 1.0
+        q_rtn = torch.clamp(torch.round(Wt / s_rtn[:, None]), -8, 7)
+
+        def objective(Q, s):
+            D = Wt - s[:, None] * Q
+            return float(((D @ H) * D).sum())
+
+        energy = float(((Wt @ H) * Wt).sum())
+        o_g = objective(torch.from_numpy(codes.astype(np.float64)).cuda(), torch.from_numpy(s_w.astype(np.float64)).cuda())
+        o_r = objective(q_rtn, s_rtn)
+        out[str(Kp)] = {"gptq_rel_objective": o_g / energy, "rtn_rel_objective": o_r / energy, "sqrt_K_over_Kp": float(np.sqrt(K / Kp)),
+                        "gptq_seconds": t_gptq}
+    print(json.dumps({"report": "gptq objective vs K' (Remark 2), 1B down projection, synthetic Hessian", "K": K, "rows": rows,
+                      "calibration_tokens": tokens, "damp": 0.01, "per_Kp": out}))
 
 
 def cpu_baseline_leg(args, table, layers, M, heavy):

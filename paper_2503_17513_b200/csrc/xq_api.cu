@@ -283,11 +283,13 @@ xq_status prepare_impl(const void* W_host, int32_t N, int32_t heads, int32_t K, 
 extern "C" {
 
 xq_status xq_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t Kp, void* stream, xq_weights** out) {
+  XQ_RANGE();
   return prepare_impl(W_host, N, 1, K, Kp, stream, out);
 }
 
 xq_status xq_prepare_weights_heads(const void* W_host, int32_t N, int32_t heads, int32_t head_dim, int32_t head_dim_p,
                                    void* stream, xq_weights** out) {
+  XQ_RANGE();
   if (heads < 2) return XQ_ERR_INVALID_ARG;
   return prepare_impl(W_host, N, heads, head_dim, head_dim_p, stream, out);
 }
@@ -296,6 +298,7 @@ int32_t xq_weights_heads(const xq_weights* w) { return w ? w->heads : 0; }
 
 xq_status xq_weights_import(const int8_t* codes, const float* s_w, int32_t N, int32_t K, int32_t Kp,
                             void* stream, xq_weights** out) {
+  XQ_RANGE();
   if (!codes || !s_w || !out || N < 1 || K < 1 || Kp < K) return XQ_ERR_INVALID_ARG;
   const size_t count = (size_t)N * Kp;
   for (size_t i = 0; i < count; ++i)
@@ -328,6 +331,7 @@ xq_status xq_weights_import(const int8_t* codes, const float* s_w, int32_t N, in
 }
 
 xq_status xq_weights_export(const xq_weights* w, int8_t* codes, float* s_w) {
+  XQ_RANGE();
   if (!w || !codes || !s_w || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   const size_t count = (size_t)w->N * w->Kp;
   DevBuf dCodes, dCanon;
@@ -454,42 +458,50 @@ extern "C" {
 
 xq_status xq_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq,
                           float* s_x, float* Yopt, void* stream) {
+  XQ_RANGE();
   return rotate_quant_impl(X, M, ldx, plan, Xq, s_x, nullptr, false, Yopt, stream);
 }
 
 xq_status xq_rotate_quant_asym(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* Xq,
                                float* s_x, int32_t* zp, float* Yopt, void* stream) {
+  XQ_RANGE();
   return rotate_quant_impl(X, M, ldx, plan, Xq, s_x, zp, true, Yopt, stream);
 }
 
 xq_status xq_rotate_quant_heads(const void* X, int32_t M, int64_t ldx, int32_t heads, const xq_hadamard_plan_t* head_plan,
                                 uint8_t* Xq, float* s_x, int32_t* zp_opt, float* Yopt, void* stream) {
+  XQ_RANGE();
   if (heads < 2) return XQ_ERR_INVALID_ARG;
   return rotate_quant_impl(X, M, ldx, head_plan, Xq, s_x, zp_opt, zp_opt != nullptr, Yopt, stream, heads);
 }
 
 xq_status xq_w4a4_gemm(const uint8_t* Xq, const float* s_x, int32_t M, const xq_weights* w, void* out,
                        int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return gemm_impl(Xq, s_x, nullptr, false, M, w, out, acc_opt, ws, ws_bytes, stream);
 }
 
 xq_status xq_w4a4_gemm_asym(const uint8_t* Xq, const float* s_x, const int32_t* zp, int32_t M, const xq_weights* w,
                             void* out, int32_t* acc_opt, void* ws, size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return gemm_impl(Xq, s_x, zp, true, M, w, out, acc_opt, ws, ws_bytes, stream);
 }
 
 xq_status xq_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out, void* ws,
                              size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return linear_impl(X, M, ldx, w, false, out, ws, ws_bytes, stream);
 }
 
 xq_status xq_expanded_linear_asym(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out, void* ws,
                                   size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return linear_impl(X, M, ldx, w, true, out, ws, ws_bytes, stream);
 }
 
 xq_status xq_expanded_linear_one_launch(const void* X, int32_t M, int64_t ldx, const xq_weights* w, int32_t asym, void* out,
                                         void* ws, size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return linear_impl(X, M, ldx, w, asym != 0, out, ws, ws_bytes, stream, true);
 }
 
@@ -531,16 +543,19 @@ extern "C" {
 
 xq_status xq_expanded_linear_host(const void* X_host, int32_t M, const xq_weights* w, void* out_host, void* ws,
                                   size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return linear_host_impl(X_host, M, w, false, out_host, ws, ws_bytes, stream);
 }
 
 xq_status xq_expanded_linear_host_asym(const void* X_host, int32_t M, const xq_weights* w, void* out_host, void* ws,
                                        size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return linear_host_impl(X_host, M, w, true, out_host, ws, ws_bytes, stream);
 }
 
 xq_status xq_expanded_linear_host_enqueue(const void* X_host, int32_t M, const xq_weights* w, void* out_host, void* ws,
                                           size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   return linear_host_impl(X_host, M, w, false, out_host, ws, ws_bytes, stream, false);
 }
 

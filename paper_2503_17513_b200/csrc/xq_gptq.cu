@@ -321,6 +321,7 @@ extern "C" {
 
 xq_status xq_gptq_codes(const double* Wt_host, const double* H_host, int32_t N, int32_t Kp, double damp, int8_t* codes_host, float* s_w_host,
                         void* stream) {
+  XQ_RANGE();
   if (!Wt_host || !H_host || !codes_host || !s_w_host || N < 1 || Kp < 1 || !(damp >= 0.0)) return XQ_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   DevMem mW, mH, mC, mS;
@@ -348,6 +349,7 @@ xq_status xq_gptq_codes(const double* Wt_host, const double* H_host, int32_t N, 
 
 xq_status xq_prepare_weights_gptq(const void* W_host, int32_t N, int32_t K, int32_t Kp, const double* H_host, double damp, void* stream,
                                   xq_weights** out) {
+  XQ_RANGE();
   if (!W_host || !H_host || !out || N < 1 || K < 1 || Kp < K || !(damp >= 0.0)) return XQ_ERR_INVALID_ARG;
   xq_hadamard_plan_t pl;
   xq_status s = xq_hadamard_plan(K, Kp, &pl);

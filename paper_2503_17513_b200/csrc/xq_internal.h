@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include "xq.h"
@@ -42,6 +43,16 @@ struct xq_weights {
   int device;
   int sms;             // multiprocessors of that device
 };
+
+// NVTX range around one entry point of the library (shows as a named span on the host timeline of a profiler; costs a
+// pointer test when none is attached).
+struct XqRange {
+  explicit XqRange(const char* name) { nvtxRangePushA(name); }
+  ~XqRange() { nvtxRangePop(); }
+  XqRange(const XqRange&) = delete;
+  XqRange& operator=(const XqRange&) = delete;
+};
+#define XQ_RANGE() XqRange xq_range_(__func__)
 
 // True when `device` (the one a weights object lives on) is the current device: the kernels dereference the
 // object's pointers, so a call made with another device current is refused on the host.

@@ -854,11 +854,13 @@ xq_status mx_prepare_impl(const void* W_host, int32_t N, int32_t heads, int32_t 
 extern "C" {
 
 xq_status xq_mx_prepare_weights(const void* W_host, int32_t N, int32_t K, int32_t Kp, void* stream, xq_mx_weights** out) {
+  XQ_RANGE();
   return mx_prepare_impl(W_host, N, 1, K, Kp, stream, out);
 }
 
 xq_status xq_mx_prepare_weights_heads(const void* W_host, int32_t N, int32_t heads, int32_t head_dim, int32_t head_dim_p, void* stream,
                                       xq_mx_weights** out) {
+  XQ_RANGE();
   if (heads < 2) return XQ_ERR_INVALID_ARG;
   return mx_prepare_impl(W_host, N, heads, head_dim, head_dim_p, stream, out);
 }
@@ -867,6 +869,7 @@ int32_t xq_mx_weights_heads(const xq_mx_weights* w) { return w ? w->heads : 0; }
 
 xq_status xq_mx_weights_import(const uint8_t* codes_packed, const uint8_t* scales, int32_t N, int32_t K, int32_t Kp, void* stream,
                                xq_mx_weights** out) {
+  XQ_RANGE();
   if (!codes_packed || !scales || !out) return XQ_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   xq_mx_weights* w = nullptr;
@@ -904,6 +907,7 @@ xq_status xq_mx_weights_import(const uint8_t* codes_packed, const uint8_t* scale
 }
 
 xq_status xq_mx_weights_export(const xq_mx_weights* w, uint8_t* codes, uint8_t* scales) {
+  XQ_RANGE();
   if (!w || !codes || !scales || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
   DevBuf dC, dS;
   const size_t nc = (size_t)w->N * w->Kp, ns = (size_t)w->N * (w->Kp / 32);
@@ -929,6 +933,7 @@ size_t xq_mx_workspace_bytes(int32_t M_max, const xq_mx_weights* w) {
 
 xq_status xq_mx_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_hadamard_plan_t* plan, uint8_t* codes, uint8_t* scales,
                              float* Y, void* stream) {
+  XQ_RANGE();
   if (!plan || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X || !codes || !scales || !Y) return XQ_ERR_INVALID_ARG;
@@ -956,6 +961,7 @@ xq_status xq_mx_rotate_quant(const void* X, int32_t M, int64_t ldx, const xq_had
 
 xq_status xq_mx_gemm(const uint8_t* codes, const uint8_t* scales, int32_t M, const xq_mx_weights* w, void* out, void* ws, size_t ws_bytes,
                      void* stream) {
+  XQ_RANGE();
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!codes || !scales || !out || !aligned16(codes) || !aligned16(out) || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
@@ -976,6 +982,7 @@ xq_status xq_mx_gemm(const uint8_t* codes, const uint8_t* scales, int32_t M, con
 }
 
 xq_status xq_mx_gemm_staged(int32_t M, const xq_mx_weights* w, void* out, void* ws, size_t ws_bytes, void* stream) {
+  XQ_RANGE();
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!out || !aligned16(out) || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
@@ -993,6 +1000,7 @@ xq_status xq_mx_gemm_staged(int32_t M, const xq_mx_weights* w, void* out, void* 
 
 xq_status xq_mx_rotate_quant_staged(const void* X, int32_t M, int64_t ldx, const xq_mx_weights* w, void* ws, size_t ws_bytes,
                                     void* stream) {
+  XQ_RANGE();
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
@@ -1026,6 +1034,7 @@ xq_status xq_mx_rotate_quant_staged(const void* X, int32_t M, int64_t ldx, const
 
 xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_mx_weights* w, void* out, void* ws, size_t ws_bytes,
                                 void* stream) {
+  XQ_RANGE();
   if (M > 0 && (!out || !aligned16(out))) return XQ_ERR_INVALID_ARG;
   const xq_status s = xq_mx_rotate_quant_staged(X, M, ldx, w, ws, ws_bytes, stream);
   if (s != XQ_OK || M == 0) return s;
@@ -1034,6 +1043,7 @@ xq_status xq_mx_expanded_linear(const void* X, int32_t M, int64_t ldx, const xq_
 
 xq_status xq_mx_expanded_linear_host(const void* X_host, int32_t M, const xq_mx_weights* w, void* out_host, void* ws, size_t ws_bytes,
                                      void* stream) {
+  XQ_RANGE();
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X_host || !out_host || w->K % 8 != 0 || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;

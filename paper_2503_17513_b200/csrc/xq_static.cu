@@ -44,6 +44,7 @@ xq_status scratch_address(unsigned char** out) {
 
 extern "C" xq_status xq_expanded_linear_static(const void* X, int32_t M, int64_t ldx, const xq_weights* w, void* out,
                                                void* stream) {
+  XQ_RANGE();
   if (!w || M < 0) return XQ_ERR_INVALID_ARG;
   if (M == 0) return XQ_OK;
   if (!X || !out || !xq_on_device(w->device)) return XQ_ERR_INVALID_ARG;
