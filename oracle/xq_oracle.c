@@ -35,7 +35,7 @@
  * non-power-of-two factor, Sylvester for the power of two.                                   */
 
 typedef struct {
-  int32_t K, Kp, p, log2n, paley_kind, q; /* paley_kind: 0 none (p == 1), 1 Paley-I, 2 Paley-II */
+  int32_t K, Kp, p, log2n, paley_kind, q; /* paley_kind: 0 none (p == 1), 1 Paley-I, 2 Paley-II, 3 Paley-I over GF(7^3) */
 } xqo_plan_t;
 
 static int is_prime(int v) {
@@ -61,8 +61,43 @@ static int legendre(int a, int q) {
   return r == 1 ? 1 : -1;
 }
 
+/* The field with 343 = 7^3 elements, for the one prime-power order the paper's sizes need (Table 1: 22016 = 344 * 64,
+ * and 344 - 1 = 7^3 = 3 mod 4, so Paley's first construction applies over GF(7^3)).  Elements are the polynomials
+ * a0 + a1 x + a2 x^2 over GF(7) modulo x^3 - 5 (irreducible: 5 is not a cube mod 7, the cubes being 0, 1, 6), numbered
+ * a0 + 7 a1 + 49 a2. */
+static int gf343_sub(int a, int b) {
+  int r = 0, w = 1;
+  for (int k = 0; k < 3; ++k, w *= 7) {
+    int d = (a / w) % 7 - (b / w) % 7;
+    if (d < 0) d += 7;
+    r += d * w;
+  }
+  return r;
+}
+static int gf343_mul(int a, int b) {
+  int x[3] = {a % 7, (a / 7) % 7, a / 49}, y[3] = {b % 7, (b / 7) % 7, b / 49}, c[5] = {0, 0, 0, 0, 0};
+  for (int i = 0; i < 3; ++i)
+    for (int j = 0; j < 3; ++j) c[i + j] += x[i] * y[j];
+  /* x^3 = 5, x^4 = 5 x */
+  c[0] += 5 * c[3];
+  c[1] += 5 * c[4];
+  return c[0] % 7 + 7 * (c[1] % 7) + 49 * (c[2] % 7);
+}
+/* Quadratic character of GF(343): 0 for 0, +1 for a non-zero square, -1 otherwise, by Euler's criterion
+ * a^((343-1)/2). */
+static int gf343_chi(int a) {
+  if (a == 0) return 0;
+  int r = 1, b = a, e = 171;
+  while (e) {
+    if (e & 1) r = gf343_mul(r, b);
+    b = gf343_mul(b, b);
+    e >>= 1;
+  }
+  return r == 1 ? 1 : -1;
+}
+
 /* Smallest p = odd(Kp) * 2^j, j >= 2, for which a Paley matrix of order p exists over a prime
- * field; p = 1 when Kp is a power of two.  Returns 0 on success, 1 on bad arguments, 2 when no
+ * field or over GF(7^3); p = 1 when Kp is a power of two.  Returns 0 on success, 1 on bad arguments, 2 when no
  * such order divides Kp. */
 int xqo_plan(int32_t K, int32_t Kp, xqo_plan_t *out) {
   if (!out || K < 1 || Kp < K) return 1;
@@ -90,6 +125,10 @@ int xqo_plan(int32_t K, int32_t Kp, xqo_plan_t *out) {
       out->p = p; out->log2n = e - j; out->paley_kind = 2; out->q = p / 2 - 1;
       return 0;
     }
+    if (p - 1 == 343) {
+      out->p = p; out->log2n = e - j; out->paley_kind = 3; out->q = 343;
+      return 0;
+    }
   }
   return 2;
 }
@@ -105,6 +144,14 @@ static int hp_entry(const xqo_plan_t *pl, int r, int c) {
     if (c == 0) return -1;
     int i = r - 1, j = c - 1;
     return i == j ? 1 : legendre(i - j, q);
+  }
+  if (pl->paley_kind == 3) {
+    /* the same construction over GF(7^3): rows and columns 1..343 stand for the field elements in their numbering,
+     * Q[i][j] = chi(e_i - e_j) */
+    if (r == 0) return 1;
+    if (c == 0) return -1;
+    int i = r - 1, j = c - 1;
+    return i == j ? 1 : gf343_chi(gf343_sub(i, j));
   }
   /* Paley-II, q = 1 mod 4: symmetric S of order q + 1 with zero diagonal (S[0][j] = S[j][0] = 1,
    * core Q); every entry of S becomes a 2 x 2 block:  s * [[1,1],[1,-1]]  off the diagonal,

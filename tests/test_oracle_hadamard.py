@@ -14,7 +14,7 @@ from paper_2503_17513_b200 import synth
 # (K, Kp): every order-p factor used by the workloads (68, 60, 36, 20, 1) on a small Sylvester
 # factor, plus further Paley orders (12, 28, 76, 140) from the paper's own Table 1 sizes.
 SMALL = [(100, 136), (60, 68), (200, 240), (130, 144), (70, 80), (64, 64), (40, 48), (20, 24),
-         (50, 56), (140, 152), (250, 280), (1, 2), (3, 4)]
+         (50, 56), (140, 152), (250, 280), (1, 2), (3, 4), (300, 344), (600, 688)]  # 344 = 7^3 + 1: Paley over GF(7^3)
 
 
 @pytest.mark.parametrize("K,Kp", SMALL)
@@ -59,16 +59,39 @@ def test_kronecker_convention_outer_factor_is_order_p(oracle, K, Kp):
 def test_paley_structure(oracle):
     """Paley-I (q = 3 mod 4): H - I is skew-symmetric with a +1 first row; Paley-II
     (q = 1 mod 4): H is symmetric.  Both are textbook properties of the two constructions."""
-    for Kp, kind, q in [(68, 1, 67), (60, 1, 59), (20, 1, 19), (12, 1, 11), (36, 2, 17), (76, 2, 37)]:
+    for Kp, kind, q in [(68, 1, 67), (60, 1, 59), (20, 1, 19), (12, 1, 11), (36, 2, 17), (76, 2, 37), (344, 3, 343)]:
         pl = oracle.plan(Kp, Kp)
         assert (pl.p, pl.paley_kind, pl.q, pl.log2n) == (Kp, kind, q, 0)
         H = oracle.hadamard_dense(pl).astype(np.int64)
-        if kind == 1:
+        if kind in (1, 3):
             S = H - np.eye(Kp, dtype=np.int64)
             assert np.array_equal(S, -S.T)
             assert np.all(H[0] == 1)
         else:
             assert np.array_equal(H, H.T)
+
+
+def test_gf343_character_is_a_character_with_as_many_squares_as_non_squares(oracle):
+    """The order-344 factor rests on the quadratic character of GF(7^3).  Read off the matrix (row i + 1, column 1 is
+    chi(e_i - e_0) = chi(e_i)): it is +1 on exactly (343 - 1) / 2 elements, and it is what squaring in an independent
+    model of the field says -- polynomials over GF(7) modulo x^3 - 5, multiplied with numpy's polynomial routines."""
+    pl = oracle.plan(344, 344)
+    H = oracle.hadamard_dense(pl).astype(np.int64)
+    chi = H[1:, 1].copy()
+    chi[0] = 0  # the diagonal entry is the +1 of the identity, not a character value
+    assert np.count_nonzero(chi == 1) == 171 and np.count_nonzero(chi == -1) == 171
+
+    def square(idx):
+        a = np.array([idx % 7, (idx // 7) % 7, idx // 49])
+        prod = np.polymul(a[::-1], a[::-1])[::-1]  # coefficients, lowest degree first
+        prod = np.concatenate([prod, np.zeros(5 - len(prod), dtype=prod.dtype)])
+        c = [prod[0] + 5 * prod[3], prod[1] + 5 * prod[4], prod[2]]  # x^3 = 5
+        return int(c[0] % 7 + 7 * (c[1] % 7) + 49 * (c[2] % 7))
+
+    squares = {square(i) for i in range(1, 343)}
+    assert len(squares) == 171
+    for i in range(1, 343):
+        assert chi[i] == (1 if i in squares else -1)
 
 
 def test_plan_factors_the_workload_and_paper_sizes(oracle):
@@ -80,14 +103,14 @@ def test_plan_factors_the_workload_and_paper_sizes(oracle):
     }.items():
         pl = oracle.plan(K, Kp)
         assert (pl.p, pl.log2n, pl.paley_kind, pl.q) == want
-    # Table 1's expanded down-projection sizes are all Hadamard orders that factor over a
-    # prime-field Paley matrix (22016 only through the large order 5504 = 5503 + 1).
+    # Table 1's expanded down-projection sizes are all Hadamard orders that factor over a Paley matrix: over a prime
+    # field, except 22016 = 344 x 64, whose order-344 factor is Paley's construction over GF(7^3).
     for K, Kp in [(8192, 8960), (8192, 9728), (8192, 10240), (8192, 12288), (14336, 15360),
                   (14336, 18432), (14336, 19968)]:
         pl = oracle.plan(K, Kp)
         assert pl.p * (1 << pl.log2n) == Kp and pl.paley_kind in (1, 2)
     pl = oracle.plan(14336, 22016)
-    assert (pl.p, pl.log2n, pl.paley_kind, pl.q) == (5504, 2, 1, 5503)
+    assert (pl.p, pl.log2n, pl.paley_kind, pl.q) == (344, 6, 3, 343)
     g = np.random.default_rng(0)
     rows = g.choice(22016, size=6, replace=False)
     R = np.array([[oracle.hadamard_entry(pl, int(r), c) for c in range(22016)] for r in rows], dtype=np.int64)
