@@ -51,7 +51,9 @@ typedef enum {
 /* Hadamard plan: Kp = p * 2^log2n and H = H_p (x) S_{2^log2n} (Kronecker product, the order-p
  * factor outermost: channel c = a * 2^log2n + b).  S is the Sylvester matrix
  * S[b][b'] = (-1)^popcount(b & b'); H_p is a Paley matrix over the prime field GF(q):
- * paley_kind 1 (q = p - 1 = 3 mod 4) or 2 (q = p/2 - 1 = 1 mod 4); paley_kind 0 means p = 1.
+ * paley_kind 1 (q = p - 1 = 3 mod 4) or 2 (q = p/2 - 1 = 1 mod 4); paley_kind 0 means p = 1;
+ * paley_kind 3 is the first construction over the field of q = 7^3 = 343 elements (p = 344: the
+ * factor that the paper's Table 1 size 22016 = 344 * 64 needs).
  * The paper asks only for "an expanded M x M Hadamard matrix" (Sec. 3); this family is the
  * library's choice of one. */
 typedef struct {

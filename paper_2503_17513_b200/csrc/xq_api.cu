@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "xq_internal.h"
 
@@ -33,8 +34,33 @@ int host_chi(int a, int q) {
 // Entry (a, a2) of the order-p Paley factor (the construction the device kernels use: Paley-I has a
 // first row of +1, a first column of -1 below it and the core chi(i - j) + identity; Paley-II
 // expands the symmetric conference matrix of order q + 1 into 2 x 2 blocks).
+// Quadratic character of the field of 7^3 elements (polynomials over GF(7) modulo x^3 - 5, numbered a0 + 7 a1 + 49 a2):
+// the non-zero squares are collected once.
+int host_chi343(int d) {
+  static const std::vector<int8_t> table = [] {
+    std::vector<int8_t> t(343, -1);
+    t[0] = 0;
+    for (int a = 1; a < 343; ++a) {
+      const int a0 = a % 7, a1 = (a / 7) % 7, a2 = a / 49;
+      const int c0 = a0 * a0 + 10 * a1 * a2, c1 = 2 * a0 * a1 + 5 * a2 * a2, c2 = 2 * a0 * a2 + a1 * a1;
+      t[c0 % 7 + 7 * (c1 % 7) + 49 * (c2 % 7)] = 1;
+    }
+    return t;
+  }();
+  return table[d];
+}
+
 int host_paley_sign(const xq_hadamard_plan_t& pl, int a, int a2) {
   const int q = pl.q;
+  if (pl.paley_kind == 3) {  // Paley-I over GF(7^3)
+    if (a == 0) return 1;
+    if (a2 == 0) return -1;
+    if (a == a2) return 1;
+    const int i = a - 1, j = a2 - 1;
+    int d = 0, w = 1;
+    for (int k = 0; k < 3; ++k, w *= 7) d += (((i / w) % 7 - (j / w) % 7 + 7) % 7) * w;
+    return host_chi343(d);
+  }
   if (pl.paley_kind == 1) {
     if (a == 0) return 1;
     if (a2 == 0) return -1;
@@ -209,6 +235,9 @@ xq_status xq_hadamard_plan(int32_t K, int32_t Kp, xq_hadamard_plan_t* out) {
         found = true;
       } else if (prime(q2) && q2 % 4 == 1) {
         pl.p = (int)p; pl.log2n = twos - j; pl.paley_kind = 2; pl.q = q2;
+        found = true;
+      } else if (q1 == 343) {  // 7^3 = 3 mod 4: Paley-I over the field of 343 elements
+        pl.p = (int)p; pl.log2n = twos - j; pl.paley_kind = 3; pl.q = 343;
         found = true;
       }
     }

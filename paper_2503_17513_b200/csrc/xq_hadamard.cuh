@@ -14,7 +14,28 @@ namespace xqhad {
 // Paley-II: symmetric S of order q + 1 (zero diagonal, border +1, core chi(i - j)); each entry s
 //           becomes s * [[1, 1], [1, -1]], each diagonal zero becomes [[1, -1], [-1, -1]].
 // ---------------------------------------------------------------------------------------------
+// kind 3: Paley-I over the field of 7^3 = 343 elements (order 344), elements numbered a0 + 7 a1 + 49 a2 for the
+// polynomial a0 + a1 x + a2 x^2 over GF(7) modulo x^3 - 5; chi2 then holds chi(element d) at index d, d < 343.
+__device__ __forceinline__ int gf343_sub(int a, int b) {
+  int d0 = a % 7 - b % 7, d1 = (a / 7) % 7 - (b / 7) % 7, d2 = a / 49 - b / 49;
+  d0 += d0 < 0 ? 7 : 0;
+  d1 += d1 < 0 ? 7 : 0;
+  d2 += d2 < 0 ? 7 : 0;
+  return d0 + 7 * d1 + 49 * d2;
+}
+__device__ __forceinline__ int gf343_square(int a) {
+  const int a0 = a % 7, a1 = (a / 7) % 7, a2 = a / 49;
+  // (a0 + a1 x + a2 x^2)^2 with x^3 = 5, x^4 = 5 x
+  const int c0 = a0 * a0 + 10 * a1 * a2, c1 = 2 * a0 * a1 + 5 * a2 * a2, c2 = 2 * a0 * a2 + a1 * a1;
+  return c0 % 7 + 7 * (c1 % 7) + 49 * (c2 % 7);
+}
+
 __device__ __forceinline__ int paley_sign(int kind, int q, const int8_t* chi2, int a, int a2) {
+  if (kind == 3) {
+    if (a == 0) return 1;
+    if (a2 == 0) return -1;
+    return a == a2 ? 1 : chi2[gf343_sub(a - 1, a2 - 1)];
+  }
   if (kind == 1) {
     if (a == 0) return 1;
     if (a2 == 0) return -1;
@@ -27,10 +48,17 @@ __device__ __forceinline__ int paley_sign(int kind, int q, const int8_t* chi2, i
   return (u & v) ? -s : s;
 }
 
-// Fill chi2 (2q + 1 entries) cooperatively; `sq` is q scratch bytes.
-__device__ __forceinline__ void build_chi(int q, int8_t* chi2, int8_t* sq) {
+// Fill chi2 (2q + 1 entries; kind 3: the first q) cooperatively; `sq` is q scratch bytes.
+__device__ __forceinline__ void build_chi(int q, int8_t* chi2, int8_t* sq, int kind = 1) {
   for (int i = threadIdx.x; i < q; i += blockDim.x) sq[i] = 0;
   __syncthreads();
+  if (kind == 3) {
+    for (int i = 1 + threadIdx.x; i < q; i += blockDim.x) sq[gf343_square(i)] = 1;
+    __syncthreads();
+    for (int d = threadIdx.x; d < q; d += blockDim.x) chi2[d] = d == 0 ? 0 : (sq[d] ? 1 : -1);
+    __syncthreads();
+    return;
+  }
   for (int i = 1 + threadIdx.x; i <= (q - 1) / 2; i += blockDim.x) sq[(i * i) % q] = 1;
   __syncthreads();
   for (int d = threadIdx.x; d < 2 * q + 1; d += blockDim.x) {

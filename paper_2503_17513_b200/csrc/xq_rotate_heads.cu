@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(kWarps * 32, MX ? 1 : 2) rotate_quant_heads_ke
     // prepared with the weights (a constant of the plan)
     for (int i = tid; i < dp * pitch / 8; i += blockDim.x) xqptx::cp_async16(Bs + 8 * i, Bimage + 8 * i);
   } else {
-    if (pl.p > 1) build_chi(q, chi2, sq);
+    if (pl.p > 1) build_chi(q, chi2, sq, pl.paley_kind);
     for (int i = tid; i < dp * pitch; i += blockDim.x) {
       const int c2 = i / pitch, c = i - c2 * pitch;
       uint16_t bits = 0;

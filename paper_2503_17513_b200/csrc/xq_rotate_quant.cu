@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(256) rotate_quant_general_kernel(const __nv_bf
   float* red = bufB + Kp;
   int8_t* chi2 = reinterpret_cast<int8_t*>(red + 32);
   int8_t* sq = chi2 + 2 * q + 1;
-  if (p > 1) build_chi(q, chi2, sq);
+  if (p > 1) build_chi(q, chi2, sq, pl.paley_kind);
   const int rows_a = (K + n - 1) / n;  // rows of the p x n view that can be non-zero
 
   for (int row = blockIdx.x; row < M; row += gridDim.x) {
@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(512) rotate_quant_tc_kernel(const __nv_bfloat1
     __syncthreads();
     xqrot::load_afrag<KS>(afrag, Hs, P16, hpitch, mt, lane);
   } else {
-  build_chi(q, chi2, sq);
+  build_chi(q, chi2, sq, pl.paley_kind);
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks) {
 #pragma unroll

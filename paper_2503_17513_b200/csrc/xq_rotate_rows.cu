@@ -44,7 +44,7 @@ template <int LOG2N, int KS, int MTW, int QM>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     rotate_quant_rows_kernel(const __nv_bfloat16* __restrict__ X, int M, long long ldx, xq_hadamard_plan_t pl, float gamma,
                              uint8_t* __restrict__ Xq, float* __restrict__ sx, float* __restrict__ Yopt, uint8_t* __restrict__ A8opt,
-                             int32_t* __restrict__ zp, uint8_t* __restrict__ sfb, int Kq, int Wr, int G, int fold) {
+                             int32_t* __restrict__ zp, uint8_t* __restrict__ sfb, int Kq, int Wr, int G, int fold, int nbuf) {
   constexpr bool ASYM = QM == 1;
   constexpr int n = 1 << LOG2N, NT8 = n / 8;
   constexpr int xpitch = n + 8;        // bf16 elements per staged row (conflict-free ldmatrix)
@@ -56,14 +56,14 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
   const int group = warp / Wr, wg = warp - group * Wr, tg = tid - group * Wr * 32, gthreads = Wr * 32;
 
   __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(smem_raw);                       // [MT * 16][hpitch]
-  __nv_bfloat16* Xs_all = Hs + MT * 16 * hpitch;                                        // [G][2][KS * 16][xpitch]
+  __nv_bfloat16* Xs_all = Hs + MT * 16 * hpitch;                                        // [G][nbuf][KS * 16][xpitch]
   constexpr int tpitch = n + 8;        // floats per row of the transpose tile
-  float* tr_all = reinterpret_cast<float*>(Xs_all + (size_t)G * 2 * KS * 16 * xpitch);  // [warps][8][tpitch]
+  float* tr_all = reinterpret_cast<float*>(Xs_all + (size_t)G * nbuf * KS * 16 * xpitch);  // [warps][8][tpitch]
   float* red_all = tr_all + (size_t)G * Wr * 8 * tpitch;                                // [G][2 Wr] + 32 spare
   int8_t* chi2 = reinterpret_cast<int8_t*>(red_all + 2 * G * Wr + 32);
   int8_t* sq = chi2 + 2 * q + 1;
 
-  if (pl.p > 1) build_chi(q, chi2, sq);
+  if (pl.p > 1) build_chi(q, chi2, sq, pl.paley_kind);
   xqptx::pdl_launch_dependents();
   // H_p^T: row a' (output index), column a (input index); zero outside p x p
   for (int i = tid; i < MT * 16 * KS * 16; i += blockDim.x) {
@@ -76,12 +76,12 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     Hs[a2 * hpitch + a] = __ushort_as_bfloat16((unsigned short)sign_bf16(s));
   }
   // zero the staged rows once: rows past the data and the tail of a partial last row stay zero
-  for (int i = tid; i < G * 2 * KS * 16 * xpitch / 8; i += blockDim.x) reinterpret_cast<uint4*>(Xs_all)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < G * nbuf * KS * 16 * xpitch / 8; i += blockDim.x) reinterpret_cast<uint4*>(Xs_all)[i] = make_uint4(0, 0, 0, 0);
   xqptx::pdl_wait();
   __syncthreads();
   if (group >= G) return;
 
-  __nv_bfloat16* Xs = Xs_all + (size_t)group * 2 * KS * 16 * xpitch;
+  __nv_bfloat16* Xs = Xs_all + (size_t)group * nbuf * KS * 16 * xpitch;
   float* tr = tr_all + (size_t)warp * 8 * tpitch;
   float* red = red_all + group * 2 * Wr;
   constexpr int TPL = NT8 / 4;  // (row, j) tuples of eight columns per lane and pass of eight rows
@@ -97,10 +97,15 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
 
+  // nbuf == 2: the next row lands while this one is computed; nbuf == 1 (long rows on a large order-p factor, whose
+  // image leaves room for one stage only): the load of a row follows the last use of the stage by the row before
   int row = blockIdx.x * G + group, buf = 0;
-  if (row < M) issue_load(row, 0);
-  for (; row < M; row += stride, buf ^= 1) {
-    if (row + stride < M) {
+  if (row < M && nbuf == 2) issue_load(row, 0);
+  for (; row < M; row += stride, buf = nbuf == 2 ? buf ^ 1 : 0) {
+    if (nbuf == 1) {
+      issue_load(row, 0);
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else if (row + stride < M) {
       issue_load(row + stride, buf ^ 1);
       asm volatile("cp.async.wait_group 1;" ::: "memory");
     } else {
@@ -303,10 +308,15 @@ cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard
   constexpr int n = 1 << LOG2N;
   const int fold = pl.log2n - LOG2N;  // Sylvester bits folded into the outer factor
   const int MT = ((pl.p << fold) + 15) / 16, Wr = (MT + MTW - 1) / MTW;
-  int G = kMaxWarps / Wr;
+  int G = kMaxWarps / Wr, nbuf = 2;
   const size_t fixed = (size_t)MT * 16 * (KS * 16 + 8) * 2 + 32 * 4 + (size_t)(3 * pl.q + 1) + 64;
-  const size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 8;
+  size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 8;
   while (G > 1 && fixed + G * per_group > 224 * 1024) --G;
+  if (fixed + G * per_group > 224 * 1024) {  // one row group and still too much: a single stage
+    nbuf = 1;
+    per_group -= (size_t)KS * 16 * (n + 8) * 2;
+  }
+  if (fixed + G * per_group > 224 * 1024 || Wr > kMaxWarps) return cudaErrorNotSupported;
   const size_t smem = fixed + G * per_group;
   auto kern = mx ? rotate_quant_rows_kernel<LOG2N, KS, MTW, 2>
                  : (zp ? rotate_quant_rows_kernel<LOG2N, KS, MTW, 1> : rotate_quant_rows_kernel<LOG2N, KS, MTW, 0>);
@@ -326,7 +336,7 @@ cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sfb, Kq, Wr, G, fold);
+  return cudaLaunchKernelEx(&cfg, kern, (const __nv_bfloat16*)X, (int)M, (long long)ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sfb, Kq, Wr, G, fold, nbuf);
 }
 
 template <int LOG2N, int MTW>
@@ -360,6 +370,9 @@ cudaError_t launch_rows_64_long(int ks, const void* X, int32_t M, int64_t ldx, c
     case 6: return launch_rows<6, 6, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
     case 7: return launch_rows<6, 7, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
     case 8: return launch_rows<6, 8, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 9: case 10: return launch_rows<6, 10, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 11: case 12: return launch_rows<6, 12, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
+    case 13: case 14: return launch_rows<6, 14, 2>(X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
     default: return launch_rows_ks<6, 2>(ks, X, M, ldx, pl, gamma, Xq, sx, Yopt, A8opt, zp, sms, st, mx);
   }
 }
@@ -371,11 +384,15 @@ bool xq_rotate_rows_supported(const xq_hadamard_plan_t& pl) {
   if (pl.p == 1 && pl.log2n < 9) return false;  // small pure Sylvester orders: the general kernel
   const int log2n = pl.log2n > 7 ? 7 : pl.log2n, fold = pl.log2n - log2n;
   const int n = 1 << log2n, rows_a = (pl.K + n - 1) / n, MT = ((pl.p << fold) + 15) / 16;
-  if (rows_a > ((fold || log2n == 6) ? 128 : 64) || MT > 15) return false;
-  if (rows_a > 64) {  // the CTA must hold at least one row group
-    const int ks = (rows_a + 15) / 16;
-    const size_t need = (size_t)MT * 16 * (ks * 16 + 8) * 2 + (size_t)2 * ks * 16 * (n + 8) * 2 + (size_t)MT * 8 * (n + 8) * 4 + 4096;
-    if (need > 224 * 1024) return false;
+  // n = 64 also takes long rows on a large order-p factor (the paper's 14336 -> 19968 = 312 x 64: 224 staged input rows,
+  // 20 tiles of 16 output rows on 10 warps, a single load stage)
+  const int max_rows = log2n == 6 && !fold ? 224 : (fold ? 128 : 64), max_mt = log2n == 6 && !fold ? 32 : 15;
+  if (rows_a > max_rows || MT > max_mt) return false;
+  if (rows_a > 64 || MT > 15) {  // the CTA must hold at least one row group, with one load stage if need be
+    const int ks = (rows_a + 15) / 16 + ((rows_a > 128) ? ((rows_a + 15) / 16) % 2 : 0);  // long rows: KS comes in steps of 2
+    const int wr = log2n == 6 ? (MT + 1) / 2 : MT;
+    const size_t need = (size_t)MT * 16 * (ks * 16 + 8) * 2 + (size_t)ks * 16 * (n + 8) * 2 + (size_t)wr * 8 * (n + 8) * 4 + 4096;
+    if (need > 224 * 1024 || wr > kMaxWarps) return false;
   }
   return true;
 }

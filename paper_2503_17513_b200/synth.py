@@ -80,9 +80,7 @@ LLAMA_8B = {
     "up": (4096, 4352, 14336),
     "down": (14336, 15360, 4096),
 }
-# Down projections at the expansion sizes of the paper's Table 1 (8192 -> 2048 and 14336 -> 4096).  The two
-# largest 8B sizes (19968 = 312 x 64, 22016 = 5504 x 4) are left to the parity tests: their order-p factors
-# are beyond the tensor-core rotate kernels and would make a timing of the table a timing of the general kernel.
+# Down projections at the expansion sizes of the paper's Table 1 (8192 -> 2048 and 14336 -> 4096).
 TABLE1_1B_DOWN = {
     "kp8960": (8192, 8960, 2048),
     "kp9728": (8192, 9728, 2048),
@@ -92,6 +90,8 @@ TABLE1_1B_DOWN = {
 TABLE1_8B_DOWN = {
     "kp15360": (14336, 15360, 4096),
     "kp18432": (14336, 18432, 4096),
+    "kp19968": (14336, 19968, 4096),
+    "kp22016": (14336, 22016, 4096),
 }
 # Attention output projections with the head-wise rotation expanded (K, K', N, heads): 32 heads of 64 -> 72 / 80
 # channels (Llama-3.2-1B-like) and of 128 -> 144 / 160 channels (Llama-3-8B-like).

@@ -83,9 +83,10 @@ ROTATE_CASES = [
     # n > 256 and pure Sylvester orders through the folded outer factor
     (50, 4096, 4096), (50, 8192, 12288), (64, 1000, 1024),
     # the expansion sizes of Table 1: 140 x 64 (128 staged input rows), 76 x 128, 20 x 512, 36 x 512, and the two
-    # orders that only the general kernel takes (312 x 64, 5504 x 4)
+    # the two largest 8B sizes: 312 x 64 and 344 x 64 (Paley over GF(7^3)), long rows on a large outer factor; 344 and
+    # 688 = 344 x 2 through the general kernel
     (3, 8192, 8960), (60, 8192, 8960), (3, 8192, 9728), (60, 8192, 9728), (3, 8192, 10240), (2, 14336, 18432),
-    (60, 14336, 18432), (1, 14336, 19968), (1, 14336, 22016),
+    (60, 14336, 18432), (1, 14336, 19968), (170, 14336, 19968), (1, 14336, 22016), (155, 14336, 22016), (5, 300, 344), (70, 600, 688),
 ]
 
 
