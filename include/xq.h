@@ -45,7 +45,8 @@ typedef enum {
   XQ_ERR_ALLOC = 4,             /* device or host allocation failed */
   XQ_ERR_CUDA = 5,              /* a CUDA runtime call or launch failed */
   XQ_ERR_TIMEOUT = 6,           /* a bounded device-side wait ran out (sticky, see xq_poll_status) */
-  XQ_ERR_BOUNDS = 7             /* device-side self check failed (sticky) */
+  XQ_ERR_BOUNDS = 7             /* an index self check of a product kernel failed (sticky); raised only by the
+                                   build made with -DXQ_DEBUG_BOUNDS, where the access is then skipped */
 } xq_status;
 
 /* Hadamard plan: Kp = p * 2^log2n and H = H_p (x) S_{2^log2n} (Kronecker product, the order-p

@@ -62,6 +62,7 @@ struct DecodeParams {
   const int32_t* zp;    // per-token zero points of asymmetric activation codes, or null
   const int32_t* wsum;  // per-channel sums of the weight codes
   int32_t* status;
+  size_t w_bytes;   // size of the weight image (read by the self checks of the debug build only)
   int M, N, Kp;
   int k_groups;     // groups of 32 codes per channel block in the weight layout (K'' / 32)
   int n_blocks;     // channel blocks holding real channels: ceil(N / 16)
@@ -261,7 +262,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         const uint32_t bytes = (uint32_t)ng * XQ_GROUP_BYTES;
         const unsigned char* src = p.W + ((size_t)(b0 + (t >> p.log2S)) * p.k_groups + g0 + 4 * c_lo) * XQ_GROUP_BYTES;
         mbar_expect_tx(&full[stage], bytes);
-        bulk_g2s_hint(ring + (size_t)stage * kStageBytes, src, bytes, &full[stage], stream_policy);
+        if (XQ_IN_BOUNDS(ng > 0 && bytes <= (uint32_t)kStageBytes && stage < p.stages && src >= p.W && (size_t)(src - p.W) + bytes <= p.w_bytes,
+                         p.status))
+          bulk_g2s_hint(ring + (size_t)stage * kStageBytes, src, bytes, &full[stage], stream_policy);
+        else
+          mbar_complete_tx(&full[stage], bytes);
         if (stage == lane) ++use_a; else ++use_b;
         n = next_n(n);
         if (!exists(n)) active = false;
@@ -353,6 +358,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
           if (i < total) {
             const int m = i / L, l = i - m * L;
             unsigned char* d = act + (size_t)m * p.act_pitch + (size_t)(l >> 2) * 128 + (size_t)(l & 3) * 8;
+            if (!XQ_IN_BOUNDS(m < MT && (size_t)(l >> 2) * 128 + (size_t)(l & 3) * 8 + 104 <= (size_t)p.act_pitch, p.status)) continue;
             uint2 e;
             split16(v[u].x, e.x, e.y);
             *reinterpret_cast<uint2*>(d) = e;
@@ -427,6 +433,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         const int2 v1 = make_int2(acc[n][0][2] + acc[n][1][2] + acc[n][2][2] + acc[n][3][2], acc[n][0][3] + acc[n][1][3] + acc[n][2][3] + acc[n][3][3]);
         int* d0 = &tl[ag * MT + 8 * n + 2 * at];
         int* d1 = &tl[(ag + 8) * MT + 8 * n + 2 * at];
+        // the tile lies inside the partial-tile area of its owner (every CTA of the cluster has the same layout)
+        if (!XQ_IN_BOUNDS(tl >= tiles && (size_t)(tl - tiles + 16 * MT) * sizeof(int) + (size_t)MT * p.act_pitch <= (size_t)p.region_bytes, p.status))
+          continue;
         if (owner == rank) {
           *reinterpret_cast<int2*>(d0) = v0;
           *reinterpret_cast<int2*>(d1) = v1;
@@ -473,6 +482,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_decode_kernel(const DecodePa
         w1 = *reinterpret_cast<const int4*>(p.wsum + n0 + 4);
       }
       const int* col = tiles + (size_t)jj * srcs * 16 * MT + (8 * h) * MT + m;
+      if (!XQ_IN_BOUNDS(((size_t)(jj + 1) * srcs * 16 * MT) * sizeof(int) + (size_t)MT * p.act_pitch <= (size_t)p.region_bytes && m < p.M &&
+                            n0 < p.n_blocks * 16,
+                        p.status))
+        continue;
       int v[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] = col[e * MT];
@@ -695,6 +708,7 @@ void fill_params(DecodeParams& p, const DecodePlan& d, const uint8_t* Xq, const 
   p.zp = zp;
   p.wsum = w->w_sum;
   p.status = status;
+  p.w_bytes = (size_t)w->Np * w->Kpp / 2;
   p.M = M;
   p.N = w->N;
   p.Kp = w->Kp;

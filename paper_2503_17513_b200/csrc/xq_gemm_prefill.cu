@@ -69,6 +69,7 @@ struct PrefillParams {
   __nv_bfloat16* out;
   int32_t* acc_opt;
   int32_t* status;
+  size_t w_bytes;      // size of the weight image (read by the self checks of the debug build only)
   int M, N, KB;        // KB = K'' / 128 (k blocks of the padded weights)
   int row_blocks;      // blocks of 16 channels in the padded weights
   int tiles_m, tiles_n;
@@ -163,7 +164,13 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
         unsigned char* stage = pk + (size_t)s * kPkBBytes;
         if (lane == 0) mbar_expect_tx(&pk_full[s], (uint32_t)nblk * (4 * XQ_GROUP_BYTES));
         __syncwarp();
-        if (lane < nblk) bulk_g2s(stage + lane * (4 * XQ_GROUP_BYTES), wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES), 4 * XQ_GROUP_BYTES, &pk_full[s]);
+        if (lane < nblk) {
+          const unsigned char* src = wsrc + (size_t)kb * (4 * XQ_GROUP_BYTES);
+          if (XQ_IN_BOUNDS(src >= p.W && (size_t)(src - p.W) + 4 * XQ_GROUP_BYTES <= p.w_bytes && (lane + 1) * (4 * XQ_GROUP_BYTES) <= kPkBBytes, p.status))
+            bulk_g2s(stage + lane * (4 * XQ_GROUP_BYTES), src, 4 * XQ_GROUP_BYTES, &pk_full[s]);
+          else
+            mbar_complete_tx(&pk_full[s], 4 * XQ_GROUP_BYTES);
+        }
       }
     }
   } else if (warp == 1) {
@@ -271,7 +278,8 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
           const size_t o = (size_t)m * p.N + nc;
 #pragma unroll
           for (int g8 = 0; g8 < 4; ++g8) {
-            if (nc + 8 * g8 < p.N) {  // N is a multiple of 8 on this path
+            if (nc + 8 * g8 < p.N &&  // N is a multiple of 8 on this path
+                XQ_IN_BOUNDS(o + 8 * g8 + 8 <= (size_t)p.M * p.N && nc + 8 * g8 + 8 <= p.N, p.status)) {
               int a[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e)  // every product carries 16 x 16; sum (c - z) qw = sum c qw - z sum qw
@@ -518,6 +526,7 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int
   p.out = (__nv_bfloat16*)out;
   p.acc_opt = acc_opt;
   p.status = status;
+  p.w_bytes = (size_t)w->Np * w->Kpp / 2;
   p.M = M;
   p.N = w->N;
   p.KB = w->Kpp / XQ_K_BLOCK;

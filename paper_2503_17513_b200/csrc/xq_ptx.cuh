@@ -53,6 +53,26 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
   return false;
 }
 
+// Counts `bytes` as arrived on the barrier without a copy: stands in for a bulk copy that a self check refused,
+// so that the waiters of the stage still wake.
+__device__ __forceinline__ void mbar_complete_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+// ---- self checks of the debug build -------------------------------------------------------------
+// Compiled with -DXQ_DEBUG_BOUNDS the product kernels test their computed indices before they use them: a failing
+// test writes 7 (XQ_ERR_BOUNDS) into the workspace status word and the access is skipped; nothing traps.  In the
+// normal build the test is the constant true and the condition is never evaluated.
+#ifdef XQ_DEBUG_BOUNDS
+__device__ __forceinline__ bool xq_bounds_report(bool ok, int* status) {
+  if (!ok) atomicExch(status, 7);
+  return ok;
+}
+#define XQ_IN_BOUNDS(cond, status) xqptx::xq_bounds_report((cond), (status))
+#else
+#define XQ_IN_BOUNDS(cond, status) (true)
+#endif
+
 // ---- bulk copy global -> shared, completion counted in bytes on an mbarrier ------------------
 // Both addresses 16-byte aligned, size a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {

@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libxq.so")
+# XQ_LIBRARY names another build of the same library (the self-checking one, see build.py) to load instead
+LIB_PATH = os.environ.get("XQ_LIBRARY") or os.path.join(_PKG, "libxq.so")
 _lib = None
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_ORDER, ERR_WORKSPACE, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = range(8)
