@@ -62,8 +62,6 @@ FALLBACK_BF16_TFLOPS = (1590.0, 1400.0)
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     ("1b-decode", 32): (6.58e6, "profiles/gemm_decode_1b_decode_m32.txt"),
     ("8b-decode", 16): ((13.47 + 31.32 + 31.32 + 31.49) * 1e6 / 4, "profiles/gemm_decode_8b_decode_m16.txt"),
-    ("8b-prefill", 4096): ((31.802368 + 4.061952 + 51.203840 + 64.903936 + 51.312128 + 65.464064 + 158.099968 + 22.970624) * 1e6 / 4,
-                           "profiles/gemm_prefill_8b_prefill_m4096.txt"),
 }
 
 
@@ -445,7 +443,7 @@ class Bench:
             achieved = ops / t_gemm / 1e12
             peak = pk["int8_burst"] * ratio / 2.0
             roofline = {"bound": "tensor",
-                        "kernel": "xq_mx_gemm (gemm_mx_kernel, tcgen05.mma kind::mxf4)" if mx else "xq_w4a4_gemm (gemm_prefill_kernel, tcgen05.mma kind::i8)",
+                        "kernel": "xq_mx_gemm (gemm_mx_kernel, tcgen05.mma kind::mxf4)" if mx else "xq_w4a4_gemm (gemm_prefill_ts_kernel / gemm_prefill_kernel, tcgen05.mma kind::i8)",
                         "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
                         "peak_source": f"{pk['source']}: {ratio:g} x burst bf16 GEMM",
                         "peak_sustained": pk["int8_sustained"] * ratio / 2.0, "frac_of_sustained": achieved / (pk["int8_sustained"] * ratio / 2.0),

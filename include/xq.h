@@ -25,6 +25,11 @@
  *    that takes the object (XQ_ERR_INVALID_ARG otherwise).
  *  - No global state, except in xq_expanded_linear_static (see there): calls on distinct streams
  *    with distinct workspaces may run concurrently.
+ *  - One environment variable is read (once, at the first product of more than 32 tokens):
+ *    XQ_PREFILL_KERNEL overrides the choice between the two forms of the tcgen05 tile kernel, for
+ *    measurements and tests: "ss" keeps the first form (expanded weights in shared memory), "ts"
+ *    or "ts:<tokens>" forces the second (expanded weights in tensor memory).  Results are the
+ *    same bits either way.
  */
 #ifndef XQ_H_
 #define XQ_H_
@@ -315,8 +320,9 @@ xq_status xq_expanded_linear_static(const void* X_bf16_dev, int32_t M, int64_t l
 /* Diagnostic, host only, nothing is launched (no counterpart in the paper): which kernel the quantized
  * product of M tokens against w runs in, and its tile.  *kind = 0: the split-K weight-stream kernel
  * of M <= 32 tokens (tile_tokens = tokens padded to 8, 16 or 32; tile_channels = 16); 1: the
- * tcgen05 tile kernel (tile_tokens x tile_channels one of 128 x 256, 256 x 256, 256 x 128, 256 x 224); 2: the
- * one-thread-per-output kernel (1 x 1).  Tests use it to name the tile shape a case exercised.
+ * tcgen05 tile kernel in its first form (tile_tokens x tile_channels one of 128 x 256, 256 x 256, 256 x 128,
+ * 256 x 224); 3: the tile kernel in its second form (tile_tokens a multiple of 32 up to 192, tile_channels = 256);
+ * 2: the one-thread-per-output kernel (1 x 1).  Tests use it to name the tile shape a case exercised.
  * Errors: INVALID_ARG (null pointer, M < 1, wrong current device), CUDA. */
 xq_status xq_gemm_kernel_info(int32_t M, const xq_weights* w, int32_t* kind, int32_t* tile_tokens,
                               int32_t* tile_channels);

@@ -97,9 +97,10 @@ extern "C" xq_status xq_gemm_kernel_info(int32_t M, const xq_weights* w, int32_t
     *tile_tokens = mt;
     *tile_channels = 16;
   } else if (xq_gemm_wants_a8(M, w)) {
-    const int c = xq_prefill_tile_choice(M, w, w->sms);
-    *kind = 1;
-    *tile_tokens = c == 0 ? 128 : 256;
+    int ts_tokens = 0;
+    const int c = xq_prefill_tile_choice(M, w, w->sms, &ts_tokens);
+    *kind = c == 4 ? 3 : 1;
+    *tile_tokens = c == 4 ? ts_tokens : (c == 0 ? 128 : 256);
     *tile_channels = c == 2 ? 128 : (c == 3 ? 224 : 256);
   } else {
     *kind = 2;

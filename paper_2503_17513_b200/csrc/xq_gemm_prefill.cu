@@ -27,6 +27,9 @@
 // status word, every role leaves its loop, and tensor memory is released before exit.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <stdlib.h>
+
+#include <string>
 
 #include "xq_internal.h"
 #include "xq_ptx.cuh"
@@ -465,6 +468,8 @@ cudaError_t launch_mh(const CUtensorMap& mapA, PrefillParams p, int sms, cudaStr
 
 }  // namespace
 
+XqEncodeTiledFn xq_encode_tiled_fn() { return (XqEncodeTiledFn)encode_tiled_fn(); }
+
 bool xq_prefill_supported(int32_t M, const xq_weights* w) {
   return M >= 1 && w->Kp % 32 == 0 && w->N % 8 == 0 && w->Np % 256 == 0;
 }
@@ -485,24 +490,63 @@ cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, ui
   return cudaLaunchKernelEx(&cfg, expand_tokens_kernel, (const uint4*)Xq, pieces, (uint4*)A8);
 }
 
-// Three tile shapes; a cost model picks one: waves of tiles over the multiprocessors times the cycles of a tile
-// (69 tensor-core cycles per 128 x 256 x 32 MMA; 128-token tiles expand every weight for half as many MMAs and run
-// at about 0.62 of that rate; an epilogue that is not hidden costs about 2000 cycles).
-// A fourth shape, 256 tokens x 224 channels, costs 7/8 of the 256 x 256 tile and exists for the wave count: 14336 =
-// 64 x 224 channels in 256-token rows are 6.9 waves on 148 SMs instead of 6.05 (which runs as 7), 8192 channels
-// and 2048 tokens are exactly 2 waves.
-// Returns 0 for 128 tokens x 256 channels, 1 for 256 x 256, 2 for 256 x 128, 3 for 256 x 224.
-int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms) {
+// Two forms of the kernel and several tile shapes; a cost model picks one.  Costs are in units of about 1.5 ns,
+// fitted to measured launches: waves of tiles over the multiprocessors times the cost of a tile.
+// First form (expanded weights in shared memory): 69 units per 128 x 256 x 32 MMA; 128-token tiles expand every
+// weight for half as many MMAs and run at about 0.62 of that rate; an epilogue that is not hidden costs about 2000.
+// 256 tokens x 224 channels costs 7/8 of the 256 x 256 tile and exists for the wave count (14336 = 64 x 224).
+// Second form (expanded weights in tensor memory, xq_gemm_prefill_ts.cu): tiles of NT tokens x 256 channels, NT in
+// {192, 160, 128} or the token count rounded up to 32 when that is less; a K block costs 206 + 92 NT / 192 (the
+// hand-over chain of the two staging stages bounds it, not the tensor pipe), a tile 2400 more (its epilogue is
+// not hidden), a launch 3400 more (inside a layer, behind the rotate kernel, it measured 4-14 us per launch slower
+// than alone, the first form less so): it is taken for the large products, where it is 10-20 % faster.
+// Returns 0 for 128 tokens x 256 channels, 1 for 256 x 256, 2 for 256 x 128, 3 for 256 x 224 (first form), 4 for
+// *ts_tokens x 256 in the second form.  XQ_PREFILL_KERNEL in the environment (read once) overrides the choice for
+// measurements and tests: "ss" keeps the first form, "ts" or "ts:<tokens>" forces the second.
+int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms, int* ts_tokens) {
+  static const std::string force = [] {
+    const char* e = getenv("XQ_PREFILL_KERNEL");
+    return std::string(e ? e : "");
+  }();
   const int KB = w->Kpp / XQ_K_BLOCK, tm1 = (M + BMH - 1) / BMH, tm2 = (M + 2 * BMH - 1) / (2 * BMH);
   auto waves = [&](int tiles) { return (double)((tiles + sms - 1) / sms); };
+  const int m32 = (M + 31) / 32 * 32;
+  auto ts_cost = [&](int nt) {
+    return waves(((M + nt - 1) / nt) * ((w->N + 255) / 256)) * (KB * (206.0 + 92.0 * nt / 192.0) + 2400.0) + 3400.0;
+  };
+  int best_nt = m32 < 128 ? m32 : 128;
+  double t_ts = ts_cost(best_nt);
+  for (int nt = 160; nt <= XQ_TS_MAX_TOKENS && nt <= m32; nt += 32)
+    if (ts_cost(nt) < t_ts) {
+      t_ts = ts_cost(nt);
+      best_nt = nt;
+    }
+  *ts_tokens = best_nt;
+  if (force.rfind("ts", 0) == 0) {
+    if (force.size() > 3) {
+      const int nt = atoi(force.c_str() + 3) / 32 * 32;
+      if (nt >= 32 && nt <= XQ_TS_MAX_TOKENS) *ts_tokens = nt < m32 ? nt : m32;
+    }
+    return 4;
+  }
   const double t_1x256 = waves(tm1 * ((w->N + 255) / 256)) * (KB * 276.0 / 0.62);
   const double t_2x256 = waves(tm2 * ((w->N + 255) / 256)) * (KB * 552.0 + 2000.0);
   const double t_2x128 = waves(tm2 * ((w->N + 127) / 128)) * (KB * 276.0 / 0.80);  // N = 128 MMAs re-read the tokens twice as often
   const double t_2x224 = waves(tm2 * ((w->N + 223) / 224)) * (KB * 483.0 + 1750.0);
-  if (t_2x224 < 0.97 * t_2x256 && t_2x224 < t_2x128 && t_2x224 < t_1x256) return 3;  // only for a clear gain
-  if (t_2x128 <= t_2x256 && t_2x128 <= t_1x256) return 2;
-  if (t_2x256 <= t_1x256) return 1;
-  return 0;
+  int c = 0;
+  double t_ss = t_1x256;
+  if (t_2x224 < 0.97 * t_2x256 && t_2x224 < t_2x128 && t_2x224 < t_1x256) {  // only for a clear gain
+    c = 3;
+    t_ss = t_2x224;
+  } else if (t_2x128 <= t_2x256 && t_2x128 <= t_1x256) {
+    c = 2;
+    t_ss = t_2x128;
+  } else if (t_2x256 <= t_1x256) {
+    c = 1;
+    t_ss = t_2x256;
+  }
+  if (force != "ss" && t_ts <= t_ss) return 4;
+  return c;
 }
 
 cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w,
@@ -533,7 +577,9 @@ cudaError_t xq_launch_gemm_prefill(const uint8_t* A8, const float* sx, const int
   p.row_blocks = w->Np / XQ_ROW_BLOCK;
   p.tiles_n = 0;
   p.tiles_m = 0;
-  switch (xq_prefill_tile_choice(M, w, sms)) {
+  int ts_tokens = 0;
+  switch (xq_prefill_tile_choice(M, w, sms, &ts_tokens)) {
+    case 4: return xq_launch_gemm_prefill_ts(A8, sx, zp, M, w, out, acc_opt, status, ts_tokens, sms, st);
     case 3: return launch_mh<2, 224>(mapA, p, sms, st);
     case 2: return launch_mh<2, 128>(mapA, p, sms, st);
     case 1: return launch_mh<2, 256>(mapA, p, sms, st);

@@ -2,6 +2,7 @@
 // included by the oracle).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
@@ -166,8 +167,18 @@ cudaError_t xq_launch_linear_decode(const void* X, int64_t ldx, uint8_t* Xq, flo
                                     void* out, int32_t* header, cudaStream_t st);
 // True when M tokens against w run in the decode kernel; then also its padded token count and cluster size.
 bool xq_decode_shape(int32_t M, const xq_weights* w, int* padded_tokens, int* cluster);
-// Tile shape the tensor-core kernel picks: 0 = 128 tokens x 256 channels, 1 = 256 x 256, 2 = 256 x 128.
-int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms);
+// Tile shape the tensor-core path picks: 0 = 128 tokens x 256 channels, 1 = 256 x 256, 2 = 256 x 128, 3 = 256 x 224
+// (first form: expanded weights in shared memory); 4 = *ts_tokens tokens x 256 channels in the second form (expanded
+// weights in tensor memory).
+#define XQ_TS_MAX_TOKENS 192
+int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms, int* ts_tokens);
+cudaError_t xq_launch_gemm_prefill_ts(const uint8_t* A8, const float* sx, const int32_t* zp, int32_t M, const xq_weights* w, void* out,
+                                      int32_t* acc_opt, int32_t* status, int tile_tokens, int sms, cudaStream_t st);
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (null when the driver lacks it).
+typedef CUresult (*XqEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+XqEncodeTiledFn xq_encode_tiled_fn();
 // Tensor-core path: takes the tokens one code per byte (16 x code, even codes of every word first),
 // as written by the rotate kernels' optional output or by xq_launch_expand_tokens.
 bool xq_prefill_supported(int32_t M, const xq_weights* w);

@@ -3,7 +3,7 @@
 In that build the product kernels test every computed index before using it (the source range and ring stage of each
 weight copy, the stores into the token slice and the partial tiles, the output offsets); a failing test writes
 XQ_ERR_BOUNDS into the workspace status word and skips the access, nothing traps.  A memory checker cannot be run
-where these tests run, so this build stands in for it: every kernel kind and tile shape is driven through shapes with
+where these tests run, so this build stands in for it: every kernel kind, both forms of the tile kernel and every tile shape are driven through shapes with
 ragged tails, the status word must stay clean and the outputs must equal those of the normal build bit for bit.
 
 The debug library is loaded in a child process (XQ_LIBRARY selects it), so that the normal one stays the library of
@@ -26,7 +26,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 CASES = [
     (1, 16, 104, 136), (8, 37, 136, 144), (3, 2048, 2048, 2176), (12, 1024, 2048, 2176), (32, 2048, 2048, 2176), (17, 384, 4096, 4352),
     (32, 2048, 8192, 8704), (130, 264, 2048, 2176), (384, 9728, 248, 256), (300, 200, 4096, 4608),
-    (2048, 4096, 2048, 2176), (2048, 3072, 2048, 2176), (2048, 2048, 8192, 8704), (33, 257, 64, 64),
+    (2048, 4096, 2048, 2176), (2048, 3072, 2048, 2176), (2048, 2048, 8192, 8704), (2048, 8192, 2048, 2176), (33, 257, 64, 64),
 ]
 
 CHILD = r"""
@@ -62,12 +62,16 @@ print("RESULT " + json.dumps(res))
 """
 
 
-def run_child(library):
+def run_child(library, tile_form):
     env = dict(os.environ)
     if library:
         env["XQ_LIBRARY"] = library
     else:
         env.pop("XQ_LIBRARY", None)
+    if tile_form:
+        env["XQ_PREFILL_KERNEL"] = tile_form
+    else:
+        env.pop("XQ_PREFILL_KERNEL", None)
     env["PYTHONPATH"] = ROOT + os.pathsep + env.get("PYTHONPATH", "")
     r = subprocess.run([sys.executable, "-c", CHILD, json.dumps(CASES)], env=env, capture_output=True, text=True, timeout=900, cwd=ROOT)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
@@ -80,15 +84,20 @@ def test_debug_build_stays_clean_and_matches_the_normal_build():
     from paper_2503_17513_b200 import build
 
     debug_lib = build.build_library(debug_bounds=True)  # no-op when the library is newer than its sources
-    dbg = run_child(debug_lib)
-    ref = run_child(None)
     kinds = set()
-    for case, d, r in zip(CASES, dbg, ref):
-        assert all(s == 0 for s in d["status"]), (case, d["status"])  # XQ_OK: neither XQ_ERR_BOUNDS nor a timeout
-        assert d["kind"] == r["kind"] and d["sums"] == r["sums"] and d["one_launch"] == r["one_launch"], case
-        assert False not in d["one_launch"], case  # the one-launch form, where the plan admits it, gives the same bits
-        kinds.add(tuple(d["kind"]))
+    sums = []
+    for tile_form in ("", "ss", "ts"):  # the library's own choice of tile kernel form, the first form only, the second only
+        dbg = run_child(debug_lib, tile_form)
+        ref = run_child(None, tile_form)
+        for case, d, r in zip(CASES, dbg, ref):
+            assert all(s == 0 for s in d["status"]), (case, d["status"])  # XQ_OK: neither XQ_ERR_BOUNDS nor a timeout
+            assert d["kind"] == r["kind"] and d["sums"] == r["sums"] and d["one_launch"] == r["one_launch"], case
+            assert False not in d["one_launch"], case  # the one-launch form, where the plan admits it, gives the same bits
+            kinds.add(tuple(d["kind"]))
+        sums.append([d["sums"] for d in dbg])
+    assert sums[0] == sums[1] == sums[2]  # both forms of the tile kernel give the same bits
     # every kernel kind and every tile shape was reached
-    assert {k[0] for k in kinds} == {0, 1, 2}
+    assert {k[0] for k in kinds} == {0, 1, 2, 3}
     assert {(k[1], k[2]) for k in kinds if k[0] == 1} == {(128, 256), (256, 256), (256, 128), (256, 224)}
+    assert len({k[1] for k in kinds if k[0] == 3}) >= 3 and all(k[2] == 256 for k in kinds if k[0] == 3)
     assert {k[1] for k in kinds if k[0] == 0} >= {8, 32}  # padded token counts of the decode stream

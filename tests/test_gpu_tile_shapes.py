@@ -1,13 +1,23 @@
-"""Bit-exact accumulators on every tile shape of the tcgen05 INT4 product kernel, each case naming the
-shape it ran on (asked from the library with xq_gemm_kernel_info, nothing is assumed).
+"""Bit-exact accumulators on every form and tile shape of the tcgen05 INT4 product kernel, each case naming
+the shape it ran on (asked from the library with xq_gemm_kernel_info, nothing is assumed).
 
 The quantized product Q(XR) Q(W~) of the paper's Sec. 3 is an integer sum, so given identical codes
-the int32 accumulators must equal the oracle's int64 sums exactly, whatever tile shape, tile count
-per CTA, K length or tail the launch has.  Cases here reach the three shapes the kernel can pick
-(128 tokens x 256 channels, 256 x 256, 256 x 128, 256 x 224) at the layer sizes the benchmark times, and the
-extreme codes (-8 against -8 and against 7) at the longest K' of the paper's Table 1, where the
-16 x 16 factor carried by the nibble expansion makes the partial sums largest.
+the int32 accumulators must equal the oracle's int64 sums exactly, whatever form, tile shape, tile count
+per CTA, K length or tail the launch has.  The kernel has two forms: the first keeps the expanded weights in
+shared memory (tiles of 128 tokens x 256 channels, 256 x 256, 256 x 128, 256 x 224), the second in tensor memory
+(tiles of 32 .. 192 tokens x 256 channels); the library picks per launch.  Cases here reach every shape at the layer
+sizes the benchmark times, and the extreme codes (-8 against -8 and against 7) at the longest K' of the paper's
+Table 1, where the 16 x 16 factor carried by the nibble expansion makes the partial sums largest.
+
+Every case names two shapes: the one the library picks by itself and the one it picks when XQ_PREFILL_KERNEL=ss
+keeps it to the first form; the last two tests run this file again in child processes, once with that setting and once
+with XQ_PREFILL_KERNEL=ts (every case on the second form, whatever its size), so that both forms are held to the oracle
+on all the cases.
 """
+import os
+import subprocess
+import sys
+
 import numpy as np
 import pytest
 import torch
@@ -16,7 +26,18 @@ from paper_2503_17513_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-TILE_KERNEL = 1
+FIRST, SECOND = 1, 3  # xq_gemm_kernel_info's kinds of the two forms
+FORCED = os.environ.get("XQ_PREFILL_KERNEL", "")
+
+
+def check_shape(info, case_default, case_first):
+    """info = (kind, tile_tokens, tile_channels) as the library reports it for the case."""
+    if FORCED == "ss":
+        assert info == case_first
+    elif FORCED == "ts":
+        assert info[0] == SECOND and info[1] % 32 == 0 and 32 <= info[1] <= 192 and info[2] == 256
+    else:
+        assert info == case_default
 
 
 @pytest.fixture(scope="module")
@@ -44,31 +65,39 @@ def sample_rows(M, count, seed=13):
     return rows
 
 
-# (M, N, K, Kp, tile the library must report, token rows compared: None = all)
+# (M, N, K, Kp, shape the library must report, shape with the first form forced, token rows compared: None = all)
 TILE_CASES = [
-    (384, 9728, 250, 256, (128, 256), None),
-    (2048, 8192, 2048, 2176, (256, 224), None),       # gate / up of the 1B prefill workload: the last 224-wide tile is ragged
-    (2048, 4096, 2048, 2176, (256, 256), None),
-    (512, 14336, 4096, 4352, (256, 224), None),       # gate / up of the 8B workload, all channels (64 x 224)
-    (2048, 2048, 8192, 8704, (256, 128), None),       # down of the 1B prefill workload
-    (2048, 3072, 2048, 2176, (256, 224), None),       # qkv of the 1B prefill workload: tiles reach past the padded rows
-    (4096, 14336, 4096, 4352, (256, 224), 64),        # the 8B prefill launches as the benchmark times them
-    (4096, 6144, 4096, 4352, (256, 256), 64),
-    (4096, 4096, 14336, 15360, (256, 256), 64),
-    (8192, 4096, 4096, 4096, (256, 128), 64),         # the expansion sweep at its two ends
-    (8192, 4096, 4096, 5120, (256, 256), 64),
+    (384, 9728, 250, 256, (FIRST, 128, 256), (FIRST, 128, 256), None),
+    (2048, 8192, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), None),     # gate / up of the 1B prefill workload: ragged last tiles
+    (2048, 4096, 2048, 2176, (FIRST, 256, 256), (FIRST, 256, 256), None),
+    (512, 14336, 4096, 4352, (FIRST, 256, 224), (FIRST, 256, 224), None),     # all channels of the 8B gate / up (64 x 224)
+    (2048, 2048, 8192, 8704, (FIRST, 256, 128), (FIRST, 256, 128), None),     # down of the 1B prefill workload
+    (2048, 3072, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), None),     # qkv of the 1B prefill workload
+    (40, 520, 4096, 4352, (FIRST, 256, 128), (FIRST, 256, 128), None),        # one ragged token tile, ragged channels
+    (4096, 14336, 4096, 4352, (SECOND, 192, 256), (FIRST, 256, 224), 64),     # the 8B prefill launches as the benchmark times them
+    (4096, 6144, 4096, 4352, (SECOND, 192, 256), (FIRST, 256, 256), 64),
+    (4096, 4096, 14336, 15360, (SECOND, 160, 256), (FIRST, 256, 256), 64),
+    (8192, 4096, 4096, 4096, (SECOND, 192, 256), (FIRST, 256, 128), 64),      # the expansion sweep at its two ends
+    (8192, 4096, 4096, 5120, (SECOND, 192, 256), (FIRST, 256, 256), 64),
 ]
-IDS = [f"M{c[0]}-N{c[1]}-Kp{c[3]}-{c[4][0]}x{c[4][1]}" for c in TILE_CASES]
 
 
-@pytest.mark.parametrize("M,N,K,Kp,tile,nrows", TILE_CASES, ids=IDS)
-def test_tile_shape_accumulators_bit_exact(xq, oracle, M, N, K, Kp, tile, nrows):
+def case_id(c):
+    d, f = c[4], c[5]
+    return f"M{c[0]}-N{c[1]}-Kp{c[3]}-{d[1]}x{d[2]}k{d[0]}-or-{f[1]}x{f[2]}"
+
+
+IDS = [case_id(c) for c in TILE_CASES]
+
+
+@pytest.mark.parametrize("M,N,K,Kp,tile,tile_first,nrows", TILE_CASES, ids=IDS)
+def test_tile_shape_accumulators_bit_exact(xq, oracle, M, N, K, Kp, tile, tile_first, nrows):
     qx = synth.int4_codes(M, Kp, seed=21, tag=f"tx{M}")
     qw = synth.int4_codes(N, Kp, seed=21, tag=f"tw{N}")
     s_x = synth.scales(M, seed=21, tag="x")
     s_w = synth.scales(N, seed=21, tag="w")
     w = xq.xq_weights_import(qw, s_w, K)
-    assert xq.xq_gemm_kernel_info(M, w) == (TILE_KERNEL, *tile)
+    check_shape(xq.xq_gemm_kernel_info(M, w), tile, tile_first)
     ws = xq.new_workspace(M, w)
     out = torch.empty((M, N), dtype=torch.int16, device="cuda")
     acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
@@ -85,16 +114,17 @@ def test_tile_shape_accumulators_bit_exact(xq, oracle, M, N, K, Kp, tile, nrows)
 
 
 ASYM_TILE_CASES = [
-    (384, 9728, 250, 256, (128, 256), None),
-    (2048, 8192, 2048, 2176, (256, 224), 256),
-    (2048, 4096, 2048, 2176, (256, 256), 256),
-    (2048, 2048, 8192, 8704, (256, 128), 256),
-    (4096, 4096, 14336, 15360, (256, 256), 64),
+    (384, 9728, 250, 256, (FIRST, 128, 256), (FIRST, 128, 256), None),
+    (2048, 8192, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), 256),
+    (2048, 4096, 2048, 2176, (FIRST, 256, 256), (FIRST, 256, 256), 256),
+    (2048, 2048, 8192, 8704, (FIRST, 256, 128), (FIRST, 256, 128), 256),
+    (2048, 3072, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), 256),
+    (4096, 4096, 14336, 15360, (SECOND, 160, 256), (FIRST, 256, 256), 64),
 ]
 
 
-@pytest.mark.parametrize("M,N,K,Kp,tile,nrows", ASYM_TILE_CASES, ids=[f"M{c[0]}-N{c[1]}-Kp{c[3]}-{c[4][0]}x{c[4][1]}" for c in ASYM_TILE_CASES])
-def test_tile_shape_zero_point_epilogue_bit_exact(xq, oracle, M, N, K, Kp, tile, nrows):
+@pytest.mark.parametrize("M,N,K,Kp,tile,tile_first,nrows", ASYM_TILE_CASES, ids=[case_id(c) for c in ASYM_TILE_CASES])
+def test_tile_shape_zero_point_epilogue_bit_exact(xq, oracle, M, N, K, Kp, tile, tile_first, nrows):
     """The zero-point term of asymmetric tokens (Sec. 4), sum (u - z) qw, on the same tile shapes."""
     ux = (synth.int4_codes(M, Kp, seed=22, tag=f"ux{M}").astype(np.int16) + 8).astype(np.uint8)
     z = (synth.int4_codes(M, 1, seed=22, tag=f"z{M}").astype(np.int32) + 8)[:, 0].copy()
@@ -102,7 +132,7 @@ def test_tile_shape_zero_point_epilogue_bit_exact(xq, oracle, M, N, K, Kp, tile,
     s_x = synth.scales(M, seed=22, tag="x")
     s_w = synth.scales(N, seed=22, tag="w")
     w = xq.xq_weights_import(qw, s_w, K)
-    assert xq.xq_gemm_kernel_info(M, w) == (TILE_KERNEL, *tile)
+    check_shape(xq.xq_gemm_kernel_info(M, w), tile, tile_first)
     ws = xq.new_workspace(M, w)
     Xq = dev(oracle.pack_int4((ux.astype(np.int16) - 8).astype(np.int8)))
     out = torch.empty((M, N), dtype=torch.int16, device="cuda")
@@ -119,25 +149,26 @@ def test_tile_shape_zero_point_epilogue_bit_exact(xq, oracle, M, N, K, Kp, tile,
     assert np.all(np.abs(got - want) <= np.abs(want) * 2.0**-7 + 1e-30)
 
 
-# (M, N, K, Kp, tile): the largest partial sums the kernel can meet -- every product is (-8)(-8) = 64 or (-8)(7) = -56,
-# times 256 inside the tensor core, over the two longest K' of Table 1.
+# (M, N, K, Kp, shape, shape with the first form forced): the largest partial sums the kernel can meet -- every product
+# is (-8)(-8) = 64 or (-8)(7) = -56, times 256 inside the tensor core, over the two longest K' of Table 1.
 EXTREME_CASES = [
-    (64, 256, 14336, 18432, (256, 128)),
-    (200, 256, 14336, 22016, (256, 128)),
-    (1024, 9472, 14336, 18432, (256, 256)),
-    (1024, 9472, 14336, 22016, (256, 256)),
-    (384, 9728, 14336, 22016, (128, 256)),
-    (512, 14336, 14336, 22016, (256, 224)),
+    (64, 256, 14336, 18432, (SECOND, 64, 256), (FIRST, 256, 128)),
+    (200, 256, 14336, 22016, (SECOND, 128, 256), (FIRST, 256, 128)),
+    (1024, 9472, 14336, 18432, (FIRST, 256, 256), (FIRST, 256, 256)),
+    (1024, 9472, 14336, 22016, (FIRST, 256, 256), (FIRST, 256, 256)),
+    (384, 9728, 14336, 22016, (SECOND, 128, 256), (FIRST, 128, 256)),
+    (512, 14336, 14336, 22016, (FIRST, 256, 224), (FIRST, 256, 224)),
+    (4096, 4096, 14336, 22016, (SECOND, 160, 256), (FIRST, 256, 256)),
 ]
 
 
-@pytest.mark.parametrize("M,N,K,Kp,tile", EXTREME_CASES, ids=[f"M{c[0]}-N{c[1]}-Kp{c[3]}-{c[4][0]}x{c[4][1]}" for c in EXTREME_CASES])
-def test_tile_shape_extreme_codes_closed_form(xq, oracle, M, N, K, Kp, tile):
+@pytest.mark.parametrize("M,N,K,Kp,tile,tile_first", EXTREME_CASES, ids=[case_id((*c, None)) for c in EXTREME_CASES])
+def test_tile_shape_extreme_codes_closed_form(xq, oracle, M, N, K, Kp, tile, tile_first):
     qx = np.full((M, Kp), -8, dtype=np.int8)
     qw = np.full((N, Kp), -8, dtype=np.int8)
     qw[1::3] = 7
     w = xq.xq_weights_import(qw, np.ones(N, np.float32), K)
-    assert xq.xq_gemm_kernel_info(M, w) == (TILE_KERNEL, *tile)
+    check_shape(xq.xq_gemm_kernel_info(M, w), tile, tile_first)
     ws = xq.new_workspace(M, w)
     out = torch.empty((M, N), dtype=torch.int16, device="cuda")
     acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
@@ -162,3 +193,25 @@ def test_i8_mma_rate_probe_runs_and_reports_its_operations(xq):
     ops = xq.xq_selftest_i8_mma_rate(50, ws)
     assert xq.xq_poll_status(ws) == xq.OK
     assert ops == sms * 50 * 4 * 2 * 128 * 256 * 32
+
+
+def rerun_forced(setting):
+    env = dict(os.environ, XQ_PREFILL_KERNEL=setting)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider"],
+                       env=env, cwd=root, capture_output=True, text=True, timeout=3000)
+    assert r.returncode == 0, r.stdout[-4000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout and "failed" not in r.stdout
+
+
+@pytest.mark.skipif(FORCED != "", reason="this is a child run")
+def test_the_same_cases_with_the_first_form_forced():
+    """This file once more in a child process with XQ_PREFILL_KERNEL=ss: the cases that the library gives to the second
+    form by default now run (and are compared with the oracle) on the first form's tile shapes."""
+    rerun_forced("ss")
+
+
+@pytest.mark.skipif(FORCED != "", reason="this is a child run")
+def test_the_same_cases_with_the_second_form_forced():
+    """And with XQ_PREFILL_KERNEL=ts: every case, the small and ragged ones included, on the second form."""
+    rerun_forced("ts")
