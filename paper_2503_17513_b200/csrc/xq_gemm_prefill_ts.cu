@@ -20,7 +20,8 @@
 // out by one tiled TMA store each (which also clips at M and N).  Every MMA accumulates; the epilogue leaves zeros behind.
 //
 // Warps: weight producer (one tiled TMA copy per K block gathers the tile's 16 channel blocks), token producer (TMA),
-// two MMA issuers (one per channel half), 8 epilogue, 8 unpack.  Every wait is time-bounded as in the first form.
+// two MMA issuers (one per channel half), 16 epilogue (the conversion is bound by instruction latency, not by
+// issue slots: twice the warps halve it), 8 unpack.  Every wait is time-bounded as in the first form.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdlib.h>
@@ -38,13 +39,13 @@ constexpr int kTokStageBytes = kMaxTokens * 128;
 constexpr int kPkStageBytes = kChannels * 64;  // packed weights of a K block
 constexpr int kTokStages = 4, kPkStages = 4, kAStages = 2, kDoneRing = 4;
 static_assert(kDoneRing >= kTokStages && kDoneRing >= kAStages, "a waiter must reach its barrier before the ring comes round again");
-constexpr int kEpiWarps = 8, kUnpackWarps = 8, kFirstEpiWarp = 4, kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
+constexpr int kEpiWarps = 16, kUnpackWarps = 8, kFirstEpiWarp = 4, kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
 constexpr int kIssuers = 1;                    // issuing threads per channel half, each with 4 / kIssuers of a K block's K steps
 constexpr int kFirstExtraIssuer = kFirstUnpackWarp + kUnpackWarps;  // issuers beyond the first two sit in warps of their own at the end
 constexpr int kThreads = (kFirstExtraIssuer + 2 * kIssuers - 2) * 32;
 constexpr int kTmemCols = 512, kStagingCol = 384;
 constexpr int kEpiStageBytes = 32 * 32 * 2;  // output stage of an epilogue warp: 32 tokens x 32 channels of bf16
-constexpr int kEpiStages = 3;
+constexpr int kEpiStages = 2;
 constexpr size_t kSmemBytes = 1024 + (size_t)kTokStages * kTokStageBytes + (size_t)kPkStages * kPkStageBytes +
                               (size_t)kEpiWarps * kEpiStages * kEpiStageBytes + 512;
 
@@ -62,12 +63,13 @@ struct TsParams {
   int tiles_m, tiles_n;
 };
 
-// The epilogue of one tile for the channels of (lane quarter q, channel half h): wait for the accumulator, then per
-// chunk of 16 tokens read it, leave zero behind, scale, and put the bf16 values into a small shared-memory stage in
+// The epilogue of one tile for the channels of (lane quarter q, channel half h), the blocks of 32 tokens with index
+// parity r: wait for the accumulator, then per chunk of 16 tokens read it, leave zero behind, scale, and put the bf16
+// values into a small shared-memory stage in
 // output order ([token][channel], 64 bytes per token, 32 tokens), which one tiled TMA store writes out (the store
 // clips at M and N); kEpiStages stages per warp take turns.  At the end the accumulator is handed back.
 __device__ __forceinline__ bool epilogue_part(const TsParams& p, const CUtensorMap* mapO, unsigned char* stages, uint32_t& blk, int tile, uint32_t tcount,
-                                              uint32_t tmem_base, int q, int h, int lane, uint64_t* acc_full, uint64_t* acc_empty,
+                                              uint32_t tmem_base, int q, int h, int r, int lane, uint64_t* acc_full, uint64_t* acc_empty,
                                               volatile int* failed) {
   const int NT = p.NT, tm = tile % p.tiles_m, tn = tile / p.tiles_m;
   const int nw = tn * kChannels + h * 128 + q * 32;  // first channel of this warp
@@ -95,7 +97,7 @@ __device__ __forceinline__ bool epilogue_part(const TsParams& p, const CUtensorM
 #pragma unroll
   for (int i = 0; i < kMaxTokens / 32; ++i) {  // blocks of 32 tokens; unrolled: the scales stay in named registers
     const int c = 32 * i;
-    if (c < c_end) {
+    if ((i & 1) == r && c < c_end) {  // the two warps of a (quarter, half) take the blocks in turn
       unsigned char* stg = stages + (blk++ % kEpiStages) * kEpiStageBytes;  // the stages take turns across tiles too
       if (lane == 0) bulk_wait_group_read<kEpiStages - 1>();  // the store that read this stage kEpiStages blocks ago has done so
       __syncwarp();
@@ -267,12 +269,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
     __syncwarp();
   } else if (warp < kFirstUnpackWarp) {
     // ---------------- epilogue ------------------------------------------------------------------
-    const int q = warp & 3;                      // tensor-memory lane quarter this warp may read
-    const int h = (warp - kFirstEpiWarp) >> 2;   // channel half of the tile
+    const int q = warp & 3;                            // tensor-memory lane quarter this warp may read
+    const int h = ((warp - kFirstEpiWarp) >> 2) & 1;   // channel half of the tile
+    const int r = (warp - kFirstEpiWarp) >> 3;         // which of the blocks of 32 tokens: even or odd
     {  // the accumulator starts at zero: every MMA accumulates
       const uint32_t zeros[16] = {};
       const uint32_t taddr0 = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * NT);
-      for (int c = 0; c < NT; c += 16) tmem_st_32x16(taddr0 + c, zeros);
+      for (int c = 32 * r; c < NT; c += 64) {
+        tmem_st_32x16(taddr0 + c, zeros);
+        tmem_st_32x16(taddr0 + c + 16, zeros);
+      }
       tmem_st_wait();
       tc_fence_before_sync();
       __syncwarp();
@@ -280,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
     }
     uint32_t tcount = 0, blk = 0;
     for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount)
-      if (!epilogue_part(p, &mapO, epi_stages + (size_t)(warp - kFirstEpiWarp) * kEpiStages * kEpiStageBytes, blk, tile, tcount, tmem_base, q, h, lane,
+      if (!epilogue_part(p, &mapO, epi_stages + (size_t)(warp - kFirstEpiWarp) * kEpiStages * kEpiStageBytes, blk, tile, tcount, tmem_base, q, h, r, lane,
                          acc_full, acc_empty, failed))
         break;
     if (lane == 0) bulk_wait_group<0>();  // the output stores have completed before the shared memory goes away
