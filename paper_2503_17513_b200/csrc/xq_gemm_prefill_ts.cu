@@ -61,7 +61,21 @@ struct TsParams {
   int M, N, KB;         // KB = K'' / 128 (K blocks of the padded weights)
   int NT;               // tokens per tile
   int tiles_m, tiles_n;
+  int tn_fast;          // order of the tiles: channel tiles fastest (the CTAs of a wave share few token tiles) or token tiles fastest
 };
+
+// Tile index -> (token tile, channel tile).  The tiles that run at the same time span all of the faster index and a few
+// values of the slower one; the operand indexed by the slower one is fetched from DRAM once, the other once per wave
+// unless it stays in L2: the launcher lets the larger operand be the one fetched once.
+__device__ __forceinline__ void tile_coords(const TsParams& p, int tile, int& tm, int& tn) {
+  if (p.tn_fast) {
+    tn = tile % p.tiles_n;
+    tm = tile / p.tiles_n;
+  } else {
+    tm = tile % p.tiles_m;
+    tn = tile / p.tiles_m;
+  }
+}
 
 // The epilogue of one tile for the channels of (lane quarter q, channel half h), the blocks of 32 tokens with index
 // parity r: wait for the accumulator, then per chunk of 16 tokens read it, leave zero behind, scale, and put the bf16
@@ -71,7 +85,9 @@ struct TsParams {
 __device__ __forceinline__ bool epilogue_part(const TsParams& p, const CUtensorMap* mapO, unsigned char* stages, uint32_t& blk, int tile, uint32_t tcount,
                                               uint32_t tmem_base, int q, int h, int r, int lane, uint64_t* acc_full, uint64_t* acc_empty,
                                               volatile int* failed) {
-  const int NT = p.NT, tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+  const int NT = p.NT;
+  int tm, tn;
+  tile_coords(p, tile, tm, tn);
   const int nw = tn * kChannels + h * 128 + q * 32;  // first channel of this warp
   const int n = nw + lane;                           // this thread's channel
   const int m0 = tm * NT;
@@ -197,7 +213,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-        const int tn = tile / p.tiles_m;
+        int tm, tn;
+        tile_coords(p, tile, tm, tn);
         for (int kb = 0; kb < p.KB; ++kb, ++it) {
           const int s = it % kPkStages;
           if (it >= (uint32_t)kPkStages) {
@@ -253,7 +270,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-        const int tm = tile % p.tiles_m;
+        int tm, tn;
+        tile_coords(p, tile, tm, tn);
         for (int kb = 0; kb < p.KB; ++kb, ++it) {
           const int s = it % kTokStages;
           if (it >= (uint32_t)kTokStages) {  // the MMAs of K block it - kTokStages, which read this stage, have completed
@@ -396,6 +414,7 @@ cudaError_t xq_launch_gemm_prefill_ts(const uint8_t* A8, const float* sx, const 
   p.NT = tile_tokens;
   p.tiles_m = (M + tile_tokens - 1) / tile_tokens;
   p.tiles_n = (w->N + kChannels - 1) / kChannels;
+  p.tn_fast = (size_t)M * w->Kp > (size_t)w->N * w->Kp / 2 ? 1 : 0;  // bytes of the token image against bytes of the weights
   auto kernel = gemm_prefill_ts_kernel;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return e;
