@@ -143,7 +143,8 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_launch_dependents();
+  // the kernel after this one is let in late (by the MMA warp, below): released before this wait it becomes eligible
+  // while the kernel before this one still runs and its waiting CTAs take SMs that this grid needs
   pdl_wait();  // tokens and their scales may come from the kernel before this one
 
   if (warp == 0) {
@@ -213,6 +214,7 @@ __global__ void __launch_bounds__(Cfg<MH, BN>::kThreads, 1) gemm_prefill_kernel(
     }
     // every MMA issued by this warp has completed before tensor memory is released
     if (lane == 0) umma_commit(drain);
+    pdl_launch_dependents();
     __syncwarp();
     mbar_wait_bounded(drain, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);
   } else if (warp == 2) {
@@ -498,8 +500,8 @@ cudaError_t xq_launch_expand_tokens(const uint8_t* Xq, int32_t M, int32_t Kp, ui
 // Second form (expanded weights in tensor memory, xq_gemm_prefill_ts.cu): tiles of NT tokens x 256 channels, NT in
 // {192, 160, 128} or the token count rounded up to 32 when that is less; a K block costs 206 + 92 NT / 192 (the
 // hand-over chain of the two staging stages bounds it, not the tensor pipe), a tile 2400 more (its epilogue is
-// not hidden), a launch 3400 more (inside a layer, behind the rotate kernel, it measured 4-14 us per launch slower
-// than alone, the first form less so): it is taken for the large products, where it is 10-20 % faster.
+// not hidden).  It is taken unless the best shape of the first form is clearly cheaper: measured inside a layer it is
+// 5-10 % faster than the first form at the 1B and 8B prefill shapes and level with it at the smallest ones.
 // Returns 0 for 128 tokens x 256 channels, 1 for 256 x 256, 2 for 256 x 128, 3 for 256 x 224 (first form), 4 for
 // *ts_tokens x 256 in the second form.  XQ_PREFILL_KERNEL in the environment (read once) overrides the choice for
 // measurements and tests: "ss" keeps the first form, "ts" or "ts:<tokens>" forces the second.
@@ -511,9 +513,7 @@ int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms, int* ts_toke
   const int KB = w->Kpp / XQ_K_BLOCK, tm1 = (M + BMH - 1) / BMH, tm2 = (M + 2 * BMH - 1) / (2 * BMH);
   auto waves = [&](int tiles) { return (double)((tiles + sms - 1) / sms); };
   const int m32 = (M + 31) / 32 * 32;
-  auto ts_cost = [&](int nt) {
-    return waves(((M + nt - 1) / nt) * ((w->N + 255) / 256)) * (KB * (206.0 + 92.0 * nt / 192.0) + 2400.0) + 3400.0;
-  };
+  auto ts_cost = [&](int nt) { return waves(((M + nt - 1) / nt) * ((w->N + 255) / 256)) * (KB * (206.0 + 92.0 * nt / 192.0) + 2400.0); };
   int best_nt = m32 < 128 ? m32 : 128;
   double t_ts = ts_cost(best_nt);
   for (int nt = 160; nt <= XQ_TS_MAX_TOKENS && nt <= m32; nt += 32)
@@ -545,7 +545,7 @@ int xq_prefill_tile_choice(int32_t M, const xq_weights* w, int sms, int* ts_toke
     c = 1;
     t_ss = t_2x256;
   }
-  if (force != "ss" && t_ts <= t_ss) return 4;
+  if (force != "ss" && t_ts <= 1.1 * t_ss) return 4;
   return c;
 }
 

@@ -202,7 +202,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_launch_dependents();
+  // The kernel after this one is let in late (by the issuing threads, below), not here: released before this wait it
+  // becomes eligible while the kernel BEFORE this one still runs, and its CTAs (which then only wait) take SMs that
+  // this grid's CTAs need; measured inside a layer, the early release cost 2-5 % of the step.
   pdl_wait();  // tokens and their scales may come from the kernel before this one
 
   if (warp == 0) {
@@ -261,6 +263,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
       }
       // every MMA issued by this thread has completed before tensor memory is released
       umma_commit(drain);
+      pdl_launch_dependents();  // the next kernel's CTAs may take the SMs as this grid's CTAs leave them
     }
     __syncwarp();
     if (warp == 1) mbar_wait_bounded(drain, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);

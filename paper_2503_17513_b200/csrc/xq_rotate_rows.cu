@@ -64,7 +64,6 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
   int8_t* sq = chi2 + 2 * q + 1;
 
   if (pl.p > 1) build_chi(q, chi2, sq, pl.paley_kind);
-  xqptx::pdl_launch_dependents();
   // H_p^T: row a' (output index), column a (input index); zero outside p x p
   for (int i = tid; i < MT * 16 * KS * 16; i += blockDim.x) {
     const int a2 = i / (KS * 16), a = i - a2 * (KS * 16);
@@ -79,6 +78,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
   for (int i = tid; i < G * nbuf * KS * 16 * xpitch / 8; i += blockDim.x) reinterpret_cast<uint4*>(Xs_all)[i] = make_uint4(0, 0, 0, 0);
   xqptx::pdl_wait();
   __syncthreads();
+  // only now may the kernel after this one be scheduled: released before the wait it would become eligible while the
+  // kernel before this one still runs, and its waiting CTAs would take SMs that this grid needs
+  xqptx::pdl_launch_dependents();
   if (group >= G) return;
 
   __nv_bfloat16* Xs = Xs_all + (size_t)group * nbuf * KS * 16 * xpitch;

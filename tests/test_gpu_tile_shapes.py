@@ -68,12 +68,12 @@ def sample_rows(M, count, seed=13):
 # (M, N, K, Kp, shape the library must report, shape with the first form forced, token rows compared: None = all)
 TILE_CASES = [
     (384, 9728, 250, 256, (FIRST, 128, 256), (FIRST, 128, 256), None),
-    (2048, 8192, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), None),     # gate / up of the 1B prefill workload: ragged last tiles
+    (2048, 8192, 2048, 2176, (SECOND, 160, 256), (FIRST, 256, 224), None),    # gate / up of the 1B prefill workload: ragged last tiles
     (2048, 4096, 2048, 2176, (FIRST, 256, 256), (FIRST, 256, 256), None),
     (512, 14336, 4096, 4352, (FIRST, 256, 224), (FIRST, 256, 224), None),     # all channels of the 8B gate / up (64 x 224)
-    (2048, 2048, 8192, 8704, (FIRST, 256, 128), (FIRST, 256, 128), None),     # down of the 1B prefill workload
-    (2048, 3072, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), None),     # qkv of the 1B prefill workload
-    (40, 520, 4096, 4352, (FIRST, 256, 128), (FIRST, 256, 128), None),        # one ragged token tile, ragged channels
+    (2048, 2048, 8192, 8704, (SECOND, 128, 256), (FIRST, 256, 128), None),    # down of the 1B prefill workload
+    (2048, 3072, 2048, 2176, (SECOND, 192, 256), (FIRST, 256, 224), None),    # qkv of the 1B prefill workload: 2048 = 10 x 192 + 128
+    (40, 520, 4096, 4352, (SECOND, 64, 256), (FIRST, 256, 128), None),        # one ragged token tile, ragged channels
     (4096, 14336, 4096, 4352, (SECOND, 192, 256), (FIRST, 256, 224), 64),     # the 8B prefill launches as the benchmark times them
     (4096, 6144, 4096, 4352, (SECOND, 192, 256), (FIRST, 256, 256), 64),
     (4096, 4096, 14336, 15360, (SECOND, 160, 256), (FIRST, 256, 256), 64),
@@ -115,10 +115,10 @@ def test_tile_shape_accumulators_bit_exact(xq, oracle, M, N, K, Kp, tile, tile_f
 
 ASYM_TILE_CASES = [
     (384, 9728, 250, 256, (FIRST, 128, 256), (FIRST, 128, 256), None),
-    (2048, 8192, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), 256),
+    (2048, 8192, 2048, 2176, (SECOND, 160, 256), (FIRST, 256, 224), 256),
     (2048, 4096, 2048, 2176, (FIRST, 256, 256), (FIRST, 256, 256), 256),
-    (2048, 2048, 8192, 8704, (FIRST, 256, 128), (FIRST, 256, 128), 256),
-    (2048, 3072, 2048, 2176, (FIRST, 256, 224), (FIRST, 256, 224), 256),
+    (2048, 2048, 8192, 8704, (SECOND, 128, 256), (FIRST, 256, 128), 256),
+    (2048, 3072, 2048, 2176, (SECOND, 192, 256), (FIRST, 256, 224), 256),
     (4096, 4096, 14336, 15360, (SECOND, 160, 256), (FIRST, 256, 256), 64),
 ]
 
@@ -154,8 +154,8 @@ def test_tile_shape_zero_point_epilogue_bit_exact(xq, oracle, M, N, K, Kp, tile,
 EXTREME_CASES = [
     (64, 256, 14336, 18432, (SECOND, 64, 256), (FIRST, 256, 128)),
     (200, 256, 14336, 22016, (SECOND, 128, 256), (FIRST, 256, 128)),
-    (1024, 9472, 14336, 18432, (FIRST, 256, 256), (FIRST, 256, 256)),
-    (1024, 9472, 14336, 22016, (FIRST, 256, 256), (FIRST, 256, 256)),
+    (1024, 9472, 14336, 18432, (SECOND, 128, 256), (FIRST, 256, 256)),
+    (1024, 9472, 14336, 22016, (SECOND, 128, 256), (FIRST, 256, 256)),
     (384, 9728, 14336, 22016, (SECOND, 128, 256), (FIRST, 128, 256)),
     (512, 14336, 14336, 22016, (FIRST, 256, 224), (FIRST, 256, 224)),
     (4096, 4096, 14336, 22016, (SECOND, 160, 256), (FIRST, 256, 256)),
