@@ -205,7 +205,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
   // The kernel after this one is let in late (by the issuing threads, below), not here: released before this wait it
   // becomes eligible while the kernel BEFORE this one still runs, and its CTAs (which then only wait) take SMs that
   // this grid's CTAs need; measured inside a layer, the early release cost 2-5 % of the step.
-  pdl_wait();  // tokens and their scales may come from the kernel before this one
+  // What the kernel before this one writes are the tokens and their scales (and zero points): the token producer and the
+  // epilogue warps wait for it (pdl_wait) before their first access; the weights are constants, so their copies, the
+  // unpack warps and the staging of the first K blocks start at once.
 
   if (warp == 0) {
     // ---------------- weight producer -----------------------------------------------------------
@@ -269,6 +271,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
     if (warp == 1) mbar_wait_bounded(drain, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);
   } else if (warp == 2) {
     // ---------------- token producer ------------------------------------------------------------
+    pdl_wait();
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
@@ -290,6 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
     __syncwarp();
   } else if (warp < kFirstUnpackWarp) {
     // ---------------- epilogue ------------------------------------------------------------------
+    pdl_wait();  // before the first read of a token scale; also orders this kernel's completion after its predecessor's
     const int q = warp & 3;                            // tensor-memory lane quarter this warp may read
     const int h = ((warp - kFirstEpiWarp) >> 2) & 1;   // channel half of the tile
     const int r = (warp - kFirstEpiWarp) >> 3;         // which of the blocks of 32 tokens: even or odd

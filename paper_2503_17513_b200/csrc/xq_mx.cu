@@ -214,7 +214,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_launch_dependents();
+  // the kernel after this one is let in late (by the MMA warp, below): released before this wait it becomes eligible
+  // while the kernel before this one still runs and its waiting CTAs take SMs that this grid needs
   pdl_wait();  // tokens and their scales come from the kernel before this one
 
   if (warp == 0) {
@@ -288,6 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
       __syncwarp();
     }
     if (lane == 0) umma_commit(drain);
+    pdl_launch_dependents();
     __syncwarp();
     mbar_wait_bounded(drain, 0, failed, p.status, (int)XQ_ERR_TIMEOUT);
   } else {
