@@ -314,6 +314,12 @@ cudaError_t launch_rows(const void* X, int32_t M, int64_t ldx, const xq_hadamard
   const size_t fixed = (size_t)MT * 16 * (KS * 16 + 8) * 2 + 32 * 4 + (size_t)(3 * pl.q + 1) + 64;
   size_t per_group = (size_t)2 * KS * 16 * (n + 8) * 2 + (size_t)Wr * 8 * (n + 8) * 4 + (size_t)Wr * 8;
   while (G > 1 && fixed + G * per_group > 224 * 1024) --G;
+  // fewer row groups than multiprocessors: spread the rows over all of them instead (2048 rows in groups of 16 are 128
+  // CTAs on 148 SMs; in groups of 14 they are 147)
+  if (G > 1 && (M + G - 1) / G < sms) {
+    const int g2 = (M + sms - 1) / sms;
+    if (g2 >= 1 && g2 < G) G = g2;
+  }
   if (fixed + G * per_group > 224 * 1024) {  // one row group and still too much: a single stage
     nbuf = 1;
     per_group -= (size_t)KS * 16 * (n + 8) * 2;
