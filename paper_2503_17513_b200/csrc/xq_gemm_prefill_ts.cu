@@ -202,9 +202,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // The kernel after this one is let in late (by the issuing threads, below), not here: released before this wait it
-  // becomes eligible while the kernel BEFORE this one still runs, and its CTAs (which then only wait) take SMs that
-  // this grid's CTAs need; measured inside a layer, the early release cost 2-5 % of the step.
+  // The kernel after this one is let in late (by the issuing threads, below), not here: released here, it is resident
+  // and waiting (and has released its own successor in turn) while this grid still has all its tiles ahead; measured
+  // inside a layer (rotate, product, rotate, ...), the early release cost 2-5 % of the step.
   // What the kernel before this one writes are the tokens and their scales (and zero points): the token producer and the
   // epilogue warps wait for it (pdl_wait) before their first access; the weights are constants, so their copies, the
   // unpack warps and the staging of the first K blocks start at once.

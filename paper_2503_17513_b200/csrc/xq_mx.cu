@@ -214,8 +214,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mx_kernel(const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // the kernel after this one is let in late (by the MMA warp, below): released before this wait it becomes eligible
-  // while the kernel before this one still runs and its waiting CTAs take SMs that this grid needs
+  // the kernel after this one is let in late (by the MMA warp, below): released here, at the start, it cost 1-5 % of a
+  // layer's step (measured)
   pdl_wait();  // tokens and their scales come from the kernel before this one
 
   if (warp == 0) {

@@ -78,8 +78,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1)
   for (int i = tid; i < G * nbuf * KS * 16 * xpitch / 8; i += blockDim.x) reinterpret_cast<uint4*>(Xs_all)[i] = make_uint4(0, 0, 0, 0);
   xqptx::pdl_wait();
   __syncthreads();
-  // only now may the kernel after this one be scheduled: released before the wait it would become eligible while the
-  // kernel before this one still runs, and its waiting CTAs would take SMs that this grid needs
+  // only now may the kernel after this one be scheduled (not before the wait: a chain in which every kernel releases its
+  // successor before its own wait measured 2-5 % slower per layer)
   xqptx::pdl_launch_dependents();
   if (group >= G) return;
 
