@@ -195,6 +195,43 @@ def test_i8_mma_rate_probe_runs_and_reports_its_operations(xq):
     assert ops == sms * 50 * 4 * 2 * 128 * 256 * 32
 
 
+# (M, N, K'): small and odd products -- one K block, eight channels, token counts around the tile sizes of both forms.
+# Whatever the library picks for them (the child runs force each form in turn), the sums are exact.
+SMALL_CASES = [
+    (33, 8, 32), (40, 16, 64), (64, 24, 96), (65, 64, 128), (96, 120, 160), (127, 248, 256), (128, 256, 288), (129, 264, 384),
+    (191, 504, 1024), (192, 512, 1152), (193, 520, 2176), (200, 1000, 32), (255, 1032, 64), (256, 8, 2176), (257, 264, 96),
+    (300, 120, 1152), (383, 520, 128), (385, 24, 1024), (500, 248, 160), (777, 64, 288), (1000, 16, 384),
+]
+
+
+@pytest.mark.parametrize("asym", [False, True], ids=["sym", "asym"])
+@pytest.mark.parametrize("M,N,Kp", SMALL_CASES)
+def test_small_and_odd_products_bit_exact(xq, oracle, M, N, Kp, asym):
+    qx = synth.int4_codes(M, Kp, seed=23, tag=f"sx{M}_{Kp}")
+    qw = synth.int4_codes(N, Kp, seed=23, tag=f"sw{N}_{Kp}")
+    s_x = synth.scales(M, seed=23, tag="x")
+    s_w = synth.scales(N, seed=23, tag="w")
+    w = xq.xq_weights_import(qw, s_w, Kp)
+    info = xq.xq_gemm_kernel_info(M, w)
+    assert info[0] in (FIRST, SECOND) and (FORCED != "ss" or info[0] == FIRST) and (FORCED != "ts" or info[0] == SECOND)
+    ws = xq.new_workspace(M, w)
+    out = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    Xq = dev(oracle.pack_int4(qx))
+    if asym:
+        z = (np.arange(M, dtype=np.int32) % 5) - 2  # zero points of the codes as stored (the unsigned code minus 8)
+        xq.xq_w4a4_gemm_asym(Xq, dev(s_x), dev(z), M, w, out, ws, acc=acc)
+        acc_ref = oracle.gemm_i64(qx, qw) - z[:, None].astype(np.int64) * qw.astype(np.int64).sum(axis=1)[None, :]
+    else:
+        xq.xq_w4a4_gemm(Xq, dev(s_x), M, w, out, ws, acc=acc)
+        acc_ref = oracle.gemm_i64(qx, qw)
+    assert xq.xq_poll_status(ws) == xq.OK
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    want = synth.bf16_bits_to_f32(oracle.epilogue(acc_ref, s_x, s_w)).astype(np.float64)
+    got = synth.bf16_bits_to_f32(host_u16(out)).astype(np.float64)
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0**-7 + 1e-30)  # one bf16 ulp
+
+
 def rerun_forced(setting):
     env = dict(os.environ, XQ_PREFILL_KERNEL=setting)
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
