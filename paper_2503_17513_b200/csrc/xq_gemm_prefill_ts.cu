@@ -40,9 +40,7 @@ constexpr int kPkStageBytes = kChannels * 64;  // packed weights of a K block
 constexpr int kTokStages = 4, kPkStages = 4, kAStages = 2, kDoneRing = 4;
 static_assert(kDoneRing >= kTokStages && kDoneRing >= kAStages, "a waiter must reach its barrier before the ring comes round again");
 constexpr int kEpiWarps = 16, kUnpackWarps = 8, kFirstEpiWarp = 4, kFirstUnpackWarp = kFirstEpiWarp + kEpiWarps;
-constexpr int kIssuers = 1;                    // issuing threads per channel half, each with 4 / kIssuers of a K block's K steps
-constexpr int kFirstExtraIssuer = kFirstUnpackWarp + kUnpackWarps;  // issuers beyond the first two sit in warps of their own at the end
-constexpr int kThreads = (kFirstExtraIssuer + 2 * kIssuers - 2) * 32;
+constexpr int kThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;
 constexpr int kTmemCols = 512, kStagingCol = 384;
 constexpr int kEpiStageBytes = 32 * 32 * 2;  // output stage of an epilogue warp: 32 tokens x 32 channels of bf16
 constexpr int kEpiStages = 2;
@@ -50,13 +48,11 @@ constexpr size_t kSmemBytes = 1024 + (size_t)kTokStages * kTokStageBytes + (size
                               (size_t)kEpiWarps * kEpiStages * kEpiStageBytes + 512;
 
 struct TsParams {
-  const uint8_t* W;     // block layout
   const float* sw;
   const float* sx;
   const int32_t* zp;    // per-token zero points of asymmetric activation codes, or null
   const int32_t* wsum;  // per-channel sums of the weight codes
-  __nv_bfloat16* out;
-  int32_t* acc_opt;
+  int32_t* acc_opt;     // int32 sums for the tests, or null (the bf16 output goes through the output tensor map)
   int32_t* status;
   int M, N, KB;         // KB = K'' / 128 (K blocks of the padded weights)
   int NT;               // tokens per tile
@@ -183,11 +179,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
       mbar_init(&pk_empty[s], kUnpackWarps);
     }
     for (int s = 0; s < kTokStages; ++s) mbar_init(&tok_full[s], 1);
-    for (int s = 0; s < kDoneRing; ++s) mbar_init(&mma_done[s], 2 * kIssuers);
+    for (int s = 0; s < kDoneRing; ++s) mbar_init(&mma_done[s], 2);
     for (int s = 0; s < kAStages; ++s) mbar_init(&a_full[s], kUnpackWarps);
-    mbar_init(acc_full, 2 * kIssuers);
+    mbar_init(acc_full, 2);
     mbar_init(acc_empty, kEpiWarps);
-    mbar_init(drain, 2 * kIssuers);
+    mbar_init(drain, 2);
     *failed = 0;
     mbar_fence_init();
     tma_prefetch_desc(&mapX);
@@ -231,14 +227,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
       }
     }
     __syncwarp();
-  } else if (warp == 1 || warp == 3 || warp >= kFirstExtraIssuer) {
+  } else if (warp == 1 || warp == 3) {
     // ---------------- MMA issue -----------------------------------------------------------------
-    // 2 x kIssuers issuing threads, each with one channel half and 4 / kIssuers of the K steps of every K block (one
-    // thread for both halves needs longer per K block than the tensor pipe; more than one per half measured no
-    // better).  Instructions of different threads are not ordered among themselves: every one accumulates, and the
-    // epilogue leaves the accumulator zeroed.  The completion barriers count all issuers.
-    const int g = warp == 1 ? 0 : (warp == 3 ? 1 : warp - kFirstExtraIssuer + 2);
-    const int h = g / kIssuers, k0 = (g % kIssuers) * (4 / kIssuers);
+    // two issuing threads, one per channel half (one thread for both needs longer per K block than the tensor pipe;
+    // two per half measured no better).  The two threads' instructions are not ordered among themselves and need not
+    // be: they write different accumulators; every instruction accumulates, the epilogue leaves the accumulator zeroed.
+    // The completion barriers count both.
+    const int h = warp == 1 ? 0 : 1;
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_s8(128, NT);
       const uint32_t d_tmem = tmem_base + (uint32_t)(h * NT);
@@ -255,10 +250,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
                mbar_wait_bounded(&a_full[u], (it / kAStages) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint64_t bdesc = umma_desc_k128(smem_u32(tok + (size_t)s * kTokStageBytes)) + 2 * k0;
-          const uint32_t a_tmem = tmem_base + (uint32_t)(kStagingCol + u * 64 + h * 32 + 8 * k0);
+          const uint64_t bdesc = umma_desc_k128(smem_u32(tok + (size_t)s * kTokStageBytes));
+          const uint32_t a_tmem = tmem_base + (uint32_t)(kStagingCol + u * 64 + h * 32);
 #pragma unroll
-          for (int k = 0; k < 4 / kIssuers; ++k) umma_i8_ts(d_tmem, a_tmem + 8 * k, bdesc + 2 * k, idesc, 1u);
+          for (int k = 0; k < 4; ++k) umma_i8_ts(d_tmem, a_tmem + 8 * k, bdesc + 2 * k, idesc, 1u);
           umma_commit(&mma_done[it % kDoneRing]);
         }
         if (ok) umma_commit(acc_full);
@@ -343,9 +338,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
           split16(v[t].z, r[8 * t + 4], r[8 * t + 5]);
           split16(v[t].w, r[8 * t + 6], r[8 * t + 7]);
         }
-        // the packed stage is in registers: hand it back before waiting for the staging area
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&pk_empty[s]);
         if (it >= (uint32_t)kAStages) {  // the MMAs that read this staging stage kAStages K blocks ago have completed
           const uint32_t j = it - kAStages;
           ok = mbar_wait_bounded(&mma_done[j % kDoneRing], (j / kDoneRing) & 1, failed, p.status, (int)XQ_ERR_TIMEOUT);
@@ -356,7 +348,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_prefill_ts_kernel(const __gr
         tmem_st_wait();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&a_full[u]);
+        // The packed stage goes back only here, after the expanded words have been used: every lane's loads from it
+        // have then certainly returned.  (Handing it back right after issuing the loads let a copy into the stage
+        // overtake a load still in flight about once in 10^5 tiles: eight channels of one K block read the wrong bytes.)
+        if (lane == 0) {
+          mbar_arrive(&a_full[u]);
+          mbar_arrive(&pk_empty[s]);
+        }
       }
     }
   }
@@ -407,12 +405,10 @@ cudaError_t xq_launch_gemm_prefill_ts(const uint8_t* A8, const float* sx, const 
                         CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
   TsParams p;
-  p.W = w->packed;
   p.sw = w->s_w;
   p.sx = sx;
   p.zp = zp;
   p.wsum = w->w_sum;
-  p.out = (__nv_bfloat16*)out;
   p.acc_opt = acc_opt;
   p.status = status;
   p.M = M;
