@@ -62,9 +62,9 @@ FALLBACK_BF16_TFLOPS = (1590.0, 1400.0)
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     ("1b-decode", 32): (6.58e6, "profiles/gemm_decode_1b_decode_m32.txt"),
     ("8b-decode", 16): ((13.47 + 31.32 + 31.32 + 31.49) * 1e6 / 4, "profiles/gemm_decode_8b_decode_m16.txt"),
-    ("8b-prefill", 4096): ((31.331840 + 7.592192 + 49.277184 + 74.973184 + 49.368064 + 74.533888 + 105.622784 + 18.824192) * 1e6 / 4,
+    ("8b-prefill", 4096): ((31.332352 + 8.125440 + 49.274368 + 75.311360 + 49.238016 + 74.736640 + 106.173952 + 18.625792) * 1e6 / 4,
                            "profiles/gemm_prefill_8b_prefill_m4096.txt"),
-    ("1b-prefill", 2048): ((7.913984 + 0.000000 + 6.732800 + 0.000000 + 13.496576 + 0.054528 + 13.496576 + 0.015104 + 26.833408 + 0.000000) * 1e6 / 5,
+    ("1b-prefill", 2048): ((7.913984 + 0.000000 + 6.732544 + 0.000000 + 13.496832 + 0.048640 + 13.496832 + 0.034816 + 26.833408 + 0.000000) * 1e6 / 5,
                            "profiles/gemm_prefill_1b_prefill_m2048.txt"),
 }
 
